@@ -1,0 +1,195 @@
+/* bsp.h — C ABI of the block-structured-pruning library for NVIDIA B200 (sm_100a).
+ *
+ * The library implements, on one GPU, the computations of
+ *   Li, Kong et al., "Efficient Transformer-based Large Scale Language Representations using
+ *   Hardware-friendly Block Structured Pruning", EMNLP-Findings 2020:
+ * per-group l2 norms with the reweighted group-Lasso penalty and its gamma update (Section 3.2,
+ * Eq. 2 and Eq. 3), threshold pruning of the groups (Algorithm 1) into a compressed
+ * block-structured storage (Section 3.1), and the linear layer Y = act(X W^T + b) evaluated on
+ * the pruned weight (the computation the pruning is meant to speed up, Sections 3.1 and 4.4).
+ *
+ * Conventions shared by every call
+ * --------------------------------
+ *  - W is one linear layer's weight, [rows = N_out, cols = K_in], row-major bf16 with leading
+ *    dimension ldw (elements).  X is [tokens, K_in] bf16 row-major (ldx), Y is [tokens, N_out]
+ *    bf16 row-major (ldy).
+ *  - Orientation BSP_ORIENT_C (Eq. 3): W is cut into rows/block row-blocks of `block`
+ *    consecutive rows; a group is one column of one row-block.  Per-group arrays are
+ *    [rows/block, cols] row-major.  A "block" owns `cols` groups.
+ *    Orientation BSP_ORIENT_R (Algorithm 1 as printed, Eq. 2): W is cut into cols/block vertical
+ *    strips of `block` consecutive columns; a group is one row of one strip.  Per-group arrays
+ *    are [rows, cols/block] row-major.  A "block" (strip) owns `rows` groups.
+ *  - All data pointers are DEVICE pointers unless a parameter says "host".  The caller owns every
+ *    buffer; the library allocates no device memory.  `stream` is a cudaStream_t passed as
+ *    void* (NULL = the legacy default stream).  Calls enqueue work on `stream` and return
+ *    without synchronising; outputs are valid once the stream has reached that point.
+ *  - Every function returns BSP_OK (0) or a negative bsp_status.  Argument and shape errors are
+ *    detected on the host before anything is launched.  Nothing aborts or throws.
+ *  - Inputs must be finite (no NaN/Inf weights).
+ */
+#ifndef BSP_H_
+#define BSP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  BSP_OK = 0,
+  BSP_ERR_ARG = -1,         /* null pointer, negative size, unknown enum value, misaligned buffer */
+  BSP_ERR_SHAPE = -2,       /* block does not divide rows (C) / cols (R); leading dimension too small */
+  BSP_ERR_WORKSPACE = -3,   /* workspace smaller than the matching *_bound / *_bytes query says   */
+  BSP_ERR_CUDA = -4,        /* a CUDA runtime or driver call failed (see bsp_last_cuda_error)     */
+  BSP_ERR_TIMEOUT = -5,     /* a bounded device-side wait expired (reported by bsp_linear_status) */
+  BSP_ERR_UNSUPPORTED = -6  /* size beyond a documented limit                                     */
+} bsp_status;
+
+typedef enum { BSP_ORIENT_C = 0, BSP_ORIENT_R = 1 } bsp_orient;
+typedef enum { BSP_PEN_L2 = 0, BSP_PEN_L2SQ = 1 } bsp_penalty;
+typedef enum { BSP_ACT_NONE = 0, BSP_ACT_GELU = 1 } bsp_act;
+
+/* Human-readable name of a status code (static string, host). */
+const char* bsp_status_string(int status);
+/* Last CUDA error code seen by the calling thread inside this library (0 if none); host. */
+int bsp_last_cuda_error(void);
+
+/* ---------------------------------------------------------------------------------------------
+ * bsp_group_norms — Section 3.2: the square-rooted sums of Eq. 2 / Eq. 3 (the `l2_norms(i,j)` of
+ * Algorithm 1), the gamma update printed under each equation, and the regulariser's value.
+ *
+ *   S_g  = sum of squares of group g (float32, elements added in increasing index order)
+ *   n_g  = sqrt(S_g)                                      -> norms      (if non-NULL)
+ *   BSP_PEN_L2   (the paper's form):
+ *       gamma_g = 1 / (n_g + eps)                         -> gamma_out  (if non-NULL)
+ *       penalty = sum_g gamma'_g * n_g                    -> *penalty   (if non-NULL)
+ *   BSP_PEN_L2SQ (squared-norm variant of the same update):
+ *       alpha_g = 1 / (S_g + eps)                         -> gamma_out
+ *       penalty = sum_g alpha'_g * S_g                    -> *penalty
+ *   gamma' (alpha') is gamma_in if it is non-NULL (weights kept from an earlier milestone of
+ *   Algorithm 2), else the value just computed from this W.  Pass gamma_in = NULL and read
+ *   sum n_g/(n_g+eps); for the plain group-Lasso term (gamma == 1) pass a gamma_in of ones.
+ *   The factor lambda of Eq. 2 / Eq. 3 is left to the caller.
+ *
+ * norms, gamma_in, gamma_out: float32 per-group arrays (shape by orientation, see above).
+ * penalty: one float64 device scalar; it is overwritten, not accumulated.  It is summed with
+ * float64 atomics, so its last bits may differ between runs.
+ * Errors: BSP_ERR_ARG (W NULL, all outputs NULL, bad enum, eps < 0), BSP_ERR_SHAPE.
+ */
+int bsp_group_norms(const void* W, int rows, int cols, int ldw, int block, int orient,
+                    float eps, int pen,
+                    float* norms, const float* gamma_in, float* gamma_out, double* penalty,
+                    void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * bsp_pack_bound — host-only size query for bsp_prune_pack (worst case: nothing pruned).
+ *   *idx_elems = number of int32 index entries, *val_elems = number of bf16 values,
+ *   *ws_bytes  = workspace bytes bsp_prune_pack / bsp_percentile_threshold need for this shape.
+ * Any of the three output pointers may be NULL.
+ */
+int bsp_pack_bound(int rows, int cols, int block, int orient,
+                   size_t* idx_elems, size_t* val_elems, size_t* ws_bytes);
+
+/* ---------------------------------------------------------------------------------------------
+ * bsp_prune_pack — Algorithm 1 followed by the compressed storage of Section 3.1 ("only the
+ * non-zero rows/columns at the block level need to be indexed").
+ *
+ * Decision (Algorithm 1 prunes a group iff its l2 norm <= t_b): group g is KEPT iff
+ *   S_g > t_b * t_b, both sides float32, S_g as defined for bsp_group_norms; a negative t_b
+ *   keeps everything.  t_b = 0 keeps exactly the groups holding a non-zero weight, i.e. the
+ *   group-level form of Algorithm 2's Mask = (W != 0).
+ *   t_b is `threshold`, or the device scalar *threshold_dev if that pointer is non-NULL (so
+ *   that bsp_percentile_threshold can feed it without a host round trip).
+ *   If keep_per_block >= 0 the threshold is ignored and exactly keep_per_block groups are kept
+ *   in every block: the largest S_g, ties broken towards the lower group index (needs at most
+ *   BSP_TOPK_MAX_GROUPS groups per block, else BSP_ERR_UNSUPPORTED).
+ *
+ * Outputs (canonical packed form; nb = number of blocks, kc_b = kept groups of block b):
+ *   keep        uint8 per-group flags (1 = kept), per-group array shape; may be NULL
+ *   blk_ptr     int32 [nb + 1], blk_ptr[b] = number of kept groups in blocks before b
+ *   idx         int32 [blk_ptr[nb]]: for each block its kept group indices (column indices for
+ *               C, row indices for R), strictly ascending
+ *   vals        bf16: for each block in order one dense tile copied bit for bit from W, at
+ *               element offset block * blk_ptr[b]:  C: [block, kc_b] row-major (row r of the
+ *               row-block, kept columns in order);  R: [kc_b, block] row-major
+ *   kept_weights int64 device scalar = block * blk_ptr[nb]; compression rate = rows*cols / it.
+ *               May be NULL.
+ * idx and vals must have room for bsp_pack_bound's counts.  ws/ws_bytes: scratch of at least
+ * bsp_pack_bound's *ws_bytes, 256-byte aligned; contents are undefined afterwards.
+ * Errors: BSP_ERR_ARG, BSP_ERR_SHAPE, BSP_ERR_WORKSPACE, BSP_ERR_UNSUPPORTED.
+ */
+#define BSP_TOPK_MAX_GROUPS 8192
+int bsp_prune_pack(const void* W, int rows, int cols, int ldw, int block, int orient,
+                   float threshold, const float* threshold_dev, int keep_per_block,
+                   uint8_t* keep, int32_t* blk_ptr, int32_t* idx, void* vals,
+                   int64_t* kept_weights, void* ws, size_t ws_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * bsp_percentile_threshold — Section 3.1: "prune ... according to our pre-set threshold or
+ * percentile".  Per-matrix threshold for a target compression rate c = total/kept:
+ * with G groups, r = floor(G * (1 - 1/c)) groups are to be removed; *threshold_out (device
+ * float) receives t_b = the float32 square root of the r-th smallest S_g, raised by single ulps
+ * until t_b * t_b >= that S_g, so that Algorithm 1's `<=` removes that group and its ties.
+ * r = 0 gives -1 (prune nothing).  ws as for bsp_prune_pack.
+ * Errors: BSP_ERR_ARG (rate < 1), BSP_ERR_SHAPE, BSP_ERR_WORKSPACE.
+ */
+int bsp_percentile_threshold(const void* W, int rows, int cols, int ldw, int block, int orient,
+                             double rate, float* threshold_out,
+                             void* ws, size_t ws_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * bsp_apply_mask — Algorithm 2's retraining step W = W * Mask, with the mask given per group:
+ * every element of a group whose keep flag is 0 is set to +0, in place.
+ */
+int bsp_apply_mask(void* W, int rows, int cols, int ldw, int block, int orient,
+                   const uint8_t* keep, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * bsp_linear — the pruned linear layer (orientation C packed form):
+ *   Y[t, b*block + r] = act( sum_{j < kc_b} X[t, idx_b[j]] * vals_b[r, j] + bias[b*block + r] )
+ * which equals act(X (W * Mask)^T + bias), the layer Algorithm 2 retrains (W = W * Mask) and
+ * Sections 3.1 / 4.4 deploy.  Products are bf16 x bf16 accumulated in float32 on the tensor
+ * cores; bias (bf16 [n_out], may be NULL) is added in float32; act is BSP_ACT_NONE or
+ * BSP_ACT_GELU (0.5 x (1 + erf(x / sqrt 2)), evaluated in float32); the result is rounded to
+ * bf16 (nearest even).
+ *
+ * bsp_linear_plan_bytes (host): bytes of the private execution layout for a packed matrix.
+ * bsp_linear_plan: builds that layout in `plan` (device, 256-byte aligned) from the canonical
+ *   packed form; do it once per packed matrix, reuse for any number of bsp_linear_planned calls.
+ * bsp_linear_planned: runs the layer from a plan.
+ * bsp_linear: plan + run in one call, the plan living in ws (>= bsp_linear_plan_bytes).
+ *
+ * Alignment for the tensor-core path: X, Y and plan 16-byte aligned, k_in, ldx and ldy multiples
+ * of 8 elements.  Other cases run on a slower CUDA-core kernel with identical semantics.
+ * Device-side waits in the tensor-core kernel are bounded; if one expires the kernel stops
+ * early and records it: bsp_linear_status (host; synchronises the stream) then returns
+ * BSP_ERR_TIMEOUT and Y is undefined.  It returns BSP_OK otherwise.
+ * Errors: BSP_ERR_ARG, BSP_ERR_SHAPE (block does not divide n_out), BSP_ERR_WORKSPACE, BSP_ERR_CUDA.
+ */
+int bsp_linear_plan_bytes(int n_out, int k_in, int block, size_t* bytes);
+int bsp_linear_plan(const int32_t* blk_ptr, const int32_t* idx, const void* vals,
+                    int n_out, int k_in, int block, void* plan, size_t plan_bytes, void* stream);
+int bsp_linear_planned(const void* plan, int n_out, int k_in, int block,
+                       const void* X, int tokens, int ldx, const void* bias, int act,
+                       void* Y, int ldy, void* stream);
+int bsp_linear(const int32_t* blk_ptr, const int32_t* idx, const void* vals,
+               int n_out, int k_in, int block,
+               const void* X, int tokens, int ldx, const void* bias, int act,
+               void* Y, int ldy, void* ws, size_t ws_bytes, void* stream);
+int bsp_linear_status(void* stream);
+
+/* bsp_linear_cuda_core — the same layer computed straight from the packed form by a plain
+ * CUDA-core kernel (one thread per output, float32 accumulation in index order).  It is what
+ * bsp_linear falls back to when the alignment rules above do not hold, and is exported so the
+ * two paths can be compared.  No workspace. */
+int bsp_linear_cuda_core(const int32_t* blk_ptr, const int32_t* idx, const void* vals,
+                         int n_out, int k_in, int block,
+                         const void* X, int tokens, int ldx, const void* bias, int act,
+                         void* Y, int ldy, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BSP_H_ */

@@ -1,0 +1,15 @@
+"""Block-structured pruning for BERT-family linear layers on NVIDIA B200 (sm_100a).
+
+Thin Python binding over the C-ABI CUDA library `libbsp.so` (declared in include/bsp.h).
+Every computation runs in the library's kernels; this package only marshals arguments.
+torch is used for device memory and streams.
+"""
+from .binding import (  # noqa: F401
+    BspError,
+    ORIENT_C, ORIENT_R, PEN_L2, PEN_L2SQ, ACT_NONE, ACT_GELU,
+    PackedMatrix,
+    lib, library_path,
+    bsp_group_norms, bsp_pack_bound, bsp_prune_pack, bsp_percentile_threshold, bsp_apply_mask,
+    bsp_linear_plan_bytes, bsp_linear_plan, bsp_linear_planned, bsp_linear, bsp_linear_status,
+    bsp_linear_cuda_core, bsp_status_string,
+)

@@ -1,0 +1,207 @@
+"""ctypes binding of libbsp.so.  Same names as the C entry points; arguments are torch CUDA
+tensors (or None) whose device pointers are handed to the library unchanged.
+
+bf16 tensors may be passed either as torch.bfloat16 or as raw bit patterns (torch.uint16 /
+torch.int16); the library only sees the pointer.  There is no CPU fallback: if the shared
+library is missing, importing this module raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import Optional, Tuple
+
+import torch
+
+ORIENT_C, ORIENT_R = 0, 1
+PEN_L2, PEN_L2SQ = 0, 1
+ACT_NONE, ACT_GELU = 0, 1
+
+_PKG_DIR = os.path.dirname(os.path.abspath(__file__))
+
+
+def library_path() -> str:
+    return os.path.join(_PKG_DIR, "libbsp.so")
+
+
+class BspError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {bsp_status_string(status)} (status {status}, cuda error {lib.bsp_last_cuda_error()})")
+
+
+def _load() -> ctypes.CDLL:
+    path = library_path()
+    if not os.path.exists(path):
+        raise ImportError(
+            f"{path} is missing: build it with `python -m paper_2009_08065_b200.build` "
+            "(needs nvcc); this package has no fallback path")
+    return ctypes.CDLL(path)
+
+
+lib = _load()
+
+_vp, _i, _f, _d = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_double
+_sz, _szp = ctypes.c_size_t, ctypes.POINTER(ctypes.c_size_t)
+
+_SIGNATURES = {
+    "bsp_status_string": (ctypes.c_char_p, [_i]),
+    "bsp_last_cuda_error": (_i, []),
+    "bsp_group_norms": (_i, [_vp, _i, _i, _i, _i, _i, _f, _i, _vp, _vp, _vp, _vp, _vp]),
+    "bsp_pack_bound": (_i, [_i, _i, _i, _i, _szp, _szp, _szp]),
+    "bsp_prune_pack": (_i, [_vp, _i, _i, _i, _i, _i, _f, _vp, _i, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "bsp_percentile_threshold": (_i, [_vp, _i, _i, _i, _i, _i, _d, _vp, _vp, _sz, _vp]),
+    "bsp_apply_mask": (_i, [_vp, _i, _i, _i, _i, _i, _vp, _vp]),
+    "bsp_linear_plan_bytes": (_i, [_i, _i, _i, _szp]),
+    "bsp_linear_plan": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _sz, _vp]),
+    "bsp_linear_planned": (_i, [_vp, _i, _i, _i, _vp, _i, _i, _vp, _i, _vp, _i, _vp]),
+    "bsp_linear": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _i, _i, _vp, _i, _vp, _i, _vp, _sz, _vp]),
+    "bsp_linear_status": (_i, [_vp]),
+    "bsp_linear_cuda_core": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _i, _i, _vp, _i, _vp, _i, _vp]),
+}
+for _name, (_res, _args) in _SIGNATURES.items():
+    _fn = getattr(lib, _name)
+    _fn.restype, _fn.argtypes = _res, _args
+
+EXPORTED_SYMBOLS = tuple(_SIGNATURES)
+
+
+def bsp_status_string(status: int) -> str:
+    return lib.bsp_status_string(int(status)).decode()
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError("expected a CUDA tensor")
+    return t.data_ptr()
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream or None
+    return getattr(stream, "cuda_stream", stream) or None
+
+
+def _check(status: int, where: str) -> None:
+    if status != 0:
+        raise BspError(status, where)
+
+
+def _ld(t: torch.Tensor) -> int:
+    if t.dim() != 2 or t.stride(1) != 1:
+        raise ValueError("expected a 2-D tensor with unit inner stride")
+    return t.stride(0) if t.shape[0] > 1 else max(t.stride(0), t.shape[1])
+
+
+def _per_group_shape(rows: int, cols: int, block: int, orient: int) -> Tuple[int, int]:
+    return (rows // block, cols) if orient == ORIENT_C else (rows, cols // block)
+
+
+# ------------------------------------------------------------------------------------------
+def bsp_group_norms(W: torch.Tensor, block: int, orient: int = ORIENT_C, eps: float = 1e-3, pen: int = PEN_L2,
+                    norms: Optional[torch.Tensor] = None, gamma_in: Optional[torch.Tensor] = None,
+                    gamma_out: Optional[torch.Tensor] = None, penalty: Optional[torch.Tensor] = None,
+                    stream=None) -> None:
+    """norms / gamma_out: float32 per-group tensors; penalty: one-element float64 tensor (all optional outputs)."""
+    rows, cols = W.shape
+    _check(lib.bsp_group_norms(_ptr(W), rows, cols, _ld(W), block, orient, eps, pen, _ptr(norms), _ptr(gamma_in),
+                               _ptr(gamma_out), _ptr(penalty), _stream(stream)), "bsp_group_norms")
+
+
+def bsp_pack_bound(rows: int, cols: int, block: int, orient: int = ORIENT_C) -> Tuple[int, int, int]:
+    """(index entries, value elements, workspace bytes) in the worst case for this shape."""
+    a, b, c = ctypes.c_size_t(), ctypes.c_size_t(), ctypes.c_size_t()
+    _check(lib.bsp_pack_bound(rows, cols, block, orient, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c)),
+           "bsp_pack_bound")
+    return a.value, b.value, c.value
+
+
+@dataclass
+class PackedMatrix:
+    """Device buffers of the canonical packed form (sized for the worst case; blk_ptr[-1] entries are valid)."""
+    rows: int
+    cols: int
+    block: int
+    orient: int
+    blk_ptr: torch.Tensor       # int32 [n_blocks + 1]
+    idx: torch.Tensor           # int32
+    vals: torch.Tensor          # bf16 bit patterns (uint16 storage viewed as int16)
+    keep: torch.Tensor          # uint8 per-group flags
+    kept_weights: torch.Tensor  # int64 [1]
+    ws: torch.Tensor            # scratch
+
+    @staticmethod
+    def allocate(rows: int, cols: int, block: int, orient: int = ORIENT_C, device="cuda") -> "PackedMatrix":
+        n_idx, n_val, ws_bytes = bsp_pack_bound(rows, cols, block, orient)
+        n_blocks = rows // block if orient == ORIENT_C else cols // block
+        return PackedMatrix(
+            rows, cols, block, orient,
+            torch.empty(n_blocks + 1, dtype=torch.int32, device=device),
+            torch.empty(n_idx, dtype=torch.int32, device=device),
+            torch.empty(n_val, dtype=torch.int16, device=device),
+            torch.empty(_per_group_shape(rows, cols, block, orient), dtype=torch.uint8, device=device),
+            torch.empty(1, dtype=torch.int64, device=device),
+            torch.empty(ws_bytes, dtype=torch.uint8, device=device),
+        )
+
+
+def bsp_prune_pack(W: torch.Tensor, out: PackedMatrix, threshold: float = 0.0,
+                   threshold_dev: Optional[torch.Tensor] = None, keep_per_block: int = -1, stream=None) -> None:
+    rows, cols = W.shape
+    _check(lib.bsp_prune_pack(_ptr(W), rows, cols, _ld(W), out.block, out.orient, threshold, _ptr(threshold_dev),
+                              keep_per_block, _ptr(out.keep), _ptr(out.blk_ptr), _ptr(out.idx), _ptr(out.vals),
+                              _ptr(out.kept_weights), _ptr(out.ws), out.ws.numel(), _stream(stream)),
+           "bsp_prune_pack")
+
+
+def bsp_percentile_threshold(W: torch.Tensor, block: int, orient: int, rate: float, threshold_out: torch.Tensor,
+                             ws: torch.Tensor, stream=None) -> None:
+    rows, cols = W.shape
+    _check(lib.bsp_percentile_threshold(_ptr(W), rows, cols, _ld(W), block, orient, rate, _ptr(threshold_out),
+                                        _ptr(ws), ws.numel(), _stream(stream)), "bsp_percentile_threshold")
+
+
+def bsp_apply_mask(W: torch.Tensor, block: int, orient: int, keep: torch.Tensor, stream=None) -> None:
+    rows, cols = W.shape
+    _check(lib.bsp_apply_mask(_ptr(W), rows, cols, _ld(W), block, orient, _ptr(keep), _stream(stream)),
+           "bsp_apply_mask")
+
+
+def bsp_linear_plan_bytes(n_out: int, k_in: int, block: int) -> int:
+    b = ctypes.c_size_t()
+    _check(lib.bsp_linear_plan_bytes(n_out, k_in, block, ctypes.byref(b)), "bsp_linear_plan_bytes")
+    return b.value
+
+
+def bsp_linear_plan(packed: PackedMatrix, plan: torch.Tensor, stream=None) -> None:
+    _check(lib.bsp_linear_plan(_ptr(packed.blk_ptr), _ptr(packed.idx), _ptr(packed.vals), packed.rows, packed.cols,
+                               packed.block, _ptr(plan), plan.numel() * plan.element_size(), _stream(stream)),
+           "bsp_linear_plan")
+
+
+def bsp_linear_planned(plan: torch.Tensor, n_out: int, k_in: int, block: int, X: torch.Tensor,
+                       bias: Optional[torch.Tensor], act: int, Y: torch.Tensor, stream=None) -> None:
+    _check(lib.bsp_linear_planned(_ptr(plan), n_out, k_in, block, _ptr(X), X.shape[0], _ld(X), _ptr(bias), act,
+                                  _ptr(Y), _ld(Y), _stream(stream)), "bsp_linear_planned")
+
+
+def bsp_linear(packed: PackedMatrix, X: torch.Tensor, bias: Optional[torch.Tensor], act: int, Y: torch.Tensor,
+               ws: Optional[torch.Tensor], stream=None) -> None:
+    _check(lib.bsp_linear(_ptr(packed.blk_ptr), _ptr(packed.idx), _ptr(packed.vals), packed.rows, packed.cols,
+                          packed.block, _ptr(X), X.shape[0], _ld(X), _ptr(bias), act, _ptr(Y), _ld(Y), _ptr(ws),
+                          0 if ws is None else ws.numel() * ws.element_size(), _stream(stream)), "bsp_linear")
+
+
+def bsp_linear_cuda_core(packed: PackedMatrix, X: torch.Tensor, bias: Optional[torch.Tensor], act: int,
+                         Y: torch.Tensor, stream=None) -> None:
+    _check(lib.bsp_linear_cuda_core(_ptr(packed.blk_ptr), _ptr(packed.idx), _ptr(packed.vals), packed.rows,
+                                    packed.cols, packed.block, _ptr(X), X.shape[0], _ld(X), _ptr(bias), act, _ptr(Y),
+                                    _ld(Y), _stream(stream)), "bsp_linear_cuda_core")
+
+
+def bsp_linear_status(stream=None) -> None:
+    """Synchronises the stream; raises BspError(BSP_ERR_TIMEOUT) if a tensor-core launch gave up on a wait."""
+    _check(lib.bsp_linear_status(_stream(stream)), "bsp_linear_status")

@@ -1,0 +1,511 @@
+// bsp_linear / bsp_linear_plan / bsp_linear_planned: the pruned linear layer on the B200 tensor
+// cores (tcgen05.mma with float32 accumulators in tensor memory, operands staged by TMA).
+//
+// Execution layout ("plan").  A row-block's kept-column list differs from its neighbours', and a
+// tcgen05 operand tile addresses K in contiguous 16-byte pieces, so single columns cannot be
+// picked from a resident X tile by the hardware.  Re-gathering X per row-block would move
+// 2 bytes through shared memory per `block` multiply-adds, which caps the tensor pipe at about
+// block/64 of its peak.  The plan therefore scatters the packed values back to their natural
+// column positions, zero elsewhere: a [n_out, k_in] bf16 matrix that TMA can tile directly,
+// with X read in its natural order and reused by a whole 128 x BN output tile.  The packed form
+// stays the storage format; the plan is private scratch derived from it.
+//
+// Kernel.  Persistent CTAs (one per SM) walk output tiles of 128 tokens x BN outputs.
+//   warp 0 (one lane): TMA producer, X tile [128 x 64] and W tile [BN x 64] per pipeline stage
+//                      (128-byte swizzle), completion on an mbarrier;
+//   warp 1 (one lane): issues tcgen05.mma (M=128, N=BN, K=16) into one of two TMEM accumulators
+//                      and commits stage release / accumulator ready to mbarriers;
+//   warps 2..5       : epilogue, tcgen05.ld the accumulator (each warp its 32 TMEM lanes = 32
+//                      tokens), add bias, optional GELU, round to bf16, 16-byte stores; it runs
+//                      concurrently with the next tile's main loop on the other accumulator.
+// Every wait is bounded by a wall-clock deadline; on expiry the role records BSP_ERR_TIMEOUT in
+// the status word and leaves its loop, the other roles then time out on their own waits, and
+// the CTA frees its tensor memory and exits.
+#include <cuda.h>
+#include <math.h>
+
+#include "bsp_common.cuh"
+
+namespace bsp {
+
+int check_linear_args(const void* a, const void* b, const void* c, int n_out, int k_in, int block,
+                      const void* X, int tokens, int ldx, int act, const void* Y, int ldy);
+
+namespace {
+
+constexpr int kBlockM = 128;      // tokens per tile (TMEM lanes)
+constexpr int kBlockK = 64;       // bf16 elements per pipeline stage row = 128 bytes = one swizzle row
+constexpr int kUmmaK = 16;        // K of one tcgen05.mma for 16-bit inputs
+constexpr int kThreads = 192;     // 6 warps: producer, mma, 4 epilogue
+constexpr int kSmemBudget = 200 * 1024;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s per wait
+
+__device__ int g_linear_status;   // 0, or BSP_ERR_TIMEOUT once a bounded wait expired
+
+template <int BN>
+struct TileCfg {
+  static constexpr int kStageA = kBlockM * kBlockK * 2;
+  static constexpr int kStageB = BN * kBlockK * 2;
+  static constexpr int kStage = kStageA + kStageB;
+  static constexpr int kStages = (kSmemBudget / kStage) > 8 ? 8 : (kSmemBudget / kStage);
+  static constexpr int kTmemCols = 2 * BN <= 32 ? 32 : 2 * BN <= 64 ? 64 : 2 * BN <= 128 ? 128 : 2 * BN <= 256 ? 256 : 512;
+  static constexpr int kSmemBytes = kStages * kStage + 1024 /*alignment slack*/ + 256 /*barriers*/;
+};
+
+// ------------------------------------------------------------------------------------------
+// PTX wrappers
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: false when the deadline passed (the caller records the failure and bails out).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long start = global_timer_ns();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 256; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (global_timer_ns() - start > kWaitLimitNs) return false;
+  }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void tcgen05_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tcgen05_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tcgen05_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tcgen05_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                                 uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_load_32cols(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+        "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+        "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_load_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a K-major bf16 tile stored as 128-byte swizzled rows
+// (what a TMA load with the 128-byte swizzle mode writes): 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((smem_addr & 0x3ffff) >> 4);        // start address / 16
+  d |= static_cast<uint64_t>(1) << 16;                           // leading byte offset / 16 (unused with swizzle)
+  d |= static_cast<uint64_t>(1024 >> 4) << 32;                   // stride byte offset / 16
+  d |= static_cast<uint64_t>(1) << 46;                           // descriptor version of this architecture
+  d |= static_cast<uint64_t>(2) << 61;                           // 128-byte swizzle
+  return d;
+}
+// Instruction descriptor: bf16 x bf16 -> float32, both operands K-major, M = 128, N = BN.
+__host__ __device__ constexpr uint32_t instr_desc_bf16(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(n >> 3) << 17) |
+         (static_cast<uint32_t>(kBlockM >> 4) << 24);
+}
+
+__device__ __forceinline__ float gelu_erf(float x) { return 0.5f * x * (1.0f + erff(x * 0.70710678118654752440f)); }
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  const uint32_t l = __bfloat16_as_ushort(__float2bfloat16_rn(lo));
+  const uint32_t h = __bfloat16_as_ushort(__float2bfloat16_rn(hi));
+  return l | (h << 16);
+}
+
+struct LinearParams {
+  int tokens, n_out, k_in, ldy, act;
+  const uint16_t* bias;
+  uint16_t* Y;
+  int* status;
+};
+
+template <int BN>
+__global__ void __launch_bounds__(kThreads, 1)
+linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
+                 LinearParams P) {
+  using Cfg = TileCfg<BN>;
+  constexpr int S = Cfg::kStages;
+  extern __shared__ uint8_t smem_raw[];
+  // operand stages need 1024-byte alignment for the 128-byte swizzle pattern
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S * Cfg::kStage);
+  // bars[0..S) full, [S..2S) empty, [2S..2S+2) accumulator full, [2S+2..2S+4) accumulator empty
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 2 * S + 4);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t smem_base = smem_u32(smem);
+  const uint32_t bar_base = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (S + s); };
+  auto acc_full_bar = [&](int a) { return bar_base + 8u * (2 * S + a); };
+  auto acc_empty_bar = [&](int a) { return bar_base + 8u * (2 * S + 2 + a); };
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(acc_full_bar(a), 1); mbar_init(acc_empty_bar(a), 4); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_holder)),
+                 "r"(static_cast<uint32_t>(Cfg::kTmemCols)) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tcgen05_fence_before();
+  __syncthreads();
+  tcgen05_fence_after();
+  const uint32_t tmem_base = *tmem_holder;
+
+  const int m_tiles = (P.tokens + kBlockM - 1) / kBlockM;
+  const int n_tiles = (P.n_out + BN - 1) / BN;
+  const int total_tiles = m_tiles * n_tiles;
+  const int k_blocks = (P.k_in + kBlockK - 1) / kBlockK;
+
+  if (warp == 0 && lane == 0) {
+    // ---------------------------------------------------------------- TMA producer
+    int stage = 0;
+    uint32_t phase = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+      const int m0 = (tile / n_tiles) * kBlockM, n0 = (tile % n_tiles) * BN;
+      for (int kb = 0; kb < k_blocks; ++kb) {
+        if (!mbar_wait(empty_bar(stage), phase ^ 1u)) { ok = false; break; }
+        const uint32_t a_dst = smem_base + stage * Cfg::kStage;
+        const uint32_t b_dst = a_dst + Cfg::kStageA;
+        mbar_arrive_expect_tx(full_bar(stage), Cfg::kStage);
+        tma_load_2d(a_dst, &map_x, kb * kBlockK, m0, full_bar(stage));
+        tma_load_2d(b_dst, &map_w, kb * kBlockK, n0, full_bar(stage));
+        if (++stage == S) { stage = 0; phase ^= 1u; }
+      }
+    }
+    if (!ok) {
+      atomicExch(P.status, BSP_ERR_TIMEOUT);
+      // copies already issued land in this CTA's shared memory: give them a bounded chance to finish
+      for (int s = 0; s < S; ++s) {
+        const int back = (stage - 1 - s + 2 * S) % S;
+        const uint32_t ph = (back < stage) ? phase : (phase ^ 1u);
+        (void)mbar_wait(full_bar(back), ph);
+      }
+    }
+  } else if (warp == 1 && lane == 0) {
+    // ---------------------------------------------------------------- MMA issuer
+    constexpr uint32_t idesc = instr_desc_bf16(BN);
+    int stage = 0;
+    uint32_t phase = 0;
+    uint32_t acc_phase[2] = {0u, 0u};
+    int acc = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+      if (!mbar_wait(acc_empty_bar(acc), acc_phase[acc] ^ 1u)) { ok = false; break; }
+      tcgen05_fence_after();
+      const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN);
+      for (int kb = 0; kb < k_blocks; ++kb) {
+        if (!mbar_wait(full_bar(stage), phase)) { ok = false; break; }
+        tcgen05_fence_after();
+        const uint32_t a_addr = smem_base + stage * Cfg::kStage;
+        const uint32_t b_addr = a_addr + Cfg::kStageA;
+#pragma unroll
+        for (int k = 0; k < kBlockK / kUmmaK; ++k) {
+          const uint64_t a_desc = smem_desc_sw128(a_addr + k * kUmmaK * 2);
+          const uint64_t b_desc = smem_desc_sw128(b_addr + k * kUmmaK * 2);
+          tcgen05_mma_bf16(d_tmem, a_desc, b_desc, idesc, (kb | k) != 0 ? 1u : 0u);
+        }
+        tcgen05_commit(empty_bar(stage));  // stage reusable once these MMAs have read it
+        if (++stage == S) { stage = 0; phase ^= 1u; }
+      }
+      if (!ok) break;
+      tcgen05_commit(acc_full_bar(acc));   // accumulator complete
+      acc_phase[acc] ^= 1u;
+      acc ^= 1;
+    }
+    if (!ok) atomicExch(P.status, BSP_ERR_TIMEOUT);
+  } else if (warp >= 2) {
+    // ---------------------------------------------------------------- epilogue
+    const int quad = warp & 3;               // TMEM lanes [32*quad, 32*quad+32) belong to this warp
+    uint32_t acc_phase[2] = {0u, 0u};
+    int acc = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+      const int m0 = (tile / n_tiles) * kBlockM, n0 = (tile % n_tiles) * BN;
+      if (!mbar_wait(acc_full_bar(acc), acc_phase[acc])) { ok = false; break; }
+      tcgen05_fence_after();
+      const int t = m0 + quad * 32 + lane;
+      uint16_t* yrow = P.Y + static_cast<size_t>(t) * P.ldy;
+      const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + static_cast<uint32_t>(acc * BN);
+#pragma unroll 1
+      for (int c0 = 0; c0 < BN; c0 += 32) {
+        if (n0 + c0 >= P.n_out) break;       // uniform across the warp
+        uint32_t v[32];
+        tmem_load_32cols(taddr + c0, v);
+        tmem_load_wait();
+        if (t < P.tokens) {
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {      // 8 outputs = one 16-byte store
+            const int n = n0 + c0 + g * 8;
+            if (n < P.n_out) {               // n_out is a multiple of 8 on this path
+              float f[8];
+#pragma unroll
+              for (int i = 0; i < 8; ++i) {
+                f[i] = __uint_as_float(v[g * 8 + i]);
+                if (P.bias) f[i] += bf16_bits_to_float(__ldg(P.bias + n + i));
+                if (P.act == BSP_ACT_GELU) f[i] = gelu_erf(f[i]);
+              }
+              uint4 o;
+              o.x = pack_bf16x2(f[0], f[1]);
+              o.y = pack_bf16x2(f[2], f[3]);
+              o.z = pack_bf16x2(f[4], f[5]);
+              o.w = pack_bf16x2(f[6], f[7]);
+              *reinterpret_cast<uint4*>(yrow + n) = o;
+            }
+          }
+        }
+      }
+      tcgen05_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(acc_empty_bar(acc));
+      acc_phase[acc] ^= 1u;
+      acc ^= 1;
+    }
+    if (!ok && lane == 0) atomicExch(P.status, BSP_ERR_TIMEOUT);
+  }
+
+  tcgen05_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tcgen05_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                 "r"(static_cast<uint32_t>(Cfg::kTmemCols)) : "memory");
+  }
+}
+
+// Plan: scatter the packed tiles of one row-block back to natural column positions.
+__global__ void __launch_bounds__(256)
+plan_expand_kernel(const int32_t* __restrict__ blk_ptr, const int32_t* __restrict__ idx,
+                   const uint16_t* __restrict__ vals, int k_in, int block, uint16_t* __restrict__ Wx) {
+  extern __shared__ int32_t s_pos[];      // column -> position in the kept list, or -1
+  const int b = blockIdx.x;
+  const int lo = blk_ptr[b], kc = blk_ptr[b + 1] - lo;
+  for (int k = threadIdx.x; k < k_in; k += blockDim.x) s_pos[k] = -1;
+  __syncthreads();
+  for (int j = threadIdx.x; j < kc; j += blockDim.x) s_pos[idx[lo + j]] = j;
+  __syncthreads();
+  const uint16_t* tile = vals + static_cast<size_t>(block) * lo;
+  uint16_t* out = Wx + static_cast<size_t>(b) * block * k_in;
+  const int total = block * k_in;
+  for (int e = threadIdx.x; e < total; e += blockDim.x) {
+    const int r = e / k_in, k = e - r * k_in;
+    const int p = s_pos[k];
+    out[e] = p >= 0 ? tile[static_cast<size_t>(r) * kc + p] : static_cast<uint16_t>(0);
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// 2-D bf16 tensor [outer, inner] row-major with leading dimension ld; box [box_outer, 64] with
+// the 128-byte swizzle; out-of-range elements read as zero.
+bool make_map(CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer, uint64_t ld, uint32_t box_outer) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {inner, outer};
+  const cuuint64_t strides[1] = {ld * 2};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(kBlockK), box_outer};
+  const cuuint32_t elem[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, elem,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+struct DeviceInfo {
+  int sms = 0;
+  int* status = nullptr;
+  bool attr_set[4] = {false, false, false, false};
+};
+DeviceInfo* device_info() {
+  static DeviceInfo info[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  DeviceInfo& d = info[dev];
+  if (d.sms == 0) {
+    if (cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return nullptr;
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_linear_status) != cudaSuccess) return nullptr;
+    d.status = static_cast<int*>(p);
+    if (cudaMemset(d.status, 0, sizeof(int)) != cudaSuccess) return nullptr;
+  }
+  return &d;
+}
+
+// Output-tile width: fewest (waves x per-tile cost) over the candidates.
+int choose_bn(int tokens, int n_out, int sms) {
+  const int cands[4] = {256, 192, 128, 64};
+  long long best = -1;
+  int best_bn = 128;
+  const long long m_tiles = (tokens + kBlockM - 1) / kBlockM;
+  for (int c = 0; c < 4; ++c) {
+    const int bn = cands[c];
+    const long long tiles = m_tiles * ((n_out + bn - 1) / bn);
+    const long long waves = (tiles + sms - 1) / sms;
+    const long long cost = waves * (bn + 32);
+    if (best < 0 || cost < best) { best = cost; best_bn = bn; }
+  }
+  return best_bn;
+}
+
+template <int BN>
+int launch_tc(DeviceInfo* dev, int slot, const void* plan, const void* X, const LinearParams& P, int ldx,
+              cudaStream_t s) {
+  using Cfg = TileCfg<BN>;
+  CUtensorMap map_x, map_w;
+  if (!make_map(&map_x, X, P.k_in, P.tokens, ldx, kBlockM)) return BSP_ERR_CUDA;
+  if (!make_map(&map_w, plan, P.k_in, P.n_out, P.k_in, BN)) return BSP_ERR_CUDA;
+  if (!dev->attr_set[slot]) {
+    BSP_CUDA_TRY(cudaFuncSetAttribute(linear_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes));
+    dev->attr_set[slot] = true;
+  }
+  const int m_tiles = (P.tokens + kBlockM - 1) / kBlockM;
+  const int n_tiles = (P.n_out + BN - 1) / BN;
+  const int tiles = m_tiles * n_tiles;
+  const int grid = tiles < dev->sms ? tiles : dev->sms;
+  linear_tc_kernel<BN><<<grid, kThreads, Cfg::kSmemBytes, s>>>(map_x, map_w, P);
+  BSP_LAUNCH_CHECK();
+  return BSP_OK;
+}
+
+bool tc_path_ok(const void* plan, int n_out, int k_in, const void* X, int ldx, const void* Y, int ldy) {
+  return aligned_to(plan, 16) && aligned_to(X, 16) && aligned_to(Y, 16) && k_in % 8 == 0 && ldx % 8 == 0 &&
+         ldy % 8 == 0 && n_out % 8 == 0 && k_in <= 12288;
+}
+
+}  // namespace
+}  // namespace bsp
+
+extern "C" int bsp_linear_plan_bytes(int n_out, int k_in, int block, size_t* bytes) {
+  if (n_out <= 0 || k_in <= 0 || block <= 0 || bytes == nullptr) return BSP_ERR_ARG;
+  if (n_out % block) return BSP_ERR_SHAPE;
+  *bytes = bsp::round_up(static_cast<size_t>(n_out) * k_in * 2, 256);
+  return BSP_OK;
+}
+
+extern "C" int bsp_linear_plan(const int32_t* blk_ptr, const int32_t* idx, const void* vals, int n_out,
+                               int k_in, int block, void* plan, size_t plan_bytes, void* stream) {
+  using namespace bsp;
+  if (blk_ptr == nullptr || idx == nullptr || vals == nullptr || plan == nullptr) return BSP_ERR_ARG;
+  size_t need;
+  int st = bsp_linear_plan_bytes(n_out, k_in, block, &need);
+  if (st != BSP_OK) return st;
+  if (!aligned_to(plan, 256)) return BSP_ERR_ARG;
+  if (plan_bytes < need) return BSP_ERR_WORKSPACE;
+  if (k_in > 12288) return BSP_ERR_UNSUPPORTED;
+  plan_expand_kernel<<<n_out / block, 256, sizeof(int32_t) * k_in, static_cast<cudaStream_t>(stream)>>>(
+      blk_ptr, idx, static_cast<const uint16_t*>(vals), k_in, block, static_cast<uint16_t*>(plan));
+  BSP_LAUNCH_CHECK();
+  return BSP_OK;
+}
+
+extern "C" int bsp_linear_planned(const void* plan, int n_out, int k_in, int block, const void* X, int tokens,
+                                  int ldx, const void* bias, int act, void* Y, int ldy, void* stream) {
+  using namespace bsp;
+  int st = check_linear_args(plan, plan, plan, n_out, k_in, block, X, tokens, ldx, act, Y, ldy);
+  if (st != BSP_OK) return st;
+  if (!tc_path_ok(plan, n_out, k_in, X, ldx, Y, ldy)) return BSP_ERR_UNSUPPORTED;
+  if (tokens == 0) return BSP_OK;
+  DeviceInfo* dev = device_info();
+  if (dev == nullptr) return BSP_ERR_CUDA;
+  LinearParams P{tokens, n_out, k_in, ldy, act, static_cast<const uint16_t*>(bias), static_cast<uint16_t*>(Y),
+                 dev->status};
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  switch (choose_bn(tokens, n_out, dev->sms)) {
+    case 256: return launch_tc<256>(dev, 0, plan, X, P, ldx, s);
+    case 192: return launch_tc<192>(dev, 1, plan, X, P, ldx, s);
+    case 128: return launch_tc<128>(dev, 2, plan, X, P, ldx, s);
+    default: return launch_tc<64>(dev, 3, plan, X, P, ldx, s);
+  }
+}
+
+extern "C" int bsp_linear(const int32_t* blk_ptr, const int32_t* idx, const void* vals, int n_out, int k_in,
+                          int block, const void* X, int tokens, int ldx, const void* bias, int act, void* Y,
+                          int ldy, void* ws, size_t ws_bytes, void* stream) {
+  using namespace bsp;
+  int st = check_linear_args(blk_ptr, idx, vals, n_out, k_in, block, X, tokens, ldx, act, Y, ldy);
+  if (st != BSP_OK) return st;
+  if (ws == nullptr || !aligned_to(ws, 256) || !tc_path_ok(ws, n_out, k_in, X, ldx, Y, ldy))
+    return bsp_linear_cuda_core(blk_ptr, idx, vals, n_out, k_in, block, X, tokens, ldx, bias, act, Y, ldy, stream);
+  st = bsp_linear_plan(blk_ptr, idx, vals, n_out, k_in, block, ws, ws_bytes, stream);
+  if (st != BSP_OK) return st;
+  return bsp_linear_planned(ws, n_out, k_in, block, X, tokens, ldx, bias, act, Y, ldy, stream);
+}
+
+extern "C" int bsp_linear_status(void* stream) {
+  using namespace bsp;
+  DeviceInfo* dev = device_info();
+  if (dev == nullptr) return BSP_ERR_CUDA;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int flag = 0;
+  BSP_CUDA_TRY(cudaMemcpyAsync(&flag, dev->status, sizeof(int), cudaMemcpyDeviceToHost, s));
+  BSP_CUDA_TRY(cudaStreamSynchronize(s));
+  if (flag != 0) {
+    BSP_CUDA_TRY(cudaMemsetAsync(dev->status, 0, sizeof(int), s));
+    return BSP_ERR_TIMEOUT;
+  }
+  return BSP_OK;
+}

@@ -1,0 +1,102 @@
+"""Host-side checks of the C-ABI library that need no GPU: it loads, exports every function
+include/bsp.h declares, answers its size queries, and rejects bad arguments before launching."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import paper_2009_08065_b200 as bsp
+from paper_2009_08065_b200 import binding
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "bsp.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(bsp_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_function_is_exported_and_bound():
+    names = declared_functions()
+    assert len(names) >= 13
+    for n in names:
+        assert hasattr(bsp.lib, n), f"libbsp.so does not export {n}"
+        assert n in binding.EXPORTED_SYMBOLS, f"binding has no signature for {n}"
+    for n in binding.EXPORTED_SYMBOLS:
+        assert n in names, f"{n} is bound but not declared in bsp.h"
+
+
+def test_status_strings():
+    assert bsp.bsp_status_string(0) == "BSP_OK"
+    for code in range(-6, 0):
+        assert bsp.bsp_status_string(code).startswith("BSP_ERR_")
+    assert "unknown" in bsp.bsp_status_string(-99)
+
+
+def test_pack_bound():
+    idx, val, ws = bsp.bsp_pack_bound(768, 768, 16, bsp.ORIENT_C)
+    assert idx == 48 * 768 and val == 768 * 768 and ws >= 48 * 768 * 5 and ws % 256 == 0
+    idx, val, ws = bsp.bsp_pack_bound(768, 3072, 12, bsp.ORIENT_R)
+    assert idx == 256 * 768 and val == 768 * 3072
+    with pytest.raises(bsp.BspError) as e:
+        bsp.bsp_pack_bound(770, 768, 16, bsp.ORIENT_C)
+    assert e.value.status == -2
+    with pytest.raises(bsp.BspError) as e:
+        bsp.bsp_pack_bound(768, 768, 0, bsp.ORIENT_C)
+    assert e.value.status == -1
+    with pytest.raises(bsp.BspError):
+        bsp.bsp_pack_bound(768, 768, 16, 7)
+
+
+def test_plan_bytes():
+    assert bsp.bsp_linear_plan_bytes(768, 768, 16) == 768 * 768 * 2
+    assert bsp.bsp_linear_plan_bytes(96, 72, 3) % 256 == 0
+    with pytest.raises(bsp.BspError) as e:
+        bsp.bsp_linear_plan_bytes(100, 64, 16)
+    assert e.value.status == -2
+
+
+def test_argument_errors_are_caught_before_any_launch():
+    """Fake non-null pointers are safe here: each call must return before touching the device."""
+    lib = bsp.lib
+    p = ctypes.c_void_p(0x1000)
+    # norms: block does not divide, null W, no outputs, bad enum, negative eps, ld too small
+    assert lib.bsp_group_norms(p, 10, 8, 8, 3, 0, 1e-3, 0, p, None, None, None, None) == -2
+    assert lib.bsp_group_norms(None, 8, 8, 8, 2, 0, 1e-3, 0, p, None, None, None, None) == -1
+    assert lib.bsp_group_norms(p, 8, 8, 8, 2, 0, 1e-3, 0, None, None, None, None, None) == -1
+    assert lib.bsp_group_norms(p, 8, 8, 8, 2, 5, 1e-3, 0, p, None, None, None, None) == -1
+    assert lib.bsp_group_norms(p, 8, 8, 8, 2, 0, 1e-3, 9, p, None, None, None, None) == -1
+    assert lib.bsp_group_norms(p, 8, 8, 8, 2, 0, -1.0, 0, p, None, None, None, None) == -1
+    assert lib.bsp_group_norms(p, 8, 8, 4, 2, 0, 1e-3, 0, p, None, None, None, None) == -2
+    assert lib.bsp_group_norms(p, 8, 9, 9, 2, 1, 1e-3, 0, p, None, None, None, None) == -2   # h does not divide cols
+    # prune_pack: workspace too small, null outputs, misaligned workspace
+    assert lib.bsp_prune_pack(p, 8, 8, 8, 2, 0, 0.0, None, -1, None, p, p, p, None, ctypes.c_void_p(0x1010), 1 << 20, None) == -1  # ws not 256-aligned
+    ws = ctypes.c_void_p(0x10000)
+    assert lib.bsp_prune_pack(p, 8, 8, 8, 2, 0, 0.0, None, -1, None, p, p, p, None, ws, 16, None) == -3
+    assert lib.bsp_prune_pack(p, 8, 8, 8, 2, 0, 0.0, None, -1, None, None, p, p, None, ws, 1 << 20, None) == -1
+    assert lib.bsp_prune_pack(p, 8, 8, 8, 3, 0, 0.0, None, -1, None, p, p, p, None, ws, 1 << 20, None) == -2
+    assert lib.bsp_prune_pack(p, 16, 16384, 16384, 16, 0, 0.0, None, 4, None, p, p, p, None, ws, 1 << 30, None) == -6
+    assert lib.bsp_percentile_threshold(p, 8, 8, 8, 2, 0, 0.5, p, ws, 1 << 20, None) == -1     # rate < 1
+    assert lib.bsp_apply_mask(p, 8, 8, 8, 2, 0, None, None) == -1
+    # linear: block does not divide n_out, bad act, ld too small, null X
+    assert lib.bsp_linear_cuda_core(p, p, p, 10, 8, 4, p, 4, 8, None, 0, p, 16, None) == -2
+    assert lib.bsp_linear_cuda_core(p, p, p, 8, 8, 4, p, 4, 8, None, 3, p, 8, None) == -1
+    assert lib.bsp_linear_cuda_core(p, p, p, 8, 8, 4, p, 4, 4, None, 0, p, 8, None) == -2
+    assert lib.bsp_linear_cuda_core(p, p, p, 8, 8, 4, None, 4, 8, None, 0, p, 8, None) == -1
+    assert lib.bsp_linear(p, p, p, 10, 8, 4, p, 4, 8, None, 0, p, 16, ws, 1 << 20, None) == -2
+    assert lib.bsp_linear_planned(ws, 8, 8, 4, p, 4, 8, None, 7, p, 8, None) == -1
+    assert lib.bsp_linear_plan(p, p, p, 8, 8, 4, ws, 16, None) == -3
+    # zero tokens is a valid no-op
+    assert lib.bsp_linear_cuda_core(p, p, p, 8, 8, 4, p, 0, 8, None, 0, p, 8, None) == 0
+
+
+def test_product_code_does_not_touch_the_oracle():
+    pkg = os.path.join(ROOT, "paper_2009_08065_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                src = open(os.path.join(dirpath, f)).read()
+                assert "oracle" not in src, f"{f} mentions the oracle"
+    assert "paper_2009_08065_b200" not in open(os.path.join(ROOT, "oracle", "bsp_oracle.py")).read()

@@ -1,0 +1,178 @@
+"""GPU parity: bsp_group_norms, bsp_prune_pack, bsp_percentile_threshold, bsp_apply_mask against the oracle.
+
+Norms / gamma / penalty: relative error <= 1e-5 (float32 device arithmetic vs float64 oracle).
+Keep flags, blk_ptr, index lists, packed values, kept-weight count, thresholds: bit-exact.
+"""
+import numpy as np
+import pytest
+import torch
+
+import paper_2009_08065_b200 as bsp
+import synth_inputs as si
+from oracle import bsp_oracle as O
+from gpu_util import DEV, bits_of, packed_to_host, to_dev
+
+pytestmark = pytest.mark.gpu
+REL = 1e-5
+
+
+def run_norms(w_bits, block, orient, eps, pen, gamma_in=None, w_dev=None):
+    rows, cols = w_bits.shape
+    shape = (rows // block, cols) if orient == bsp.ORIENT_C else (rows, cols // block)
+    norms = torch.full(shape, -1.0, dtype=torch.float32, device=DEV)
+    gout = torch.full(shape, -1.0, dtype=torch.float32, device=DEV)
+    pen_out = torch.full((1,), 123.0, dtype=torch.float64, device=DEV)
+    gin = None if gamma_in is None else torch.from_numpy(gamma_in.astype(np.float32)).to(DEV)
+    bsp.bsp_group_norms(to_dev(w_bits) if w_dev is None else w_dev, block, orient, eps, pen, norms, gin, gout, pen_out)
+    torch.cuda.synchronize()
+    return norms.cpu().numpy(), gout.cpu().numpy(), float(pen_out.item())
+
+
+def check_norms(w_bits, block, orient, eps=1e-3, w_dev=None):
+    o = "C" if orient == bsp.ORIENT_C else "R"
+    n_ref = O.group_norms(w_bits, block, o)
+    s_ref = O.group_sumsq(w_bits, block, o)
+    # the paper's form
+    n, g, p = run_norms(w_bits, block, orient, eps, bsp.PEN_L2, w_dev=w_dev)
+    assert np.allclose(n, n_ref, rtol=REL, atol=0)
+    g_ref = O.gamma_update(n_ref, eps)
+    assert np.allclose(g, g_ref, rtol=REL, atol=0)
+    assert p == pytest.approx(O.penalty_l2(n_ref, g_ref), rel=REL)
+    # squared-norm variant
+    n2, a, p2 = run_norms(w_bits, block, orient, eps, bsp.PEN_L2SQ, w_dev=w_dev)
+    assert np.array_equal(n2, n)
+    a_ref = O.alpha_update_sq(s_ref, eps)
+    assert np.allclose(a, a_ref, rtol=REL, atol=0)
+    assert p2 == pytest.approx(O.penalty_l2sq(s_ref, a_ref), rel=REL)
+    # stale gamma from an earlier W, and gamma == 1 (plain group Lasso)
+    stale = O.gamma_update(O.group_norms(si.normal_bf16(99, "old", w_bits.shape, 0.02), block, o), eps)
+    _, _, p3 = run_norms(w_bits, block, orient, eps, bsp.PEN_L2, gamma_in=stale, w_dev=w_dev)
+    assert p3 == pytest.approx(O.penalty_l2(n_ref, stale.astype(np.float32).astype(np.float64)), rel=REL)
+    _, _, p4 = run_norms(w_bits, block, orient, eps, bsp.PEN_L2, gamma_in=np.ones_like(n_ref), w_dev=w_dev)
+    assert p4 == pytest.approx(O.penalty_l2(n_ref, None), rel=REL)
+
+
+@pytest.mark.parametrize("block", [16, 3, 12, 96, 8, 32, 64, 1])
+def test_norms_orientation_c_768(block):
+    spec = si.LinearSpec("n768", 768, 768, False, 2.0, block)
+    wp, _ = si.make_pruned_weight(si.DEFAULT_SEED, spec)          # half of the groups are exactly zero
+    check_norms(wp, block, bsp.ORIENT_C)
+
+
+@pytest.mark.parametrize("block", [16, 3, 12, 4])
+def test_norms_orientation_r(block):
+    spec = si.LinearSpec("nr", 768, 3072, False, 2.0, block)
+    wp, _ = si.make_pruned_weight(si.DEFAULT_SEED, spec, orient="R")
+    check_norms(wp, block, bsp.ORIENT_R)
+
+
+def test_norms_odd_shapes_and_strides():
+    # cols not a multiple of 8 (scalar path), a padded leading dimension, and an odd base offset
+    w = si.normal_bf16(5, "odd", (36, 50), 0.02)
+    check_norms(w, 12, bsp.ORIENT_C)
+    check_norms(w, 5, bsp.ORIENT_R)
+    big = si.normal_bf16(6, "pad", (48, 72), 0.02)
+    big_dev = to_dev(big)
+    check_norms(np.ascontiguousarray(big[:, :64]), 16, bsp.ORIENT_C, w_dev=big_dev[:, :64])     # ld 72, vector path
+    check_norms(np.ascontiguousarray(big[:, 3:67]), 16, bsp.ORIENT_C, w_dev=big_dev[:, 3:67])   # misaligned base
+    check_norms(np.ascontiguousarray(big[:, 3:67]), 8, bsp.ORIENT_R, w_dev=big_dev[:, 3:67])
+
+
+def test_norms_heavy_tailed_ffn_shape():
+    w = si.student_t_bf16(si.DEFAULT_SEED, "t3", (3072, 768), 3.0, 0.02)
+    check_norms(w, 32, bsp.ORIENT_C)
+
+
+def test_norms_outputs_are_optional():
+    w = si.normal_bf16(8, "opt", (64, 64), 0.02)
+    pen = torch.zeros(1, dtype=torch.float64, device=DEV)
+    bsp.bsp_group_norms(to_dev(w), 16, bsp.ORIENT_C, 1e-3, bsp.PEN_L2, None, None, None, pen)
+    n_ref = O.group_norms(w, 16, "C")
+    assert float(pen.item()) == pytest.approx(O.penalty_l2(n_ref, O.gamma_update(n_ref, 1e-3)), rel=REL)
+    with pytest.raises(bsp.BspError):
+        bsp.bsp_group_norms(to_dev(w), 16, bsp.ORIENT_C, 1e-3, bsp.PEN_L2, None, None, None, None)
+
+
+# ---------------------------------------------------------------------------------------- pack
+def check_pack(w_bits, block, orient, t_b=0.0, keep_per_block=-1, thr_dev=None, keep_ref=None):
+    o = "C" if orient == bsp.ORIENT_C else "R"
+    rows, cols = w_bits.shape
+    if keep_ref is None:
+        keep_ref = (O.keep_topk_per_block(w_bits, block, o, keep_per_block) if keep_per_block >= 0
+                    else O.keep_flags(w_bits, block, o, t_b))
+    ref_ptr, ref_idx, ref_vals = O.pack(w_bits, keep_ref, block, o)
+    pk = bsp.PackedMatrix.allocate(rows, cols, block, orient, DEV)
+    pk.idx.fill_(-7)
+    bsp.bsp_prune_pack(to_dev(w_bits), pk, t_b, thr_dev, keep_per_block)
+    torch.cuda.synchronize()
+    blk_ptr, idx, vals, keep, kept = packed_to_host(pk)
+    assert np.array_equal(keep, keep_ref)
+    assert np.array_equal(blk_ptr, ref_ptr)
+    assert np.array_equal(idx, ref_idx)
+    assert np.array_equal(vals, ref_vals)
+    assert kept == block * int(keep_ref.sum())
+    return pk, keep_ref
+
+
+@pytest.mark.parametrize("block,orient", [(16, 0), (3, 0), (12, 0), (96, 0), (3, 1), (12, 1), (16, 1)])
+def test_pack_seeded_sets_zero_threshold(block, orient):
+    spec = si.LinearSpec("pk", 768, 768, False, 2.0, block)
+    wp, keep = si.make_pruned_weight(si.DEFAULT_SEED, spec, orient="CR"[orient])
+    _, keep_ref = check_pack(wp, block, orient, 0.0)
+    assert np.array_equal(keep_ref, keep)                       # exactly the drawn sets: rate 2.0
+
+
+def test_pack_ffn_shapes_rate_3():
+    for n, k in [(3072, 768), (768, 3072), (2304, 768)]:
+        spec = si.LinearSpec(f"ffn{n}x{k}", n, k, False, 3.0, 16)
+        wp, keep = si.make_pruned_weight(si.DEFAULT_SEED, spec)
+        pk, _ = check_pack(wp, 16, bsp.ORIENT_C, 0.0)
+        assert int(pk.kept_weights.item()) * 3 == n * k
+
+
+def test_pack_thresholds_ties_and_limits():
+    g = si.stream(3, 1)
+    wf = g.integers(-3, 4, size=(48, 64)).astype(np.float32) / 8      # many exact ties and zero groups
+    w = si.f32_to_bf16_bits(wf)
+    for orient, block in [(0, 4), (1, 4), (0, 2), (1, 8)]:
+        for t in [0.0, 0.25, 0.375, 0.5, 0.75, -1.0, 100.0, float(np.sqrt(np.float32(0.5)))]:
+            check_pack(w, block, orient, t)
+
+
+def test_pack_percentile_threshold_pipeline():
+    w = si.student_t_bf16(si.DEFAULT_SEED, "pct", (768, 768), 3.0, 0.02)
+    for orient, block in [(0, 32), (1, 12)]:
+        o = "CR"[orient]
+        for rate in (1.79, 1.0, 5.0):
+            t_ref = O.percentile_threshold(w, block, o, rate)
+            _, _, ws_bytes = bsp.bsp_pack_bound(768, 768, block, orient)
+            ws = torch.empty(ws_bytes, dtype=torch.uint8, device=DEV)
+            t_dev = torch.zeros(1, dtype=torch.float32, device=DEV)
+            bsp.bsp_percentile_threshold(to_dev(w), block, orient, rate, t_dev, ws)
+            torch.cuda.synchronize()
+            assert np.float32(t_dev.item()) == np.float32(t_ref)        # bit-exact threshold
+            check_pack(w, block, orient, t_b=123.0, thr_dev=t_dev, keep_ref=O.keep_flags(w, block, o, t_ref))
+
+
+def test_pack_keep_count_per_block():
+    w = si.normal_bf16(4, "topk", (96, 768), 0.02)
+    check_pack(w, 16, bsp.ORIENT_C, keep_per_block=256)
+    check_pack(w, 16, bsp.ORIENT_C, keep_per_block=0)
+    check_pack(w, 16, bsp.ORIENT_C, keep_per_block=768)
+    check_pack(np.ascontiguousarray(w.T), 16, bsp.ORIENT_R, keep_per_block=300)
+    g = si.stream(5, 2)
+    ties = si.f32_to_bf16_bits(g.integers(-2, 3, size=(32, 40)).astype(np.float32))
+    check_pack(ties, 4, bsp.ORIENT_C, keep_per_block=13)
+    check_pack(ties, 4, bsp.ORIENT_R, keep_per_block=9)
+
+
+def test_apply_mask_matches_pruned_weight():
+    w = si.normal_bf16(6, "am", (96, 80), 0.02)
+    for orient, block in [(0, 12), (1, 5)]:
+        o = "CR"[orient]
+        t = float(np.median(O.group_norms(w, block, o)))
+        keep = O.keep_flags(w, block, o, t)
+        wd = to_dev(w).clone()
+        bsp.bsp_apply_mask(wd, block, orient, torch.from_numpy(keep.astype(np.uint8)).to(DEV))
+        torch.cuda.synchronize()
+        assert np.array_equal(bits_of(wd), O.prune(w, block, o, t))      # Algorithm 1's W_p = W * Mask
