@@ -1,0 +1,425 @@
+#!/usr/bin/env python
+"""Benchmark of the block-structured-pruning hot path on B200.
+
+One *step* = one pass of the whole path over one batch of synthetic input, for each of the four
+linears of a BERT-base encoder layer at 4096 tokens (16-row blocks, 3.0x compression):
+    bsp_group_norms (norms, gamma, penalty)  ->  bsp_prune_pack (Algorithm 1 + packed storage)
+    ->  bsp_linear_plan  ->  bsp_linear_planned (tcgen05 GEMM + bias [+ GELU]),
+with the layer's outputs chained (attention-output reads the V third of QKV's output, FFN-up
+reads attention-output's result through GELU, FFN-down reads FFN-up's).
+
+    python bench.py --gpus N --steps K --warmup W            # the CUDA path
+    python bench.py --impl reference ...                     # the CPU oracle, timed as it stands
+
+The metric is TFLOP/s counted on non-zero multiply-adds: 2 * tokens * kept weights per step.
+Prints one JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import synth_inputs as si  # noqa: E402
+
+METRIC = "block-sparse linear TFLOP/s (nonzero) & % bf16 tensor peak, BERT-base shapes"
+UNIT = "TFLOP/s"
+EPS = 1e-3
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+L2_FLUSH_BYTES = 256 << 20      # larger than the 126 MB L2
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f), "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def workload():
+    return si.bert_base_layer(tokens=4096, rate=3.0, block=16)
+
+
+# ------------------------------------------------------------------------------------------------
+# clocks during the timed region (read-only NVML queries)
+# ------------------------------------------------------------------------------------------------
+class ClockSampler:
+    REASONS = {
+        0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap",
+        0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting", 0x100: "display_clock_setting",
+    }
+
+    def __init__(self, device_index: int, period_s: float = 0.002):
+        self.samples, self.reasons, self.period = [], set(), period_s
+        self.max_mhz, self._stop, self._thread, self._h, self._nv = None, threading.Event(), None, None, None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            import torch
+            uuid = torch.cuda.get_device_properties(device_index).uuid
+            self._h = None
+            for i in range(pynvml.nvmlDeviceGetCount()):
+                h = pynvml.nvmlDeviceGetHandleByIndex(i)
+                u = pynvml.nvmlDeviceGetUUID(h)
+                u = u.decode() if isinstance(u, bytes) else u
+                if str(uuid) in u:
+                    self._h = h
+            if self._h is None:
+                self._h = pynvml.nvmlDeviceGetHandleByIndex(device_index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self._h = None
+
+    def _run(self):
+        nv = self._nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM))
+                mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self._h)
+                for bit, name in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def __enter__(self):
+        if self._h is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread:
+            self._thread.join()
+
+    def summary(self):
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# ------------------------------------------------------------------------------------------------
+# the CUDA arm
+# ------------------------------------------------------------------------------------------------
+class LayerOnDevice:
+    """Device buffers and the per-step call sequence for one rank's batch."""
+
+    def __init__(self, wl, seed, rank, device):
+        import torch
+        import paper_2009_08065_b200 as bsp
+        self.torch, self.bsp, self.wl, self.device = torch, bsp, wl, device
+        self.host = {}          # pinned host copies of the inputs, for the end-to-end leg
+        x = si.make_activations(seed + 1000 * rank, "layer_in", wl.tokens, wl.linears[0].k_in)
+        self.host["x"] = torch.from_numpy(x.view(np.int16)).pin_memory()
+        self.x = self.host["x"].to(device)
+        self.lin = []
+        for spec in wl.linears:
+            wp, _ = si.make_pruned_weight(seed, spec)          # weights are replicated across ranks
+            b = si.make_bias(seed, spec)
+            hw = torch.from_numpy(wp.view(np.int16)).pin_memory()
+            hb = torch.from_numpy(b.view(np.int16)).pin_memory()
+            n_blocks = spec.n_out // spec.block
+            e = {
+                "spec": spec, "hW": hw, "hb": hb, "W": hw.to(device), "b": hb.to(device),
+                "norms": torch.empty((n_blocks, spec.k_in), dtype=torch.float32, device=device),
+                "gamma": torch.empty((n_blocks, spec.k_in), dtype=torch.float32, device=device),
+                "penalty": torch.zeros(1, dtype=torch.float64, device=device),
+                "pk": bsp.PackedMatrix.allocate(spec.n_out, spec.k_in, spec.block, bsp.ORIENT_C, device),
+                "plan": torch.empty(bsp.bsp_linear_plan_bytes(spec.n_out, spec.k_in, spec.block), dtype=torch.uint8, device=device),
+                "Y": torch.empty((wl.tokens, spec.n_out), dtype=torch.int16, device=device),
+            }
+            self.lin.append(e)
+        self.kernels_per_step = 6 * len(self.lin)   # norms, flags, scan, compact, plan, gemm per matrix
+
+    def source(self, spec, outs):
+        if spec.src == "x":
+            return self.x
+        if spec.src == "qkv_v":
+            h = spec.k_in
+            return outs["qkv"][:, 2 * h: 3 * h]
+        return outs[spec.src]
+
+    def step(self, gemm_events=None):
+        bsp, outs = self.bsp, {}
+        for i, e in enumerate(self.lin):
+            spec = e["spec"]
+            bsp.bsp_group_norms(e["W"], spec.block, bsp.ORIENT_C, EPS, bsp.PEN_L2, e["norms"], None, e["gamma"], e["penalty"])
+            bsp.bsp_prune_pack(e["W"], e["pk"], 0.0)
+            bsp.bsp_linear_plan(e["pk"], e["plan"])
+            src = self.source(spec, outs)
+            if gemm_events is not None:
+                gemm_events[i][0].record()
+            bsp.bsp_linear_planned(e["plan"], spec.n_out, spec.k_in, spec.block, src, e["b"], int(spec.gelu), e["Y"])
+            if gemm_events is not None:
+                gemm_events[i][1].record()
+            outs[spec.name.split(".")[1]] = e["Y"]
+        return outs
+
+    def upload_inputs(self):
+        self.x.copy_(self.host["x"], non_blocking=True)
+        for e in self.lin:
+            e["W"].copy_(e["hW"], non_blocking=True)
+            e["b"].copy_(e["hb"], non_blocking=True)
+
+    def h2d_bytes(self):
+        return self.host["x"].numel() * 2 + sum(e["hW"].numel() * 2 + e["hb"].numel() * 2 for e in self.lin)
+
+    def nonzero_flops(self):
+        self.torch.cuda.synchronize()
+        return [2 * self.wl.tokens * int(e["pk"].kept_weights.item()) for e in self.lin]
+
+
+def dense_context(wl, device, iters=20):
+    """torch.matmul (cuBLAS) bf16 on the same (tokens, N, K), L2 flushed: context, not part of the path."""
+    import torch
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=device)
+    out = {}
+    for spec in wl.linears:
+        a = torch.randn(wl.tokens, spec.k_in, device=device, dtype=torch.bfloat16)
+        w = torch.randn(spec.n_out, spec.k_in, device=device, dtype=torch.bfloat16)
+        for _ in range(3):
+            torch.matmul(a, w.t())
+        ms = []
+        for _ in range(iters):
+            flush.zero_()
+            s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            s.record()
+            torch.matmul(a, w.t())
+            e.record()
+            torch.cuda.synchronize()
+            ms.append(s.elapsed_time(e))
+        t = statistics.median(ms)
+        out[spec.name.split(".")[1]] = {"ms": round(t, 5), "dense_tflops": round(2 * wl.tokens * spec.n_out * spec.k_in / t / 1e9, 1)}
+    return out
+
+
+def run_cuda(args):
+    import torch
+    import torch.distributed as dist
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the library has no CPU path (use --impl reference for the oracle)")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+
+    wl = workload()
+    layer = LayerOnDevice(wl, si.DEFAULT_SEED, rank, device)
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=device)
+
+    # warm-up outside any graph (first calls set function attributes and the status word)
+    for _ in range(max(args.warmup, 3)):
+        layer.step()
+    layer.bsp.bsp_linear_status()
+    flops = layer.nonzero_flops()
+    step_flops = sum(flops)
+
+    # the step as a CUDA graph, with external timing events around the step and around each GEMM
+    ev = lambda: torch.cuda.Event(enable_timing=True, external=True)  # noqa: E731
+    ev_step = (ev(), ev())
+    ev_gemm = [(ev(), ev()) for _ in layer.lin]
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        ev_step[0].record()
+        layer.step(gemm_events=ev_gemm)
+        ev_step[1].record()
+    for _ in range(max(args.warmup, 3)):
+        flush.zero_()
+        graph.replay()
+    torch.cuda.synchronize()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    step_ms, gemm_ms = [], [[] for _ in layer.lin]
+    barrier()
+    with ClockSampler(local_rank) as clocks:
+        for _ in range(args.steps):
+            flush.zero_()                  # untimed: evict the step's inputs from L2
+            graph.replay()
+            torch.cuda.synchronize()
+            step_ms.append(ev_step[0].elapsed_time(ev_step[1]))
+            for i, (a, b) in enumerate(ev_gemm):
+                gemm_ms[i].append(a.elapsed_time(b))
+    barrier()
+    layer.bsp.bsp_linear_status()
+    total_ms = sum(step_ms)
+
+    # end to end: pinned host inputs -> device, the step, result back to the host
+    y_host = torch.empty_like(layer.lin[-1]["Y"], device="cpu").pin_memory()
+    pen_host = torch.empty(len(layer.lin), dtype=torch.float64).pin_memory()
+    e2e_ms = []
+    e_s, e_e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for it in range(args.warmup + args.steps):
+        barrier() if it == args.warmup else None
+        e_s.record()
+        layer.upload_inputs()
+        graph.replay()
+        y_host.copy_(layer.lin[-1]["Y"], non_blocking=True)
+        for i, e in enumerate(layer.lin):
+            pen_host[i:i + 1].copy_(e["penalty"], non_blocking=True)
+        e_e.record()
+        torch.cuda.synchronize()
+        if it >= args.warmup:
+            e2e_ms.append(e_s.elapsed_time(e_e))
+    e2e_total_ms = sum(e2e_ms)
+
+    if world > 1:
+        t = torch.tensor([total_ms, e2e_total_ms], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms, e2e_total_ms = float(t[0]), float(t[1])
+
+    if rank == 0:
+        peaks, peak_src = measured_peaks()
+        gemm_mean_ms = [statistics.mean(v) for v in gemm_ms]
+        gemm_total = sum(gemm_mean_ms)
+        achieved = step_flops / gemm_total / 1e9          # TFLOP/s over the four GEMM launches of a step
+        peak = float(peaks["bf16_tflops"])
+        value = world * step_flops * args.steps / total_ms / 1e9
+        line = {
+            "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": round(total_ms / args.steps, 5), "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {
+                "workload": wl.name + " (one BERT-base encoder layer: QKV, attn-out, FFN-up+GELU, FFN-down; "
+                            "tokens per GPU 4096; 16-row blocks; 3.0x compression)",
+                "step": "group norms+gamma+penalty, prune/pack, plan, linear for each of the 4 matrices, one CUDA graph",
+                "l2": f"flushed between steps by writing {L2_FLUSH_BYTES >> 20} MiB",
+                "parallelism": "token split, replicated weights, no collective" if world > 1 else "single GPU",
+                "nonzero_gflop_per_step_per_gpu": round(step_flops / 1e9, 3),
+            },
+            "percent_of_bf16_peak": round(100 * value / world / peak, 2),
+            "e2e": {"value": round(world * step_flops * len(e2e_ms) / e2e_total_ms / 1e9, 3), "unit": UNIT,
+                    "h2d_bytes_per_step": layer.h2d_bytes(),
+                    "d2h_bytes_per_step": y_host.numel() * 2 + pen_host.numel() * 8},
+            "gpu_launches": layer.kernels_per_step * args.steps,
+            "clocks": clocks.summary(),
+            "roofline": {
+                "kernel": "linear_tc_kernel (bsp_linear_planned), the four launches of a step",
+                "bound": "tensor", "achieved": round(achieved, 2), "peak": peak, "unit": "TFLOP/s",
+                "frac": round(achieved / peak, 4), "traffic": None,
+                "peak_source": f"bf16_tflops burst, {peak_src}",
+                "per_launch": {e["spec"].name.split(".")[1]: {
+                    "ms": round(gemm_mean_ms[i], 5), "nonzero_tflops": round(flops[i] / gemm_mean_ms[i] / 1e9, 1)}
+                    for i, e in enumerate(layer.lin)},
+            },
+        }
+        if world == 1:
+            line["dense_gemm_context"] = dense_context(wl, device)
+            line["cpu_baseline"] = oracle_baseline(wl, reps=3)
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# ------------------------------------------------------------------------------------------------
+# the CPU oracle, timed as it stands
+# ------------------------------------------------------------------------------------------------
+def oracle_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info()]
+        return max(n) if n else os.cpu_count()
+    except Exception:
+        return os.cpu_count()
+
+
+def oracle_step(wl, inputs):
+    """The same step on the oracle: norms, gamma, penalty, keep flags, pack, masked dense product."""
+    from oracle import bsp_oracle as O
+    x, mats = inputs
+    kept = 0
+    for spec, wp, b, xin in mats:
+        n = O.group_norms(wp, spec.block, "C")
+        g = O.gamma_update(n, EPS)
+        O.penalty_l2(n, g)
+        keep = O.keep_flags(wp, spec.block, "C", 0.0)
+        O.pack(wp, keep, spec.block, "C")
+        O.linear_masked_dense(xin, wp, O.mask_of(wp), b, int(spec.gelu))
+        kept += spec.block * int(keep.sum())
+    return kept
+
+
+def oracle_inputs(wl, seed, tokens):
+    x = si.make_activations(seed, "layer_in", tokens, wl.linears[0].k_in)
+    mats = []
+    for spec in wl.linears:
+        wp, _ = si.make_pruned_weight(seed, spec)
+        # each linear gets fresh N(0,1) activations of its input width (the oracle is not chained)
+        xin = x if spec.src == "x" else si.make_activations(seed, spec.name, tokens, spec.k_in)
+        mats.append((spec, wp, si.make_bias(seed, spec), xin))
+    return x, mats
+
+
+def oracle_baseline(wl, reps):
+    inputs = oracle_inputs(wl, si.DEFAULT_SEED, wl.tokens)
+    oracle_step(wl, inputs)                                  # first call pays imports and page faults
+    t0 = time.perf_counter()
+    for _ in range(reps):
+        kept = oracle_step(wl, inputs)
+    dt = (time.perf_counter() - t0) / reps
+    return {"value": round(2 * wl.tokens * kept / dt / 1e12, 5), "unit": UNIT, "cores": oracle_threads(),
+            "kind": "oracle", "seconds_per_step": round(dt, 4),
+            "sample": f"the full workload ({wl.tokens} tokens, 4 matrices), {reps} steps after one untimed step"}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    wl = workload()
+    inputs = oracle_inputs(wl, si.DEFAULT_SEED, wl.tokens)
+    steps = min(args.steps, 20)                              # about 1 s each: keeps the run within minutes
+    warm = min(max(args.warmup, 1), 3)
+    for _ in range(warm):
+        kept = oracle_step(wl, inputs)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        kept = oracle_step(wl, inputs)
+    dt = time.perf_counter() - t0
+    value = round(2 * wl.tokens * kept * steps / dt / 1e12, 5)
+    sample = f"the full workload ({wl.tokens} tokens, 4 matrices) per step; {steps} timed steps"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
+        "steps": steps, "warmup": warm, "ms_per_step": round(1e3 * dt / steps, 3), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name + " on the CPU oracle (numpy float64), rank 0 only"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", choices=["cuda", "reference"], default="cuda")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_cuda(args)
+
+
+if __name__ == "__main__":
+    main()
