@@ -16,8 +16,10 @@
 //   warp 1 (one lane): issues tcgen05.mma (M=128, N=BN, K=16) into one of two TMEM accumulators
 //                      and commits stage release / accumulator ready to mbarriers;
 //   warps 2..5       : epilogue, tcgen05.ld the accumulator (each warp its 32 TMEM lanes = 32
-//                      tokens), add bias, optional GELU, round to bf16, 16-byte stores; it runs
-//                      concurrently with the next tile's main loop on the other accumulator.
+//                      tokens), add bias, optional GELU, round to bf16, stage 128 x 64 pieces in
+//                      swizzled shared memory and hand them to TMA stores (full-line writes,
+//                      tails clipped by the tensor map); it runs concurrently with the next
+//                      tile's main loop on the other accumulator.
 // Every wait is bounded by a wall-clock deadline; on expiry the role records BSP_ERR_TIMEOUT in
 // the status word and leaves its loop, the other roles then time out on their own waits, and
 // the CTA frees its tensor memory and exits.
@@ -37,7 +39,9 @@ constexpr int kBlockM = 128;      // tokens per tile (TMEM lanes)
 constexpr int kBlockK = 64;       // bf16 elements per pipeline stage row = 128 bytes = one swizzle row
 constexpr int kUmmaK = 16;        // K of one tcgen05.mma for 16-bit inputs
 constexpr int kThreads = 192;     // 6 warps: producer, mma, 4 epilogue
-constexpr int kSmemBudget = 200 * 1024;
+constexpr int kSmemLimit = 232448;              // 227 KB of dynamic shared memory per CTA
+constexpr int kEpiCols = 64;                    // columns per epilogue piece = one 128-byte swizzle row of bf16
+constexpr int kEpiStage = kBlockM * kEpiCols * 2;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s per wait
 
 __device__ int g_linear_status;   // 0, or BSP_ERR_TIMEOUT once a bounded wait expired
@@ -47,9 +51,10 @@ struct TileCfg {
   static constexpr int kStageA = kBlockM * kBlockK * 2;
   static constexpr int kStageB = BN * kBlockK * 2;
   static constexpr int kStage = kStageA + kStageB;
-  static constexpr int kStages = (kSmemBudget / kStage) > 8 ? 8 : (kSmemBudget / kStage);
+  static constexpr int kFixed = 1024 /*alignment slack*/ + 2 * kEpiStage + BN * 4 /*bias*/ + 256 /*barriers*/;
+  static constexpr int kStages = ((kSmemLimit - kFixed) / kStage) > 8 ? 8 : ((kSmemLimit - kFixed) / kStage);
   static constexpr int kTmemCols = 2 * BN <= 32 ? 32 : 2 * BN <= 64 ? 64 : 2 * BN <= 128 ? 128 : 2 * BN <= 256 ? 256 : 512;
-  static constexpr int kSmemBytes = kStages * kStage + 1024 /*alignment slack*/ + 256 /*barriers*/;
+  static constexpr int kSmemBytes = kStages * kStage + kFixed;
 };
 
 // ------------------------------------------------------------------------------------------
@@ -126,6 +131,23 @@ __device__ __forceinline__ void tmem_load_32cols(uint32_t taddr, uint32_t (&v)[3
       : "r"(taddr)
       : "memory");
 }
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int x, int y, uint32_t src) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(src)
+               : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void tma_store_wait_read() {
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+// Barrier among the 128 epilogue threads only (barrier 0 is __syncthreads).
+__device__ __forceinline__ void epilogue_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
 __device__ __forceinline__ void tmem_load_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // Shared-memory matrix descriptor of a K-major bf16 tile stored as 128-byte swizzled rows
@@ -145,7 +167,20 @@ __host__ __device__ constexpr uint32_t instr_desc_bf16(int n) {
          (static_cast<uint32_t>(kBlockM >> 4) << 24);
 }
 
-__device__ __forceinline__ float gelu_erf(float x) { return 0.5f * x * (1.0f + erff(x * 0.70710678118654752440f)); }
+// GELU(x) = x * Phi(x) with Phi from the rational-exponential approximation of erfc published as
+// formula 7.1.26 in Abramowitz & Stegun's handbook (absolute error of erf below 1.5e-7, far under
+// the bf16 rounding of the output): erfc(z) ~ (a1 t + ... + a5 t^5) exp(-z^2), t = 1/(1 + p z),
+// z = |x| / sqrt(2).  Branch-free: Phi(x) = q for x < 0 and 1 - q otherwise, q = erfc(z) / 2.
+__device__ __forceinline__ float gelu_erf(float x) {
+  const float z = fabsf(x) * 0.70710678118654752440f;
+  const float t = __fdividef(1.0f, fmaf(0.3275911f, z, 1.0f));
+  float poly = fmaf(1.061405429f, t, -1.453152027f);
+  poly = fmaf(poly, t, 1.421413741f);
+  poly = fmaf(poly, t, -0.284496736f);
+  poly = fmaf(poly, t, 0.254829592f);
+  const float q = 0.5f * poly * t * __expf(-z * z);
+  return x * (x < 0.0f ? q : 1.0f - q);
+}
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   const uint32_t l = __bfloat16_as_ushort(__float2bfloat16_rn(lo));
@@ -154,22 +189,22 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 }
 
 struct LinearParams {
-  int tokens, n_out, k_in, ldy, act;
+  int tokens, n_out, k_in, act;
   const uint16_t* bias;
-  uint16_t* Y;
   int* status;
 };
 
 template <int BN>
 __global__ void __launch_bounds__(kThreads, 1)
 linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
-                 LinearParams P) {
+                 const __grid_constant__ CUtensorMap map_y, LinearParams P) {
   using Cfg = TileCfg<BN>;
   constexpr int S = Cfg::kStages;
   extern __shared__ uint8_t smem_raw[];
   // operand stages need 1024-byte alignment for the 128-byte swizzle pattern
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S * Cfg::kStage);
+  // [S operand stages][2 epilogue staging buffers][bias as float][mbarriers, TMEM base]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S * Cfg::kStage + 2 * kEpiStage + BN * 4);
   // bars[0..S) full, [S..2S) empty, [2S..2S+2) accumulator full, [2S+2..2S+4) accumulator empty
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 2 * S + 4);
 
@@ -263,50 +298,68 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
   } else if (warp >= 2) {
     // ---------------------------------------------------------------- epilogue
     const int quad = warp & 3;               // TMEM lanes [32*quad, 32*quad+32) belong to this warp
+    const int row = quad * 32 + lane;        // token row of this thread inside the tile
+    const int epi_tid = threadIdx.x - 64;    // 0..127 among the epilogue threads
+    const uint32_t stage_base = smem_base + S * Cfg::kStage;
+    float* s_bias = reinterpret_cast<float*>(smem + S * Cfg::kStage + 2 * kEpiStage);
+    const uint32_t row_off = static_cast<uint32_t>(row) * 128u;
+    const uint32_t row_xor = static_cast<uint32_t>(row & 7);
     uint32_t acc_phase[2] = {0u, 0u};
     int acc = 0;
+    uint32_t piece = 0;                      // pieces stored so far: selects the staging buffer
     bool ok = true;
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
       const int m0 = (tile / n_tiles) * kBlockM, n0 = (tile % n_tiles) * BN;
+      // bias of this tile's columns as float; readers of the previous tile's values are all past
+      // the last epilogue_sync of that tile, and the first one below publishes these
+      for (int c = epi_tid; c < BN; c += 128)
+        s_bias[c] = (P.bias != nullptr && n0 + c < P.n_out) ? bf16_bits_to_float(__ldg(P.bias + n0 + c)) : 0.0f;
       if (!mbar_wait(acc_full_bar(acc), acc_phase[acc])) { ok = false; break; }
       tcgen05_fence_after();
-      const int t = m0 + quad * 32 + lane;
-      uint16_t* yrow = P.Y + static_cast<size_t>(t) * P.ldy;
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + static_cast<uint32_t>(acc * BN);
+      const int pieces = (min(BN, P.n_out - n0) + kEpiCols - 1) / kEpiCols;
 #pragma unroll 1
-      for (int c0 = 0; c0 < BN; c0 += 32) {
-        if (n0 + c0 >= P.n_out) break;       // uniform across the warp
-        uint32_t v[32];
-        tmem_load_32cols(taddr + c0, v);
+      for (int pc = 0; pc < pieces; ++pc) {
+        const int c0 = pc * kEpiCols;
+        const uint32_t buf = stage_base + (piece & 1u) * kEpiStage;
+        if (epi_tid == 0) tma_store_wait_read<1>();   // the store issued two pieces ago has read this buffer
+        epilogue_sync();
+        uint32_t v0[32], v1[32];
+        tmem_load_32cols(taddr + c0, v0);
+        tmem_load_32cols(taddr + c0 + 32, v1);
         tmem_load_wait();
-        if (t < P.tokens) {
-#pragma unroll
-          for (int g = 0; g < 4; ++g) {      // 8 outputs = one 16-byte store
-            const int n = n0 + c0 + g * 8;
-            if (n < P.n_out) {               // n_out is a multiple of 8 on this path
-              float f[8];
-#pragma unroll
-              for (int i = 0; i < 8; ++i) {
-                f[i] = __uint_as_float(v[g * 8 + i]);
-                if (P.bias) f[i] += bf16_bits_to_float(__ldg(P.bias + n + i));
-                if (P.act == BSP_ACT_GELU) f[i] = gelu_erf(f[i]);
-              }
-              uint4 o;
-              o.x = pack_bf16x2(f[0], f[1]);
-              o.y = pack_bf16x2(f[2], f[3]);
-              o.z = pack_bf16x2(f[4], f[5]);
-              o.w = pack_bf16x2(f[6], f[7]);
-              *reinterpret_cast<uint4*>(yrow + n) = o;
-            }
-          }
+        if (pc == pieces - 1) {              // accumulator fully read: the MMA warp may overwrite it
+          tcgen05_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(acc_empty_bar(acc));
         }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {        // 8 outputs -> one 16-byte piece of the swizzled staging row
+          const uint32_t* v = j < 4 ? &v0[j * 8] : &v1[(j - 4) * 8];
+          const float4 b0 = *reinterpret_cast<const float4*>(s_bias + c0 + j * 8);
+          const float4 b1 = *reinterpret_cast<const float4*>(s_bias + c0 + j * 8 + 4);
+          float f[8] = {__uint_as_float(v[0]) + b0.x, __uint_as_float(v[1]) + b0.y, __uint_as_float(v[2]) + b0.z,
+                        __uint_as_float(v[3]) + b0.w, __uint_as_float(v[4]) + b1.x, __uint_as_float(v[5]) + b1.y,
+                        __uint_as_float(v[6]) + b1.z, __uint_as_float(v[7]) + b1.w};
+          if (P.act == BSP_ACT_GELU) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) f[i] = gelu_erf(f[i]);
+          }
+          st_shared_v4(buf + row_off + ((static_cast<uint32_t>(j) ^ row_xor) << 4), pack_bf16x2(f[0], f[1]),
+                       pack_bf16x2(f[2], f[3]), pack_bf16x2(f[4], f[5]), pack_bf16x2(f[6], f[7]));
+        }
+        fence_async_smem();                  // make the staged piece visible to the TMA engine
+        epilogue_sync();
+        if (epi_tid == 0) {
+          tma_store_2d(&map_y, n0 + c0, m0, buf);   // rows beyond `tokens` / columns beyond `n_out` are clipped
+          tma_store_commit();
+        }
+        ++piece;
       }
-      tcgen05_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(acc_empty_bar(acc));
       acc_phase[acc] ^= 1u;
       acc ^= 1;
     }
+    if (epi_tid == 0) tma_store_wait_all();
     if (!ok && lane == 0) atomicExch(P.status, BSP_ERR_TIMEOUT);
   }
 
@@ -412,12 +465,15 @@ int choose_bn(int tokens, int n_out, int sms) {
 }
 
 template <int BN>
-int launch_tc(DeviceInfo* dev, int slot, const void* plan, const void* X, const LinearParams& P, int ldx,
-              cudaStream_t s) {
+int launch_tc(DeviceInfo* dev, int slot, const void* plan, const void* X, void* Y, const LinearParams& P, int ldx,
+              int ldy, cudaStream_t s) {
   using Cfg = TileCfg<BN>;
-  CUtensorMap map_x, map_w;
+  static_assert(Cfg::kStages >= 3, "pipeline too shallow");
+  static_assert(BN % kEpiCols == 0, "tile width must be a multiple of the epilogue piece");
+  CUtensorMap map_x, map_w, map_y;
   if (!make_map(&map_x, X, P.k_in, P.tokens, ldx, kBlockM)) return BSP_ERR_CUDA;
   if (!make_map(&map_w, plan, P.k_in, P.n_out, P.k_in, BN)) return BSP_ERR_CUDA;
+  if (!make_map(&map_y, Y, P.n_out, P.tokens, ldy, kBlockM)) return BSP_ERR_CUDA;
   if (!dev->attr_set[slot]) {
     BSP_CUDA_TRY(cudaFuncSetAttribute(linear_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes));
     dev->attr_set[slot] = true;
@@ -426,7 +482,7 @@ int launch_tc(DeviceInfo* dev, int slot, const void* plan, const void* X, const 
   const int n_tiles = (P.n_out + BN - 1) / BN;
   const int tiles = m_tiles * n_tiles;
   const int grid = tiles < dev->sms ? tiles : dev->sms;
-  linear_tc_kernel<BN><<<grid, kThreads, Cfg::kSmemBytes, s>>>(map_x, map_w, P);
+  linear_tc_kernel<BN><<<grid, kThreads, Cfg::kSmemBytes, s>>>(map_x, map_w, map_y, P);
   BSP_LAUNCH_CHECK();
   return BSP_OK;
 }
@@ -471,14 +527,13 @@ extern "C" int bsp_linear_planned(const void* plan, int n_out, int k_in, int blo
   if (tokens == 0) return BSP_OK;
   DeviceInfo* dev = device_info();
   if (dev == nullptr) return BSP_ERR_CUDA;
-  LinearParams P{tokens, n_out, k_in, ldy, act, static_cast<const uint16_t*>(bias), static_cast<uint16_t*>(Y),
-                 dev->status};
+  LinearParams P{tokens, n_out, k_in, act, static_cast<const uint16_t*>(bias), dev->status};
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   switch (choose_bn(tokens, n_out, dev->sms)) {
-    case 256: return launch_tc<256>(dev, 0, plan, X, P, ldx, s);
-    case 192: return launch_tc<192>(dev, 1, plan, X, P, ldx, s);
-    case 128: return launch_tc<128>(dev, 2, plan, X, P, ldx, s);
-    default: return launch_tc<64>(dev, 3, plan, X, P, ldx, s);
+    case 256: return launch_tc<256>(dev, 0, plan, X, Y, P, ldx, ldy, s);
+    case 192: return launch_tc<192>(dev, 1, plan, X, Y, P, ldx, ldy, s);
+    case 128: return launch_tc<128>(dev, 2, plan, X, Y, P, ldx, ldy, s);
+    default: return launch_tc<64>(dev, 3, plan, X, Y, P, ldx, ldy, s);
   }
 }
 
