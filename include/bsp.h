@@ -158,6 +158,7 @@ int bsp_apply_mask(void* W, int rows, int cols, int ldw, int block, int orient,
  * bsp_linear_plan_bytes (host): bytes of the private execution layout for a packed matrix.
  * bsp_linear_plan: builds that layout in `plan` (device, 256-byte aligned) from the canonical
  *   packed form; do it once per packed matrix, reuse for any number of bsp_linear_planned calls.
+ *   Needs k_in to be a multiple of 8 and at most 12288 (else BSP_ERR_UNSUPPORTED).
  * bsp_linear_planned: runs the layer from a plan.
  * bsp_linear: plan + run in one call, the plan living in ws (>= bsp_linear_plan_bytes).
  *

@@ -372,24 +372,39 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
   }
 }
 
-// Plan: scatter the packed tiles of one row-block back to natural column positions.
+// Plan: put the packed tiles of one row-block back at their natural column positions, zero
+// elsewhere.  grid = (row-blocks, row splits); one thread produces 8 adjacent columns of a row
+// (one 16-byte store), looking the columns up in a shared column -> kept-position table.
 __global__ void __launch_bounds__(256)
 plan_expand_kernel(const int32_t* __restrict__ blk_ptr, const int32_t* __restrict__ idx,
                    const uint16_t* __restrict__ vals, int k_in, int block, uint16_t* __restrict__ Wx) {
-  extern __shared__ int32_t s_pos[];      // column -> position in the kept list, or -1
+  extern __shared__ int16_t s_pos[];      // column -> position in the kept list, or -1 (k_in < 32768)
   const int b = blockIdx.x;
   const int lo = blk_ptr[b], kc = blk_ptr[b + 1] - lo;
   for (int k = threadIdx.x; k < k_in; k += blockDim.x) s_pos[k] = -1;
   __syncthreads();
-  for (int j = threadIdx.x; j < kc; j += blockDim.x) s_pos[idx[lo + j]] = j;
+  for (int j = threadIdx.x; j < kc; j += blockDim.x) s_pos[idx[lo + j]] = static_cast<int16_t>(j);
   __syncthreads();
   const uint16_t* tile = vals + static_cast<size_t>(block) * lo;
-  uint16_t* out = Wx + static_cast<size_t>(b) * block * k_in;
-  const int total = block * k_in;
-  for (int e = threadIdx.x; e < total; e += blockDim.x) {
-    const int r = e / k_in, k = e - r * k_in;
-    const int p = s_pos[k];
-    out[e] = p >= 0 ? tile[static_cast<size_t>(r) * kc + p] : static_cast<uint16_t>(0);
+  const int rows_per = (block + gridDim.y - 1) / gridDim.y;
+  const int r_lo = blockIdx.y * rows_per;
+  const int r_hi = min(block, r_lo + rows_per);
+  const int chunks = k_in >> 3;
+  for (int e = threadIdx.x; e < (r_hi - r_lo) * chunks; e += blockDim.x) {
+    const int r = r_lo + e / chunks, q = e % chunks;
+    const uint4 pos4 = *reinterpret_cast<const uint4*>(s_pos + (q << 3));
+    const uint32_t pw[4] = {pos4.x, pos4.y, pos4.z, pos4.w};
+    const uint16_t* trow = tile + static_cast<size_t>(r) * kc;
+    uint32_t out[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int p0 = static_cast<int16_t>(pw[i] & 0xffffu), p1 = static_cast<int16_t>(pw[i] >> 16);
+      const uint32_t v0 = p0 >= 0 ? __ldg(trow + p0) : 0u;
+      const uint32_t v1 = p1 >= 0 ? __ldg(trow + p1) : 0u;
+      out[i] = v0 | (v1 << 16);
+    }
+    *reinterpret_cast<uint4*>(Wx + (static_cast<size_t>(b) * block + r) * k_in + (q << 3)) =
+        make_uint4(out[0], out[1], out[2], out[3]);
   }
 }
 
@@ -512,7 +527,9 @@ extern "C" int bsp_linear_plan(const int32_t* blk_ptr, const int32_t* idx, const
   if (!aligned_to(plan, 256)) return BSP_ERR_ARG;
   if (plan_bytes < need) return BSP_ERR_WORKSPACE;
   if (k_in > 12288) return BSP_ERR_UNSUPPORTED;
-  plan_expand_kernel<<<n_out / block, 256, sizeof(int32_t) * k_in, static_cast<cudaStream_t>(stream)>>>(
+  if (k_in % 8) return BSP_ERR_UNSUPPORTED;
+  const int splits = block >= 4 ? 4 : 1;
+  plan_expand_kernel<<<dim3(n_out / block, splits), 256, sizeof(int16_t) * k_in, static_cast<cudaStream_t>(stream)>>>(
       blk_ptr, idx, static_cast<const uint16_t*>(vals), k_in, block, static_cast<uint16_t*>(plan));
   BSP_LAUNCH_CHECK();
   return BSP_OK;
