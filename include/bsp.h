@@ -127,6 +127,35 @@ int bsp_prune_pack(const void* W, int rows, int cols, int ldw, int block, int or
                    int64_t* kept_weights, void* ws, size_t ws_bytes, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * bsp_prune_pack_static — bsp_prune_pack for callers that cannot provide a workspace.
+ * (Library convenience; the paper has no counterpart to this call.)
+ *
+ * Some hosts of this library may not allocate device memory at the point where they prune: a
+ * serving process whose framework reserved the whole GPU for its own pool at start-up (a later
+ * cudaMalloc simply fails), a latency-critical thread that must avoid cudaMalloc/cudaFree because
+ * they can synchronise the device, or a plug-in that is handed input and output buffers and
+ * nothing else.  For them this variant keeps bsp_prune_pack's scratch (per-block counts and
+ * per-group flags) in a fixed array of BSP_STATIC_SCRATCH_BYTES inside the library's device
+ * image.  Each GPU on which the library is loaded holds that array until the process ends.
+ *
+ * Arguments, outputs, semantics and results are exactly those of bsp_prune_pack without
+ * ws/ws_bytes; inputs and outputs are still the caller's buffers.  The call itself allocates
+ * and frees nothing.
+ *  - Limit: shapes whose bsp_pack_bound workspace exceeds BSP_STATIC_SCRATCH_BYTES (about
+ *    800 thousand groups) are refused with BSP_ERR_UNSUPPORTED before anything is launched.
+ *  - The first call on each device looks up the array's device address (with that device
+ *    current); make that first call outside any stream capture.
+ *  - All calls on a device share the one array.  It needs no clearing between calls (each call
+ *    writes every scratch byte before reading it), but two calls that can overlap on the GPU —
+ *    different streams, or different host threads without ordering — race on it: serialise them.
+ */
+#define BSP_STATIC_SCRATCH_BYTES (4u << 20)
+int bsp_prune_pack_static(const void* W, int rows, int cols, int ldw, int block, int orient,
+                          float threshold, const float* threshold_dev, int keep_per_block,
+                          uint8_t* keep, int32_t* blk_ptr, int32_t* idx, void* vals,
+                          int64_t* kept_weights, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
  * bsp_percentile_threshold — Section 3.1: "prune ... according to our pre-set threshold or
  * percentile".  Per-matrix threshold for a target compression rate c = total/kept:
  * with G groups, r = floor(G * (1 - 1/c)) groups are to be removed; *threshold_out (device

@@ -51,6 +51,7 @@ _SIGNATURES = {
     "bsp_group_norms": (_i, [_vp, _i, _i, _i, _i, _i, _f, _i, _vp, _vp, _vp, _vp, _vp]),
     "bsp_pack_bound": (_i, [_i, _i, _i, _i, _szp, _szp, _szp]),
     "bsp_prune_pack": (_i, [_vp, _i, _i, _i, _i, _i, _f, _vp, _i, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "bsp_prune_pack_static": (_i, [_vp, _i, _i, _i, _i, _i, _f, _vp, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
     "bsp_percentile_threshold": (_i, [_vp, _i, _i, _i, _i, _i, _d, _vp, _vp, _sz, _vp]),
     "bsp_apply_mask": (_i, [_vp, _i, _i, _i, _i, _i, _vp, _vp]),
     "bsp_linear_plan_bytes": (_i, [_i, _i, _i, _szp]),
@@ -155,6 +156,16 @@ def bsp_prune_pack(W: torch.Tensor, out: PackedMatrix, threshold: float = 0.0,
                               keep_per_block, _ptr(out.keep), _ptr(out.blk_ptr), _ptr(out.idx), _ptr(out.vals),
                               _ptr(out.kept_weights), _ptr(out.ws), out.ws.numel(), _stream(stream)),
            "bsp_prune_pack")
+
+
+def bsp_prune_pack_static(W: torch.Tensor, out: PackedMatrix, threshold: float = 0.0,
+                          threshold_dev: Optional[torch.Tensor] = None, keep_per_block: int = -1, stream=None) -> None:
+    """bsp_prune_pack without a caller workspace: the scratch is a fixed array inside the library (out.ws is unused)."""
+    rows, cols = W.shape
+    _check(lib.bsp_prune_pack_static(_ptr(W), rows, cols, _ld(W), out.block, out.orient, threshold,
+                                     _ptr(threshold_dev), keep_per_block, _ptr(out.keep), _ptr(out.blk_ptr),
+                                     _ptr(out.idx), _ptr(out.vals), _ptr(out.kept_weights), _stream(stream)),
+           "bsp_prune_pack_static")
 
 
 def bsp_percentile_threshold(W: torch.Tensor, block: int, orient: int, rate: float, threshold_out: torch.Tensor,

@@ -371,6 +371,10 @@ apply_mask_kernel(uint16_t* __restrict__ W, Geometry G, const uint8_t* __restric
   if (!keep[slot]) W[static_cast<size_t>(i) * G.ldw + j] = 0;
 }
 
+// Fixed scratch for bsp_prune_pack_static: lives in the library's device image, so every GPU
+// that loads the library holds these bytes until the process exits.
+static __device__ __align__(256) unsigned char g_static_pack_scratch[BSP_STATIC_SCRATCH_BYTES];
+
 struct WsLayout {
   size_t counts_off, keep_off, sumsq_off, total;
 };
@@ -482,4 +486,35 @@ extern "C" int bsp_apply_mask(void* W, int rows, int cols, int ldw, int block, i
       static_cast<uint16_t*>(W), G, keep);
   BSP_LAUNCH_CHECK();
   return BSP_OK;
+}
+
+extern "C" int bsp_prune_pack_static(const void* W, int rows, int cols, int ldw, int block, int orient,
+                                     float threshold, const float* threshold_dev, int keep_per_block,
+                                     uint8_t* keep, int32_t* blk_ptr, int32_t* idx, void* vals,
+                                     int64_t* kept_weights, void* stream) {
+  using namespace bsp;
+  int st = check_matrix_args(W, rows, cols, ldw, block, orient);
+  if (st != BSP_OK) return st;
+  size_t need = 0;
+  st = bsp_pack_bound(rows, cols, block, orient, nullptr, nullptr, &need);
+  if (st != BSP_OK) return st;
+  if (need > static_cast<size_t>(BSP_STATIC_SCRATCH_BYTES)) return BSP_ERR_UNSUPPORTED;
+
+  // In host code the array's name is only a handle; the device address has to be asked for,
+  // once per device, while that device is current.
+  static void* scratch_of_device[64] = {nullptr};
+  int dev = -1;
+  BSP_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return BSP_ERR_UNSUPPORTED;
+  if (scratch_of_device[dev] == nullptr) {
+    void* ptr = nullptr;
+    BSP_CUDA_TRY(cudaGetSymbolAddress(&ptr, g_static_pack_scratch));
+    if (ptr == nullptr) return BSP_ERR_CUDA;
+    scratch_of_device[dev] = ptr;
+  }
+  // Every byte of the scratch that the kernels read (per-block counts, per-group flags) is
+  // written earlier in the same call, so nothing left over from the previous call is observed
+  // and nothing needs clearing.
+  return bsp_prune_pack(W, rows, cols, ldw, block, orient, threshold, threshold_dev, keep_per_block, keep, blk_ptr,
+                        idx, vals, kept_weights, scratch_of_device[dev], BSP_STATIC_SCRATCH_BYTES, stream);
 }
