@@ -142,7 +142,7 @@ class LayerOnDevice:
                 "Y": torch.empty((wl.tokens, spec.n_out), dtype=torch.int16, device=device),
             }
             self.lin.append(e)
-        self.kernels_per_step = 6 * len(self.lin)   # norms, flags, scan, compact, plan, gemm per matrix
+        self.kernels_per_step = 5 * len(self.lin)   # norms, flags, compact, plan, gemm per matrix
 
     def source(self, spec, outs):
         if spec.src == "x":
@@ -153,12 +153,34 @@ class LayerOnDevice:
         return outs[spec.src]
 
     def step(self, gemm_events=None):
-        bsp, outs = self.bsp, {}
+        """One pass of the path.  The weight-side work of the four matrices (norms/gamma/penalty on one
+        stream, prune/pack -> plan on another, per matrix) does not depend on activations, so it is issued
+        on side streams that fork from the current stream; the four GEMMs run in order on the current
+        stream, each after its own plan.  Under graph capture this becomes the graph's dependency structure."""
+        torch, bsp, outs = self.torch, self.bsp, {}
+        main = torch.cuda.current_stream()
+        if not hasattr(self, "side"):
+            self.side = [(torch.cuda.Stream(), torch.cuda.Stream()) for _ in self.lin]
+        fork = torch.cuda.Event()
+        fork.record(main)
+        ready = []
+        for e, (s_norm, s_pack) in zip(self.lin, self.side):
+            spec = e["spec"]
+            s_norm.wait_event(fork)
+            s_pack.wait_event(fork)
+            with torch.cuda.stream(s_norm):
+                bsp.bsp_group_norms(e["W"], spec.block, bsp.ORIENT_C, EPS, bsp.PEN_L2, e["norms"], None, e["gamma"], e["penalty"])
+                d_norm = torch.cuda.Event()
+                d_norm.record(s_norm)
+            with torch.cuda.stream(s_pack):
+                bsp.bsp_prune_pack(e["W"], e["pk"], 0.0)
+                bsp.bsp_linear_plan(e["pk"], e["plan"])
+                d_plan = torch.cuda.Event()
+                d_plan.record(s_pack)
+            ready.append((d_norm, d_plan))
         for i, e in enumerate(self.lin):
             spec = e["spec"]
-            bsp.bsp_group_norms(e["W"], spec.block, bsp.ORIENT_C, EPS, bsp.PEN_L2, e["norms"], None, e["gamma"], e["penalty"])
-            bsp.bsp_prune_pack(e["W"], e["pk"], 0.0)
-            bsp.bsp_linear_plan(e["pk"], e["plan"])
+            main.wait_event(ready[i][1])
             src = self.source(spec, outs)
             if gemm_events is not None:
                 gemm_events[i][0].record()
@@ -166,6 +188,8 @@ class LayerOnDevice:
             if gemm_events is not None:
                 gemm_events[i][1].record()
             outs[spec.name.split(".")[1]] = e["Y"]
+        for d_norm, _ in ready:
+            main.wait_event(d_norm)          # join: the step ends when the norm branches have ended too
         return outs
 
     def upload_inputs(self):
@@ -302,7 +326,8 @@ def run_cuda(args):
             "config": {
                 "workload": wl.name + " (one BERT-base encoder layer: QKV, attn-out, FFN-up+GELU, FFN-down; "
                             "tokens per GPU 4096; 16-row blocks; 3.0x compression)",
-                "step": "group norms+gamma+penalty, prune/pack, plan, linear for each of the 4 matrices, one CUDA graph",
+                "step": "group norms+gamma+penalty, prune/pack, plan, linear for each of the 4 matrices; one CUDA graph, "
+                        "weight-side kernels of the 4 matrices on parallel branches, the 4 GEMMs in sequence",
                 "l2": f"flushed between steps by writing {L2_FLUSH_BYTES >> 20} MiB",
                 "parallelism": "token split, replicated weights, no collective" if world > 1 else "single GPU",
                 "nonzero_gflop_per_step_per_gpu": round(step_flops / 1e9, 3),

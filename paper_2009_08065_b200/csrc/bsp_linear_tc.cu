@@ -15,11 +15,13 @@
 //                      (128-byte swizzle), completion on an mbarrier;
 //   warp 1 (one lane): issues tcgen05.mma (M=128, N=BN, K=16) into one of two TMEM accumulators
 //                      and commits stage release / accumulator ready to mbarriers;
-//   warps 2..5       : epilogue, tcgen05.ld the accumulator (each warp its 32 TMEM lanes = 32
-//                      tokens), add bias, optional GELU, round to bf16, stage 128 x 64 pieces in
-//                      swizzled shared memory and hand them to TMA stores (full-line writes,
-//                      tails clipped by the tensor map); it runs concurrently with the next
-//                      tile's main loop on the other accumulator.
+//   warps 2..9       : epilogue, two groups of four warps; group g takes the 64-column pieces of
+//                      the tile with index = g (mod 2).  Each warp tcgen05.ld's its 32 TMEM lanes
+//                      (= 32 tokens), adds bias, optional GELU, rounds to bf16, writes its rows
+//                      into the group's swizzled staging buffer, and one thread hands the
+//                      128 x 64 piece to a TMA store (full-line writes, tails clipped by the
+//                      tensor map).  The epilogue runs concurrently with the next tile's main
+//                      loop on the other accumulator.
 // Every wait is bounded by a wall-clock deadline; on expiry the role records BSP_ERR_TIMEOUT in
 // the status word and leaves its loop, the other roles then time out on their own waits, and
 // the CTA frees its tensor memory and exits.
@@ -38,7 +40,7 @@ namespace {
 constexpr int kBlockM = 128;      // tokens per tile (TMEM lanes)
 constexpr int kBlockK = 64;       // bf16 elements per pipeline stage row = 128 bytes = one swizzle row
 constexpr int kUmmaK = 16;        // K of one tcgen05.mma for 16-bit inputs
-constexpr int kThreads = 192;     // 6 warps: producer, mma, 4 epilogue
+constexpr int kThreads = 320;     // 10 warps: producer, mma, 2 x 4 epilogue
 constexpr int kSmemLimit = 232448;              // 227 KB of dynamic shared memory per CTA
 constexpr int kEpiCols = 64;                    // columns per epilogue piece = one 128-byte swizzle row of bf16
 constexpr int kEpiStage = kBlockM * kEpiCols * 2;
@@ -51,7 +53,7 @@ struct TileCfg {
   static constexpr int kStageA = kBlockM * kBlockK * 2;
   static constexpr int kStageB = BN * kBlockK * 2;
   static constexpr int kStage = kStageA + kStageB;
-  static constexpr int kFixed = 1024 /*alignment slack*/ + 2 * kEpiStage + BN * 4 /*bias*/ + 256 /*barriers*/;
+  static constexpr int kFixed = 1024 /*alignment slack*/ + 2 * kEpiStage + 2 * BN * 2 /*bias, two tiles*/ + 256 /*barriers*/;
   static constexpr int kStages = ((kSmemLimit - kFixed) / kStage) > 8 ? 8 : ((kSmemLimit - kFixed) / kStage);
   static constexpr int kTmemCols = 2 * BN <= 32 ? 32 : 2 * BN <= 64 ? 64 : 2 * BN <= 128 ? 128 : 2 * BN <= 256 ? 256 : 512;
   static constexpr int kSmemBytes = kStages * kStage + kFixed;
@@ -143,8 +145,10 @@ __device__ __forceinline__ void tma_store_wait_read() {
 }
 __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-// Barrier among the 128 epilogue threads only (barrier 0 is __syncthreads).
-__device__ __forceinline__ void epilogue_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+// Named barriers of the epilogue (barrier 0 is __syncthreads): 1 + g among the 128 threads of
+// epilogue group g, 3 among all 256 epilogue threads.
+__device__ __forceinline__ void group_sync(int g) { asm volatile("bar.sync %0, 128;" ::"r"(1 + g) : "memory"); }
+__device__ __forceinline__ void epilogue_sync_all() { asm volatile("bar.sync 3, 256;" ::: "memory"); }
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
   asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
@@ -167,18 +171,19 @@ __host__ __device__ constexpr uint32_t instr_desc_bf16(int n) {
          (static_cast<uint32_t>(kBlockM >> 4) << 24);
 }
 
-// GELU(x) = x * Phi(x) with Phi from the rational-exponential approximation of erfc published as
-// formula 7.1.26 in Abramowitz & Stegun's handbook (absolute error of erf below 1.5e-7, far under
-// the bf16 rounding of the output): erfc(z) ~ (a1 t + ... + a5 t^5) exp(-z^2), t = 1/(1 + p z),
-// z = |x| / sqrt(2).  Branch-free: Phi(x) = q for x < 0 and 1 - q otherwise, q = erfc(z) / 2.
+// GELU(x) = x * Phi(x), Phi the standard normal distribution function (the erf form, 0.5 (1 + erf(x / sqrt 2))).
+// The lower tail is evaluated as Phi(-a) = 2^(-P(a)), a = min(|x|, 6), with P a degree-5 polynomial
+// fitted by weighted least squares to -log2 Phi(-a) on [0, 6]; the largest absolute error of Phi in
+// float32 is 3.2e-7 (below 1e-9 beyond a = 6), far under the bf16 rounding of the output.  One
+// special-function operation (ex2) per element, no branch: Phi(x) = q for x < 0, 1 - q otherwise.
 __device__ __forceinline__ float gelu_erf(float x) {
-  const float z = fabsf(x) * 0.70710678118654752440f;
-  const float t = __fdividef(1.0f, fmaf(0.3275911f, z, 1.0f));
-  float poly = fmaf(1.061405429f, t, -1.453152027f);
-  poly = fmaf(poly, t, 1.421413741f);
-  poly = fmaf(poly, t, -0.284496736f);
-  poly = fmaf(poly, t, 0.254829592f);
-  const float q = 0.5f * poly * t * __expf(-z * z);
+  const float a = fminf(fabsf(x), 6.0f);
+  float p = fmaf(-0.000518865308f, a, 0.00738722592f);
+  p = fmaf(p, a, -0.0525380379f);
+  p = fmaf(p, a, -0.459276694f);
+  p = fmaf(p, a, -1.15108313f);
+  p = fmaf(p, a, -1.00000084f);
+  const float q = exp2f(p);   // maps to the hardware ex2 for arguments in this range
   return x * (x < 0.0f ? q : 1.0f - q);
 }
 
@@ -203,8 +208,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
   extern __shared__ uint8_t smem_raw[];
   // operand stages need 1024-byte alignment for the 128-byte swizzle pattern
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
-  // [S operand stages][2 epilogue staging buffers][bias as float][mbarriers, TMEM base]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S * Cfg::kStage + 2 * kEpiStage + BN * 4);
+  // [S operand stages][2 epilogue staging buffers][bias, bf16, for two tiles][mbarriers, TMEM base]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S * Cfg::kStage + 2 * kEpiStage + 2 * BN * 2);
   // bars[0..S) full, [S..2S) empty, [2S..2S+2) accumulator full, [2S+2..2S+4) accumulator empty
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 2 * S + 4);
 
@@ -218,7 +223,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(acc_full_bar(a), 1); mbar_init(acc_empty_bar(a), 4); }
+    for (int a = 0; a < 2; ++a) { mbar_init(acc_full_bar(a), 1); mbar_init(acc_empty_bar(a), 8); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -297,50 +302,58 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     if (!ok) atomicExch(P.status, BSP_ERR_TIMEOUT);
   } else if (warp >= 2) {
     // ---------------------------------------------------------------- epilogue
+    const int group = (warp - 2) >> 2;       // 0 or 1
     const int quad = warp & 3;               // TMEM lanes [32*quad, 32*quad+32) belong to this warp
     const int row = quad * 32 + lane;        // token row of this thread inside the tile
-    const int epi_tid = threadIdx.x - 64;    // 0..127 among the epilogue threads
-    const uint32_t stage_base = smem_base + S * Cfg::kStage;
-    float* s_bias = reinterpret_cast<float*>(smem + S * Cfg::kStage + 2 * kEpiStage);
+    const int epi_tid = threadIdx.x - 64;    // 0..255 among the epilogue threads
+    const bool issuer = (epi_tid & 127) == 0;  // the thread of each group that owns its TMA stores
+    const uint32_t buf = smem_base + S * Cfg::kStage + group * kEpiStage;   // this group's staging buffer
+    uint16_t* s_bias = reinterpret_cast<uint16_t*>(smem + S * Cfg::kStage + 2 * kEpiStage);  // [2][BN] bf16
     const uint32_t row_off = static_cast<uint32_t>(row) * 128u;
     const uint32_t row_xor = static_cast<uint32_t>(row & 7);
     uint32_t acc_phase[2] = {0u, 0u};
     int acc = 0;
-    uint32_t piece = 0;                      // pieces stored so far: selects the staging buffer
     bool ok = true;
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
       const int m0 = (tile / n_tiles) * kBlockM, n0 = (tile % n_tiles) * BN;
-      // bias of this tile's columns as float; readers of the previous tile's values are all past
-      // the last epilogue_sync of that tile, and the first one below publishes these
-      for (int c = epi_tid; c < BN; c += 128)
-        s_bias[c] = (P.bias != nullptr && n0 + c < P.n_out) ? bf16_bits_to_float(__ldg(P.bias + n0 + c)) : 0.0f;
+      // Bias of this tile's columns, in the half of s_bias that belongs to this accumulator.  The
+      // other group can lag by at most one tile (it has to reach the barrier below for this tile),
+      // so the values it may still be reading are in the other half.
+      for (int c = epi_tid; c < BN; c += 256)
+        s_bias[acc * BN + c] = (P.bias != nullptr && n0 + c < P.n_out) ? __ldg(P.bias + n0 + c) : static_cast<uint16_t>(0);
+      epilogue_sync_all();
       if (!mbar_wait(acc_full_bar(acc), acc_phase[acc])) { ok = false; break; }
       tcgen05_fence_after();
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + static_cast<uint32_t>(acc * BN);
       const int pieces = (min(BN, P.n_out - n0) + kEpiCols - 1) / kEpiCols;
+      bool released = false;
 #pragma unroll 1
-      for (int pc = 0; pc < pieces; ++pc) {
+      for (int pc = group; pc < pieces; pc += 2) {
         const int c0 = pc * kEpiCols;
-        const uint32_t buf = stage_base + (piece & 1u) * kEpiStage;
-        if (epi_tid == 0) tma_store_wait_read<1>();   // the store issued two pieces ago has read this buffer
-        epilogue_sync();
+        if (issuer) tma_store_wait_read<0>();   // this group's previous store has read the staging buffer
+        group_sync(group);
         uint32_t v0[32], v1[32];
         tmem_load_32cols(taddr + c0, v0);
         tmem_load_32cols(taddr + c0 + 32, v1);
         tmem_load_wait();
-        if (pc == pieces - 1) {              // accumulator fully read: the MMA warp may overwrite it
+        if (pc + 2 >= pieces) {              // this warp's last read of the accumulator
           tcgen05_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(acc_empty_bar(acc));
+          released = true;
         }
+        const uint16_t* bias_c = s_bias + acc * BN + c0;
 #pragma unroll
         for (int j = 0; j < 8; ++j) {        // 8 outputs -> one 16-byte piece of the swizzled staging row
           const uint32_t* v = j < 4 ? &v0[j * 8] : &v1[(j - 4) * 8];
-          const float4 b0 = *reinterpret_cast<const float4*>(s_bias + c0 + j * 8);
-          const float4 b1 = *reinterpret_cast<const float4*>(s_bias + c0 + j * 8 + 4);
-          float f[8] = {__uint_as_float(v[0]) + b0.x, __uint_as_float(v[1]) + b0.y, __uint_as_float(v[2]) + b0.z,
-                        __uint_as_float(v[3]) + b0.w, __uint_as_float(v[4]) + b1.x, __uint_as_float(v[5]) + b1.y,
-                        __uint_as_float(v[6]) + b1.z, __uint_as_float(v[7]) + b1.w};
+          const uint4 b8 = *reinterpret_cast<const uint4*>(bias_c + j * 8);
+          const uint32_t bw[4] = {b8.x, b8.y, b8.z, b8.w};
+          float f[8];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            f[2 * i] = __uint_as_float(v[2 * i]) + __uint_as_float(bw[i] << 16);
+            f[2 * i + 1] = __uint_as_float(v[2 * i + 1]) + __uint_as_float(bw[i] & 0xffff0000u);
+          }
           if (P.act == BSP_ACT_GELU) {
 #pragma unroll
             for (int i = 0; i < 8; ++i) f[i] = gelu_erf(f[i]);
@@ -349,17 +362,21 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                        pack_bf16x2(f[2], f[3]), pack_bf16x2(f[4], f[5]), pack_bf16x2(f[6], f[7]));
         }
         fence_async_smem();                  // make the staged piece visible to the TMA engine
-        epilogue_sync();
-        if (epi_tid == 0) {
+        group_sync(group);
+        if (issuer) {
           tma_store_2d(&map_y, n0 + c0, m0, buf);   // rows beyond `tokens` / columns beyond `n_out` are clipped
           tma_store_commit();
         }
-        ++piece;
+      }
+      if (!released) {                       // a group without a piece in this tile still releases the accumulator
+        tcgen05_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(acc_empty_bar(acc));
       }
       acc_phase[acc] ^= 1u;
       acc ^= 1;
     }
-    if (epi_tid == 0) tma_store_wait_all();
+    if (issuer) tma_store_wait_all();
     if (!ok && lane == 0) atomicExch(P.status, BSP_ERR_TIMEOUT);
   }
 
