@@ -3,8 +3,8 @@
 
 One *step* = one pass of the whole path over one batch of synthetic input, for each of the four
 linears of a BERT-base encoder layer at 4096 tokens (16-row blocks, 3.0x compression):
-    bsp_group_norms (norms, gamma, penalty)  ->  bsp_prune_pack (Algorithm 1 + packed storage)
-    ->  bsp_linear_plan  ->  bsp_linear_planned (tcgen05 GEMM + bias [+ GELU]),
+    norms, gamma, penalty  ->  Algorithm 1 keep flags + packed storage  ->  execution layout
+    (bsp_prepare_batched: one call for the four matrices)  ->  bsp_linear_planned (tcgen05 GEMM + bias [+ GELU]),
 with the layer's outputs chained (attention-output reads the V third of QKV's output, FFN-up
 reads attention-output's result through GELU, FFN-down reads FFN-up's).
 
@@ -142,7 +142,7 @@ class LayerOnDevice:
                 "Y": torch.empty((wl.tokens, spec.n_out), dtype=torch.int16, device=device),
             }
             self.lin.append(e)
-        self.kernels_per_step = 5 * len(self.lin)   # norms, flags, compact, plan, gemm per matrix
+        self.kernels_per_step = 2 + len(self.lin)   # two weight-side launches for the batch, one GEMM per matrix
 
     def source(self, spec, outs):
         if spec.src == "x":
@@ -153,34 +153,16 @@ class LayerOnDevice:
         return outs[spec.src]
 
     def step(self, gemm_events=None):
-        """One pass of the path.  The weight-side work of the four matrices (norms/gamma/penalty on one
-        stream, prune/pack -> plan on another, per matrix) does not depend on activations, so it is issued
-        on side streams that fork from the current stream; the four GEMMs run in order on the current
-        stream, each after its own plan.  Under graph capture this becomes the graph's dependency structure."""
-        torch, bsp, outs = self.torch, self.bsp, {}
-        main = torch.cuda.current_stream()
-        if not hasattr(self, "side"):
-            self.side = [(torch.cuda.Stream(), torch.cuda.Stream()) for _ in self.lin]
-        fork = torch.cuda.Event()
-        fork.record(main)
-        ready = []
-        for e, (s_norm, s_pack) in zip(self.lin, self.side):
-            spec = e["spec"]
-            s_norm.wait_event(fork)
-            s_pack.wait_event(fork)
-            with torch.cuda.stream(s_norm):
-                bsp.bsp_group_norms(e["W"], spec.block, bsp.ORIENT_C, EPS, bsp.PEN_L2, e["norms"], None, e["gamma"], e["penalty"])
-                d_norm = torch.cuda.Event()
-                d_norm.record(s_norm)
-            with torch.cuda.stream(s_pack):
-                bsp.bsp_prune_pack(e["W"], e["pk"], 0.0)
-                bsp.bsp_linear_plan(e["pk"], e["plan"])
-                d_plan = torch.cuda.Event()
-                d_plan.record(s_pack)
-            ready.append((d_norm, d_plan))
+        """One pass of the path: one batched weight-side call for the four matrices (norms, gamma, penalty,
+        keep flags, pack, plan: two launches), then the four GEMMs in order."""
+        bsp, outs = self.bsp, {}
+        if not hasattr(self, "jobs"):
+            self.jobs = bsp.make_job_array([
+                bsp.LayerJob(W=e["W"], out=e["pk"], threshold=0.0, norms=e["norms"], gamma_out=e["gamma"],
+                             penalty=e["penalty"], plan=e["plan"]) for e in self.lin])
+        bsp.bsp_prepare_batched(self.jobs, self.wl.linears[0].block, EPS, bsp.PEN_L2)
         for i, e in enumerate(self.lin):
             spec = e["spec"]
-            main.wait_event(ready[i][1])
             src = self.source(spec, outs)
             if gemm_events is not None:
                 gemm_events[i][0].record()
@@ -188,8 +170,6 @@ class LayerOnDevice:
             if gemm_events is not None:
                 gemm_events[i][1].record()
             outs[spec.name.split(".")[1]] = e["Y"]
-        for d_norm, _ in ready:
-            main.wait_event(d_norm)          # join: the step ends when the norm branches have ended too
         return outs
 
     def upload_inputs(self):
@@ -255,18 +235,25 @@ def run_cuda(args):
     flops = layer.nonzero_flops()
     step_flops = sum(flops)
 
-    # the step as a CUDA graph, with external timing events around the step and around each GEMM
+    # The step as a CUDA graph.  Two captures of the same call sequence: `graph` carries only the two
+    # events that bracket the step and gives `value`; `graph_k` also brackets every GEMM launch and gives
+    # the per-kernel durations of the roofline block (event nodes between kernels cost a few microseconds
+    # each, so they are kept out of the step that is timed as a whole).
     ev = lambda: torch.cuda.Event(enable_timing=True, external=True)  # noqa: E731
     ev_step = (ev(), ev())
     ev_gemm = [(ev(), ev()) for _ in layer.lin]
-    graph = torch.cuda.CUDAGraph()
+    graph, graph_k = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
     with torch.cuda.graph(graph):
         ev_step[0].record()
-        layer.step(gemm_events=ev_gemm)
+        layer.step()
         ev_step[1].record()
+    with torch.cuda.graph(graph_k):
+        layer.step(gemm_events=ev_gemm)
     for _ in range(max(args.warmup, 3)):
         flush.zero_()
         graph.replay()
+        flush.zero_()
+        graph_k.replay()
     torch.cuda.synchronize()
 
     def barrier():
@@ -282,6 +269,9 @@ def run_cuda(args):
             graph.replay()
             torch.cuda.synchronize()
             step_ms.append(ev_step[0].elapsed_time(ev_step[1]))
+            flush.zero_()
+            graph_k.replay()               # same step again, instrumented per kernel (not part of `value`)
+            torch.cuda.synchronize()
             for i, (a, b) in enumerate(ev_gemm):
                 gemm_ms[i].append(a.elapsed_time(b))
     barrier()
@@ -326,8 +316,8 @@ def run_cuda(args):
             "config": {
                 "workload": wl.name + " (one BERT-base encoder layer: QKV, attn-out, FFN-up+GELU, FFN-down; "
                             "tokens per GPU 4096; 16-row blocks; 3.0x compression)",
-                "step": "group norms+gamma+penalty, prune/pack, plan, linear for each of the 4 matrices; one CUDA graph, "
-                        "weight-side kernels of the 4 matrices on parallel branches, the 4 GEMMs in sequence",
+                "step": "bsp_prepare_batched (norms+gamma+penalty, keep flags, pack, plan of the 4 matrices: 2 launches) "
+                        "then the 4 GEMMs in sequence; one CUDA graph",
                 "l2": f"flushed between steps by writing {L2_FLUSH_BYTES >> 20} MiB",
                 "parallelism": "token split, replicated weights, no collective" if world > 1 else "single GPU",
                 "nonzero_gflop_per_step_per_gpu": round(step_flops / 1e9, 3),
@@ -336,7 +326,7 @@ def run_cuda(args):
             "e2e": {"value": round(world * step_flops * len(e2e_ms) / e2e_total_ms / 1e9, 3), "unit": UNIT,
                     "h2d_bytes_per_step": layer.h2d_bytes(),
                     "d2h_bytes_per_step": y_host.numel() * 2 + pen_host.numel() * 8},
-            "gpu_launches": layer.kernels_per_step * args.steps,
+            "gpu_launches": 2 * layer.kernels_per_step * args.steps,
             "clocks": clocks.summary(),
             "roofline": {
                 "kernel": "linear_tc_kernel (bsp_linear_planned), the four launches of a step",

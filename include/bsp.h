@@ -176,6 +176,32 @@ int bsp_apply_mask(void* W, int rows, int cols, int ldw, int block, int orient,
                    const uint8_t* keep, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * bsp_prepare_batched — the weight-side steps of the path for several matrices at once
+ * (orientation C): the norms / gamma / penalty of Section 3.2, Algorithm 1's keep decision, the
+ * packed storage of Section 3.1 and, optionally, bsp_linear's execution layout, in two launches
+ * for the whole batch instead of four or more per matrix.  Results are those of
+ * bsp_group_norms + bsp_prune_pack (threshold mode) + bsp_linear_plan called per matrix, bit
+ * for bit; the penalty is summed in a fixed order here and is reproducible run to run.
+ *
+ * jobs: HOST array of n_jobs descriptors; the pointers inside are device pointers with the
+ * meaning they have in the single-matrix calls.  norms, gamma_in, gamma_out, penalty, keep,
+ * kept_weights, plan may be NULL (that output is skipped).  ws/ws_bytes as bsp_prune_pack.
+ * block, eps and pen apply to every job.
+ * Needs, for every job: cols and ldw multiples of 8, W 16-byte aligned, cols <= 12288,
+ * rows/block <= 8192 (else BSP_ERR_UNSUPPORTED, and nothing is launched: use the per-matrix
+ * calls).  Other errors as the per-matrix calls; all jobs are validated before the first launch.
+ */
+typedef struct bsp_layer_job {
+  const void* W; int rows, cols, ldw;
+  float threshold; const float* threshold_dev;
+  float* norms; const float* gamma_in; float* gamma_out; double* penalty;
+  uint8_t* keep; int32_t* blk_ptr; int32_t* idx; void* vals; int64_t* kept_weights;
+  void* plan; size_t plan_bytes;
+  void* ws; size_t ws_bytes;
+} bsp_layer_job;
+int bsp_prepare_batched(const bsp_layer_job* jobs, int n_jobs, int block, float eps, int pen, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
  * bsp_linear — the pruned linear layer (orientation C packed form):
  *   Y[t, b*block + r] = act( sum_{j < kc_b} X[t, idx_b[j]] * vals_b[r, j] + bias[b*block + r] )
  * which equals act(X (W * Mask)^T + bias), the layer Algorithm 2 retrains (W = W * Mask) and

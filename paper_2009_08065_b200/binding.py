@@ -45,6 +45,18 @@ lib = _load()
 _vp, _i, _f, _d = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_double
 _sz, _szp = ctypes.c_size_t, ctypes.POINTER(ctypes.c_size_t)
 
+class _LayerJob(ctypes.Structure):
+    """Mirror of `bsp_layer_job` in bsp.h."""
+    _fields_ = [
+        ("W", _vp), ("rows", _i), ("cols", _i), ("ldw", _i),
+        ("threshold", _f), ("threshold_dev", _vp),
+        ("norms", _vp), ("gamma_in", _vp), ("gamma_out", _vp), ("penalty", _vp),
+        ("keep", _vp), ("blk_ptr", _vp), ("idx", _vp), ("vals", _vp), ("kept_weights", _vp),
+        ("plan", _vp), ("plan_bytes", _sz),
+        ("ws", _vp), ("ws_bytes", _sz),
+    ]
+
+
 _SIGNATURES = {
     "bsp_status_string": (ctypes.c_char_p, [_i]),
     "bsp_last_cuda_error": (_i, []),
@@ -54,6 +66,7 @@ _SIGNATURES = {
     "bsp_prune_pack_static": (_i, [_vp, _i, _i, _i, _i, _i, _f, _vp, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
     "bsp_percentile_threshold": (_i, [_vp, _i, _i, _i, _i, _i, _d, _vp, _vp, _sz, _vp]),
     "bsp_apply_mask": (_i, [_vp, _i, _i, _i, _i, _i, _vp, _vp]),
+    "bsp_prepare_batched": (_i, [ctypes.POINTER(_LayerJob), _i, _i, _f, _i, _vp]),
     "bsp_linear_plan_bytes": (_i, [_i, _i, _i, _szp]),
     "bsp_linear_plan": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _sz, _vp]),
     "bsp_linear_planned": (_i, [_vp, _i, _i, _i, _vp, _i, _i, _vp, _i, _vp, _i, _vp]),
@@ -179,6 +192,42 @@ def bsp_apply_mask(W: torch.Tensor, block: int, orient: int, keep: torch.Tensor,
     rows, cols = W.shape
     _check(lib.bsp_apply_mask(_ptr(W), rows, cols, _ld(W), block, orient, _ptr(keep), _stream(stream)),
            "bsp_apply_mask")
+
+
+@dataclass
+class LayerJob:
+    """One matrix of a bsp_prepare_batched call (tensors as in the single-matrix calls; None = skip)."""
+    W: torch.Tensor
+    out: PackedMatrix
+    threshold: float = 0.0
+    threshold_dev: Optional[torch.Tensor] = None
+    norms: Optional[torch.Tensor] = None
+    gamma_in: Optional[torch.Tensor] = None
+    gamma_out: Optional[torch.Tensor] = None
+    penalty: Optional[torch.Tensor] = None
+    plan: Optional[torch.Tensor] = None
+
+
+def make_job_array(jobs):
+    """The host descriptor array for bsp_prepare_batched; build it once and reuse it for repeated calls."""
+    arr = (_LayerJob * len(jobs))()
+    for a, j in zip(arr, jobs):
+        rows, cols = j.W.shape
+        a.W, a.rows, a.cols, a.ldw = _ptr(j.W), rows, cols, _ld(j.W)
+        a.threshold, a.threshold_dev = j.threshold, _ptr(j.threshold_dev)
+        a.norms, a.gamma_in, a.gamma_out, a.penalty = _ptr(j.norms), _ptr(j.gamma_in), _ptr(j.gamma_out), _ptr(j.penalty)
+        a.keep, a.blk_ptr, a.idx, a.vals = _ptr(j.out.keep), _ptr(j.out.blk_ptr), _ptr(j.out.idx), _ptr(j.out.vals)
+        a.kept_weights = _ptr(j.out.kept_weights)
+        a.plan = _ptr(j.plan)
+        a.plan_bytes = 0 if j.plan is None else j.plan.numel() * j.plan.element_size()
+        a.ws, a.ws_bytes = _ptr(j.out.ws), j.out.ws.numel()
+    return arr
+
+
+def bsp_prepare_batched(jobs, block: int, eps: float = 1e-3, pen: int = PEN_L2, stream=None) -> None:
+    """jobs: a list of LayerJob, or an array made by make_job_array."""
+    arr = jobs if isinstance(jobs, ctypes.Array) else make_job_array(jobs)
+    _check(lib.bsp_prepare_batched(arr, len(arr), block, eps, pen, _stream(stream)), "bsp_prepare_batched")
 
 
 def bsp_linear_plan_bytes(n_out: int, k_in: int, block: int) -> int:

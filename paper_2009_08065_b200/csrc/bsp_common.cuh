@@ -60,6 +60,22 @@ inline int check_matrix_args(const void* W, int rows, int cols, int ldw, int blo
   return BSP_OK;
 }
 
+// Workspace of the pack calls: [per-block counts][per-group flags][per-group float32 S], each
+// region 256-byte aligned.  (The fused call keeps per-block penalty partials in the S region.)
+struct WsLayout {
+  size_t counts_off, keep_off, sumsq_off, total;
+};
+inline WsLayout ws_layout(int n_blocks, int n_groups) {
+  WsLayout L;
+  const size_t groups = static_cast<size_t>(n_blocks) * n_groups;
+  L.counts_off = 0;
+  L.keep_off = round_up(sizeof(int32_t) * (static_cast<size_t>(n_blocks) + 1), 256);
+  L.sumsq_off = L.keep_off + round_up(groups, 256);
+  L.total = L.sumsq_off + round_up(groups * sizeof(float), 256);
+  return L;
+}
+
+
 #ifdef __CUDACC__
 __device__ __forceinline__ float bf16_bits_to_float(uint16_t b) {
   return __uint_as_float(static_cast<uint32_t>(b) << 16);
@@ -87,6 +103,87 @@ __device__ __forceinline__ int warp_sum(int v) {
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
   return v;
 }
+
+// Float32 sums of squares of 8 adjacent columns over the d rows of a row-block: eight independent
+// sequential chains, each the defined decision quantity of its group.
+__device__ __forceinline__ void sumsq8(const uint16_t* __restrict__ p, int d, int ldw, float (&acc)[8]) {
+#pragma unroll
+  for (int i = 0; i < 8; ++i) acc[i] = 0.0f;
+  int r = 0;
+  for (; r + 8 <= d; r += 8) {
+    uint4 v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) v[u] = __ldg(reinterpret_cast<const uint4*>(p + static_cast<size_t>(r + u) * ldw));
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const uint32_t w32[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float lo = __uint_as_float(w32[i] << 16), hi = __uint_as_float(w32[i] & 0xffff0000u);
+        acc[2 * i] = __fmaf_rn(lo, lo, acc[2 * i]);
+        acc[2 * i + 1] = __fmaf_rn(hi, hi, acc[2 * i + 1]);
+      }
+    }
+  }
+  for (; r < d; ++r) {
+    const uint4 v = __ldg(reinterpret_cast<const uint4*>(p + static_cast<size_t>(r) * ldw));
+    const uint32_t w32[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float lo = __uint_as_float(w32[i] << 16), hi = __uint_as_float(w32[i] & 0xffff0000u);
+      acc[2 * i] = __fmaf_rn(lo, lo, acc[2 * i]);
+      acc[2 * i + 1] = __fmaf_rn(hi, hi, acc[2 * i + 1]);
+    }
+  }
+}
+
+// Block-wide exclusive prefix sum of one int per thread (blockDim.x a multiple of 32, <= 1024).
+__device__ __forceinline__ int block_exclusive_scan(int v, int* s_warp, int* total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+  int incl = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int up = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += up;
+  }
+  if (lane == 31) s_warp[warp] = incl;
+  __syncthreads();
+  if (warp == 0) {
+    int w = lane < n_warps ? s_warp[lane] : 0;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int up = __shfl_up_sync(0xffffffffu, w, o);
+      if (lane >= o) w += up;
+    }
+    s_warp[lane] = w;  // inclusive totals of warps
+  }
+  __syncthreads();
+  const int before = warp ? s_warp[warp - 1] : 0;
+  *total = s_warp[n_warps - 1];
+  __syncthreads();  // s_warp may be reused by the caller's next round
+  return before + incl - v;
+}
+
+struct NormOut {
+  float* norms;
+  const float* gamma_in;
+  float* gamma_out;
+  double* penalty;
+  float eps;
+  int squared;  // 0: gamma = 1/(n+eps), term gamma*n ; 1: alpha = 1/(S+eps), term alpha*S
+};
+
+// Finishes one group from its float32 sum of squares; returns the group's penalty term.
+__device__ __forceinline__ double finish_group(const NormOut& o, size_t g, float S) {
+  const float n = __fsqrt_rn(S);
+  const float base = o.squared ? S : n;
+  const float fresh = __fdiv_rn(1.0f, base + o.eps);
+  if (o.norms) o.norms[g] = n;
+  if (o.gamma_out) o.gamma_out[g] = fresh;
+  const float weight = o.gamma_in ? o.gamma_in[g] : fresh;
+  return static_cast<double>(weight) * static_cast<double>(base);
+}
+
 #endif  // __CUDACC__
 
 }  // namespace bsp

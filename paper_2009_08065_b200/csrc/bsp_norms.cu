@@ -12,26 +12,6 @@ int& last_cuda_error_ref() {
 
 namespace {
 
-struct NormOut {
-  float* norms;
-  const float* gamma_in;
-  float* gamma_out;
-  double* penalty;
-  float eps;
-  int squared;  // 0: gamma = 1/(n+eps), term gamma*n ; 1: alpha = 1/(S+eps), term alpha*S
-};
-
-// Finishes one group from its float32 sum of squares; returns the group's penalty term.
-__device__ __forceinline__ double finish_group(const NormOut& o, size_t g, float S) {
-  const float n = __fsqrt_rn(S);
-  const float base = o.squared ? S : n;
-  const float fresh = __fdiv_rn(1.0f, base + o.eps);
-  if (o.norms) o.norms[g] = n;
-  if (o.gamma_out) o.gamma_out[g] = fresh;
-  const float weight = o.gamma_in ? o.gamma_in[g] : fresh;
-  return static_cast<double>(weight) * static_cast<double>(base);
-}
-
 __device__ __forceinline__ void add_penalty(const NormOut& o, double local) {
   if (o.penalty == nullptr) return;  // uniform across the grid
   local = warp_sum(local);

@@ -87,33 +87,6 @@ flags_topk_kernel(const uint16_t* __restrict__ W, Geometry G, int keep_count,
   if (threadIdx.x == 0) counts[b] = keep_count < G.n_groups ? keep_count : G.n_groups;
 }
 
-// Block-wide exclusive prefix sum of one int per thread (blockDim.x a multiple of 32, <= 1024).
-__device__ __forceinline__ int block_exclusive_scan(int v, int* s_warp, int* total) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
-  int incl = v;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const int up = __shfl_up_sync(0xffffffffu, incl, o);
-    if (lane >= o) incl += up;
-  }
-  if (lane == 31) s_warp[warp] = incl;
-  __syncthreads();
-  if (warp == 0) {
-    int w = lane < n_warps ? s_warp[lane] : 0;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const int up = __shfl_up_sync(0xffffffffu, w, o);
-      if (lane >= o) w += up;
-    }
-    s_warp[lane] = w;  // inclusive totals of warps
-  }
-  __syncthreads();
-  const int before = warp ? s_warp[warp - 1] : 0;
-  *total = s_warp[n_warps - 1];
-  __syncthreads();  // s_warp may be reused by the caller's next round
-  return before + incl - v;
-}
-
 // (2) counts -> blk_ptr (exclusive scan) and the kept-weight total.
 __global__ void __launch_bounds__(1024)
 scan_counts_kernel(const int32_t* __restrict__ counts, int n_blocks, int block,
@@ -171,39 +144,6 @@ compact_kernel(const uint16_t* __restrict__ W, Geometry G, const uint8_t* __rest
 // ------------------------------------------------------------------------------------------
 // Orientation C fast path (cols, ldw multiples of 8; W 16-byte aligned; keep 8-byte aligned)
 // ------------------------------------------------------------------------------------------
-
-// Float32 sums of squares of 8 adjacent columns over the d rows of a row-block: eight independent
-// sequential chains, each the defined decision quantity of its group.
-__device__ __forceinline__ void sumsq8(const uint16_t* __restrict__ p, int d, int ldw, float (&acc)[8]) {
-#pragma unroll
-  for (int i = 0; i < 8; ++i) acc[i] = 0.0f;
-  int r = 0;
-  for (; r + 8 <= d; r += 8) {
-    uint4 v[8];
-#pragma unroll
-    for (int u = 0; u < 8; ++u) v[u] = __ldg(reinterpret_cast<const uint4*>(p + static_cast<size_t>(r + u) * ldw));
-#pragma unroll
-    for (int u = 0; u < 8; ++u) {
-      const uint32_t w32[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const float lo = __uint_as_float(w32[i] << 16), hi = __uint_as_float(w32[i] & 0xffff0000u);
-        acc[2 * i] = __fmaf_rn(lo, lo, acc[2 * i]);
-        acc[2 * i + 1] = __fmaf_rn(hi, hi, acc[2 * i + 1]);
-      }
-    }
-  }
-  for (; r < d; ++r) {
-    const uint4 v = __ldg(reinterpret_cast<const uint4*>(p + static_cast<size_t>(r) * ldw));
-    const uint32_t w32[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const float lo = __uint_as_float(w32[i] << 16), hi = __uint_as_float(w32[i] & 0xffff0000u);
-      acc[2 * i] = __fmaf_rn(lo, lo, acc[2 * i]);
-      acc[2 * i + 1] = __fmaf_rn(hi, hi, acc[2 * i + 1]);
-    }
-  }
-}
 
 // (1) threshold mode, vectorised: one thread per 8 columns of one row-block.
 __global__ void __launch_bounds__(kPackThreads)
@@ -374,19 +314,6 @@ apply_mask_kernel(uint16_t* __restrict__ W, Geometry G, const uint8_t* __restric
 // Fixed scratch for bsp_prune_pack_static: lives in the library's device image, so every GPU
 // that loads the library holds these bytes until the process exits.
 static __device__ __align__(256) unsigned char g_static_pack_scratch[BSP_STATIC_SCRATCH_BYTES];
-
-struct WsLayout {
-  size_t counts_off, keep_off, sumsq_off, total;
-};
-WsLayout ws_layout(int n_blocks, int n_groups) {
-  WsLayout L;
-  const size_t groups = static_cast<size_t>(n_blocks) * n_groups;
-  L.counts_off = 0;
-  L.keep_off = round_up(sizeof(int32_t) * (static_cast<size_t>(n_blocks) + 1), 256);
-  L.sumsq_off = L.keep_off + round_up(groups, 256);
-  L.total = L.sumsq_off + round_up(groups * sizeof(float), 256);
-  return L;
-}
 
 }  // namespace
 }  // namespace bsp

@@ -88,6 +88,14 @@ def test_argument_errors_are_caught_before_any_launch():
     assert lib.bsp_linear(p, p, p, 10, 8, 4, p, 4, 8, None, 0, p, 16, ws, 1 << 20, None) == -2
     assert lib.bsp_linear_planned(ws, 8, 8, 4, p, 4, 8, None, 7, p, 8, None) == -1
     assert lib.bsp_linear_plan(p, p, p, 8, 8, 4, ws, 16, None) == -3
+    # batched weight-side call: null / empty job list, bad enum
+    assert lib.bsp_prepare_batched(None, 1, 16, 1e-3, 0, None) == -1
+    job = binding._LayerJob()
+    assert lib.bsp_prepare_batched(ctypes.pointer(job), 0, 16, 1e-3, 0, None) == -1
+    assert lib.bsp_prepare_batched(ctypes.pointer(job), 1, 16, 1e-3, 5, None) == -1
+    assert lib.bsp_prepare_batched(ctypes.pointer(job), 1, 16, 1e-3, 0, None) == -1      # W is NULL
+    job.W, job.rows, job.cols, job.ldw = 0x1000, 40, 64, 64
+    assert lib.bsp_prepare_batched(ctypes.pointer(job), 1, 16, 1e-3, 0, None) == -2      # 16 does not divide 40
     # zero tokens is a valid no-op
     assert lib.bsp_linear_cuda_core(p, p, p, 8, 8, 4, p, 0, 8, None, 0, p, 8, None) == 0
 

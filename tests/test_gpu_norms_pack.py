@@ -176,3 +176,87 @@ def test_apply_mask_matches_pruned_weight():
         bsp.bsp_apply_mask(wd, block, orient, torch.from_numpy(keep.astype(np.uint8)).to(DEV))
         torch.cuda.synchronize()
         assert np.array_equal(bits_of(wd), O.prune(w, block, o, t))      # Algorithm 1's W_p = W * Mask
+
+
+# ---------------------------------------------------------------------------------------- fused, batched
+def test_prepare_batched_matches_oracle_and_single_calls():
+    """One call for four matrices of different shapes: norms, gamma, penalty, flags, pack and plan."""
+    eps, block = 1e-3, 16
+    shapes = [(2304, 768), (768, 768), (3072, 768), (768, 3072)]
+    jobs, refs = [], []
+    for n, (rows, cols) in enumerate(shapes):
+        w = si.student_t_bf16(50 + n, f"batched{n}", (rows, cols), 3.0, 0.02)
+        t_b = float(np.quantile(O.group_norms(w, block, "C"), 0.55 + 0.1 * n))
+        pk = bsp.PackedMatrix.allocate(rows, cols, block, bsp.ORIENT_C, DEV)
+        pk.idx.fill_(-7)
+        shape = (rows // block, cols)
+        job = bsp.LayerJob(
+            W=to_dev(w), out=pk, threshold=t_b,
+            norms=torch.empty(shape, dtype=torch.float32, device=DEV),
+            gamma_out=torch.empty(shape, dtype=torch.float32, device=DEV),
+            penalty=torch.full((1,), -5.0, dtype=torch.float64, device=DEV),
+            plan=torch.empty(bsp.bsp_linear_plan_bytes(rows, cols, block), dtype=torch.uint8, device=DEV))
+        jobs.append(job)
+        refs.append((w, t_b))
+    bsp.bsp_prepare_batched(jobs, block, eps, bsp.PEN_L2)
+    torch.cuda.synchronize()
+    for job, (w, t_b) in zip(jobs, refs):
+        rows, cols = w.shape
+        n_ref = O.group_norms(w, block, "C")
+        g_ref = O.gamma_update(n_ref, eps)
+        assert np.allclose(job.norms.cpu().numpy(), n_ref, rtol=REL, atol=0)
+        assert np.allclose(job.gamma_out.cpu().numpy(), g_ref, rtol=REL, atol=0)
+        assert float(job.penalty.item()) == pytest.approx(O.penalty_l2(n_ref, g_ref), rel=REL)
+        keep_ref = O.keep_flags(w, block, "C", t_b)
+        ref_ptr, ref_idx, ref_vals = O.pack(w, keep_ref, block, "C")
+        blk_ptr, idx, vals, keep, kept = packed_to_host(job.out)
+        assert np.array_equal(keep, keep_ref) and np.array_equal(blk_ptr, ref_ptr)
+        assert np.array_equal(idx, ref_idx) and np.array_equal(vals, ref_vals)
+        assert kept == block * int(keep_ref.sum())
+        plan = bits_of(job.plan.view(torch.int16)[: rows * cols].reshape(rows, cols))
+        assert np.array_equal(plan, O.prune(w, block, "C", t_b))          # W * Mask, densely laid out
+        # and the per-matrix calls give the same bits
+        single = bsp.PackedMatrix.allocate(rows, cols, block, bsp.ORIENT_C, DEV)
+        bsp.bsp_prune_pack(job.W, single, t_b)
+        plan1 = torch.empty_like(job.plan)
+        bsp.bsp_linear_plan(single, plan1)
+        norms1 = torch.empty_like(job.norms)
+        bsp.bsp_group_norms(job.W, block, bsp.ORIENT_C, eps, bsp.PEN_L2, norms1)
+        torch.cuda.synchronize()
+        assert torch.equal(norms1, job.norms) and torch.equal(plan1[: rows * cols * 2], job.plan[: rows * cols * 2])
+        assert torch.equal(single.blk_ptr, job.out.blk_ptr)
+    # repeated call: penalty is reproducible bit for bit
+    first = [float(j.penalty.item()) for j in jobs]
+    bsp.bsp_prepare_batched(jobs, block, eps, bsp.PEN_L2)
+    torch.cuda.synchronize()
+    assert [float(j.penalty.item()) for j in jobs] == first
+
+
+def test_prepare_batched_optional_outputs_and_many_jobs():
+    """More jobs than one launch holds, outputs skipped, the squared-norm penalty, stale gamma."""
+    eps, block = 1e-2, 8
+    jobs, ws = [], []
+    for n in range(19):
+        w = si.normal_bf16(70 + n, f"many{n}", (64 + 8 * n, 72), 0.02)
+        pk = bsp.PackedMatrix.allocate(w.shape[0], 72, block, bsp.ORIENT_C, DEV)
+        stale = (np.abs(si.bf16_bits_to_f32(si.normal_bf16(90 + n, "g", (w.shape[0] // block, 72), 1.0))) + 0.5).astype(np.float32)
+        jobs.append(bsp.LayerJob(W=to_dev(w), out=pk, threshold=0.05,
+                                 gamma_in=torch.from_numpy(stale).to(DEV) if n % 2 else None,
+                                 penalty=torch.zeros(1, dtype=torch.float64, device=DEV)))
+        ws.append((w, stale if n % 2 else None))
+    bsp.bsp_prepare_batched(jobs, block, eps, bsp.PEN_L2SQ)
+    torch.cuda.synchronize()
+    for job, (w, stale) in zip(jobs, ws):
+        s_ref = O.group_sumsq(w, block, "C")
+        alpha = stale.astype(np.float64) if stale is not None else O.alpha_update_sq(s_ref, eps)
+        assert float(job.penalty.item()) == pytest.approx(O.penalty_l2sq(s_ref, alpha), rel=REL)
+        keep_ref = O.keep_flags(w, block, "C", 0.05)
+        ref_ptr, ref_idx, ref_vals = O.pack(w, keep_ref, block, "C")
+        blk_ptr, idx, vals, keep, kept = packed_to_host(job.out)
+        assert np.array_equal(blk_ptr, ref_ptr) and np.array_equal(idx, ref_idx) and np.array_equal(vals, ref_vals)
+    # shapes the fused kernels do not take are refused as a whole
+    odd = si.normal_bf16(1, "odd", (16, 50), 0.02)
+    pk = bsp.PackedMatrix.allocate(16, 50, 8, bsp.ORIENT_C, DEV)
+    with pytest.raises(bsp.BspError) as e:
+        bsp.bsp_prepare_batched([jobs[0], bsp.LayerJob(W=to_dev(odd), out=pk)], 8)
+    assert e.value.status == -6
