@@ -187,9 +187,9 @@ int bsp_apply_mask(void* W, int rows, int cols, int ldw, int block, int orient,
  * meaning they have in the single-matrix calls.  norms, gamma_in, gamma_out, penalty, keep,
  * kept_weights, plan may be NULL (that output is skipped).  ws/ws_bytes as bsp_prune_pack.
  * block, eps and pen apply to every job.
- * Needs, for every job: cols and ldw multiples of 8, W 16-byte aligned, cols <= 12288,
- * rows/block <= 8192 (else BSP_ERR_UNSUPPORTED, and nothing is launched: use the per-matrix
- * calls).  Other errors as the per-matrix calls; all jobs are validated before the first launch.
+ * Needs, for every job: cols and ldw multiples of 8, W and the float arrays 16-byte aligned,
+ * cols <= 4096, rows/block <= 1024 (else BSP_ERR_UNSUPPORTED, and nothing is launched: use the
+ * per-matrix calls).  Other errors as the per-matrix calls; all jobs are validated before the first launch.
  */
 typedef struct bsp_layer_job {
   const void* W; int rows, cols, ldw;

@@ -76,6 +76,38 @@ inline WsLayout ws_layout(int n_blocks, int n_groups) {
 }
 
 
+// One matrix of a launch of the vectorised orientation-C kernels (bsp_fused.cu).  Null output
+// pointers switch the matching work off.
+struct FusedJob {
+  const uint16_t* W;
+  int rows, cols, ldw, n_blocks;
+  float threshold;
+  const float* threshold_dev;
+  float* norms;
+  const float* gamma_in;
+  float* gamma_out;
+  double* penalty;             // job total (written by stage 2 from `partial`, or by atomics in stage 1)
+  double* partial;             // per-block penalty partial sums, or null: stage 1 adds into *penalty
+  uint8_t* flags;              // per-group keep flags (null: stage 1 skips the keep decision)
+  int32_t* counts;             // per-block kept counts
+  int32_t* blk_ptr;
+  int32_t* idx;
+  uint16_t* vals;
+  int64_t* kept_weights;
+  uint16_t* plan;
+};
+constexpr int kFusedMaxJobs = 16;
+constexpr int kFusedMaxCols = 4096;     // stage 2 keeps 12 bytes of shared memory per column
+constexpr int kFusedMaxBlocks = 1024;   // stage 2 sums the counts before its block directly
+// Stage 1: sums of squares -> norms / gamma / penalty and/or keep flags + counts, one pass over W.
+int fused_stage1(const FusedJob* jobs, int n_jobs, int block, float eps, int squared, cudaStream_t s);
+// Stage 2: blk_ptr, index lists, packed tiles, penalty totals, optional execution layout.
+int fused_stage2(const FusedJob* jobs, int n_jobs, int block, cudaStream_t s);
+// Whether a matrix can go through the vectorised kernels.
+inline bool fused_shape_ok(const void* W, int rows, int cols, int ldw, int block) {
+  return cols % 8 == 0 && ldw % 8 == 0 && aligned_to(W, 16) && cols <= kFusedMaxCols && rows / block <= kFusedMaxBlocks;
+}
+
 #ifdef __CUDACC__
 __device__ __forceinline__ float bf16_bits_to_float(uint16_t b) {
   return __uint_as_float(static_cast<uint32_t>(b) << 16);

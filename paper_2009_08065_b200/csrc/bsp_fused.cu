@@ -1,38 +1,27 @@
-// bsp_prepare_batched: for a batch of weight matrices (orientation C), everything the path does
-// on the weight side in two launches — (1) group norms, gamma, penalty partials, keep flags and
-// per-block counts in one pass over W; (2) blk_ptr, ascending index lists, packed tiles, the
-// penalty total, and (optionally) the linear layer's execution layout.  Results are bit-identical
-// to bsp_group_norms + bsp_prune_pack + bsp_linear_plan called per matrix (the penalty up to its
-// summation order, which here is fixed, so it is reproducible run to run).
+// Vectorised orientation-C kernels shared by bsp_group_norms, bsp_prune_pack and
+// bsp_prepare_batched.  Two stages over a batch of matrices:
+//   stage 1  one CTA per row-block, one thread per 8 adjacent columns: 16-byte loads down the
+//            block's rows (8 rows in flight), eight independent sequential float32 sums of
+//            squares (the defined decision quantity), then any of: norms / gamma (two 16-byte
+//            stores each), penalty partial, keep flags (one 8-byte store) and the block's count.
+//   stage 2  grid (row-blocks, groups of 4 rows): blk_ptr from the counts before the block, the
+//            ascending index list from the flags, the rows staged once in shared memory (16-byte
+//            loads) and from there (a) the zero-expanded execution layout, (b) the packed tile,
+//            written as 16-byte vectors wherever the output is 16-byte aligned.
+#include <new>
+
 #include "bsp_common.cuh"
 
 namespace bsp {
 namespace {
 
-constexpr int kMaxJobs = 16;
-constexpr int kThreads = 256;
-
-struct Job {
-  const uint16_t* W;
-  int rows, cols, ldw, n_blocks;
-  float threshold;
-  const float* threshold_dev;
-  NormOut out;                 // norms / gamma_in / gamma_out / (penalty unused here) / eps / squared
-  double* penalty;
-  uint8_t* flags;
-  int32_t* counts;
-  double* partial;             // per-block penalty partial sums
-  int32_t* blk_ptr;
-  int32_t* idx;
-  uint16_t* vals;
-  int64_t* kept_weights;
-  uint16_t* plan;
-};
+constexpr int kRowsPerCta = 4;
 
 struct Batch {
-  int n_jobs, block;
-  int first_block[kMaxJobs + 1];   // CTA index of each job's first row-block
-  Job job[kMaxJobs];
+  int n_jobs, block, squared;
+  float eps;
+  int first_block[kFusedMaxJobs + 1];   // CTA index of each job's first row-block
+  FusedJob job[kFusedMaxJobs];
 };
 
 __device__ __forceinline__ int find_job(const Batch& B, int cta) {
@@ -41,68 +30,107 @@ __device__ __forceinline__ int find_job(const Batch& B, int cta) {
   return j;
 }
 
-// (1) one CTA per row-block of some job; one thread per 8 adjacent columns.
-__global__ void __launch_bounds__(kThreads)
-fused_norms_flags_kernel(const __grid_constant__ Batch B) {
-  __shared__ int s_cnt[kThreads / 32];
-  __shared__ double s_pen[kThreads / 32];
+__global__ void __launch_bounds__(256)
+fused_stage1_kernel(const __grid_constant__ Batch B) {
+  __shared__ int s_cnt[8];
+  __shared__ double s_pen[8];
   const int j = find_job(B, blockIdx.x);
-  const Job& J = B.job[j];
+  const FusedJob& J = B.job[j];
   const int b = blockIdx.x - B.first_block[j];
-  const float t = J.threshold_dev ? *J.threshold_dev : J.threshold;
-  const bool keep_all = t < 0.0f;
-  const float t2 = __fmul_rn(t, t);
-  const bool want_norms = J.out.norms || J.out.gamma_out || J.penalty;
-  NormOut o = J.out;
+  const bool want_flags = J.flags != nullptr;
+  const bool want_pen = J.penalty != nullptr;
+  const bool want_norms = J.norms != nullptr || J.gamma_out != nullptr || want_pen;
+  float t2 = 0.0f;
+  bool keep_all = false;
+  if (want_flags) {
+    const float t = J.threshold_dev ? *J.threshold_dev : J.threshold;
+    keep_all = t < 0.0f;
+    t2 = __fmul_rn(t, t);
+  }
   int count = 0;
-  double pen = 0.0;
+  float pen = 0.0f;
   for (int q = threadIdx.x; q < (J.cols >> 3); q += blockDim.x) {
     float acc[8];
     sumsq8(J.W + static_cast<size_t>(b) * B.block * J.ldw + (q << 3), B.block, J.ldw, acc);
-    uint32_t lo = 0, hi = 0;
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const uint32_t k0 = (keep_all || acc[i] > t2) ? 1u : 0u;
-      const uint32_t k1 = (keep_all || acc[4 + i] > t2) ? 1u : 0u;
-      lo |= k0 << (8 * i);
-      hi |= k1 << (8 * i);
-      count += static_cast<int>(k0 + k1);
-    }
     const size_t g0 = static_cast<size_t>(b) * J.cols + (q << 3);
-    *reinterpret_cast<uint2*>(J.flags + g0) = make_uint2(lo, hi);
-    if (want_norms) {
+    if (want_flags) {
+      uint32_t lo = 0, hi = 0;
 #pragma unroll
-      for (int i = 0; i < 8; ++i) pen += finish_group(o, g0 + i, acc[i]);
+      for (int i = 0; i < 4; ++i) {
+        const uint32_t k0 = (keep_all || acc[i] > t2) ? 1u : 0u;
+        const uint32_t k1 = (keep_all || acc[4 + i] > t2) ? 1u : 0u;
+        lo |= k0 << (8 * i);
+        hi |= k1 << (8 * i);
+        count += static_cast<int>(k0 + k1);
+      }
+      *reinterpret_cast<uint2*>(J.flags + g0) = make_uint2(lo, hi);
+    }
+    if (want_norms) {
+      float n[8], base[8], fresh[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        n[i] = __fsqrt_rn(acc[i]);
+        base[i] = B.squared ? acc[i] : n[i];
+        fresh[i] = __fdiv_rn(1.0f, base[i] + B.eps);
+      }
+      if (J.norms) {
+        *reinterpret_cast<float4*>(J.norms + g0) = make_float4(n[0], n[1], n[2], n[3]);
+        *reinterpret_cast<float4*>(J.norms + g0 + 4) = make_float4(n[4], n[5], n[6], n[7]);
+      }
+      if (J.gamma_out) {
+        *reinterpret_cast<float4*>(J.gamma_out + g0) = make_float4(fresh[0], fresh[1], fresh[2], fresh[3]);
+        *reinterpret_cast<float4*>(J.gamma_out + g0 + 4) = make_float4(fresh[4], fresh[5], fresh[6], fresh[7]);
+      }
+      if (want_pen) {
+        if (J.gamma_in) {
+          const float4 a = __ldg(reinterpret_cast<const float4*>(J.gamma_in + g0));
+          const float4 c = __ldg(reinterpret_cast<const float4*>(J.gamma_in + g0 + 4));
+          const float w[8] = {a.x, a.y, a.z, a.w, c.x, c.y, c.z, c.w};
+#pragma unroll
+          for (int i = 0; i < 8; ++i) pen = fmaf(w[i], base[i], pen);
+        } else {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) pen = fmaf(fresh[i], base[i], pen);
+        }
+      }
     }
   }
+  // block totals: count (int) and penalty (float per thread, float64 from here on, fixed order)
   count = warp_sum(count);
-  pen = warp_sum(pen);
-  const int warp = threadIdx.x >> 5;
-  if ((threadIdx.x & 31) == 0) { s_cnt[warp] = count; s_pen[warp] = pen; }
+  double pd = warp_sum(static_cast<double>(pen));
+  const int warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+  if ((threadIdx.x & 31) == 0) { s_cnt[warp] = count; s_pen[warp] = pd; }
   __syncthreads();
   if (threadIdx.x == 0) {
     int c = 0;
     double p = 0.0;
-    for (int w = 0; w < kThreads / 32; ++w) { c += s_cnt[w]; p += s_pen[w]; }   // fixed order
-    J.counts[b] = c;
-    J.partial[b] = p;
+    for (int w = 0; w < n_warps; ++w) { c += s_cnt[w]; p += s_pen[w]; }
+    if (want_flags) J.counts[b] = c;
+    if (want_pen) {
+      if (J.partial) J.partial[b] = p;
+      else if (p != 0.0) atomicAdd(J.penalty, p);
+    }
   }
 }
 
-// (2) grid = (row-blocks of all jobs, row splits).
-__global__ void __launch_bounds__(kThreads)
-fused_compact_plan_kernel(const __grid_constant__ Batch B) {
-  extern __shared__ int32_t s_idx[];   // kept column indices of this block, ascending
+__global__ void __launch_bounds__(256)
+fused_stage2_kernel(const __grid_constant__ Batch B) {
+  extern __shared__ __align__(16) uint8_t s_raw[];
   __shared__ int s_warp[32];
-  __shared__ double s_red[kThreads / 32];
+  __shared__ double s_red[8];
   __shared__ int s_base;
   const int j = find_job(B, blockIdx.x);
-  const Job& J = B.job[j];
+  const FusedJob& J = B.job[j];
   const int b = blockIdx.x - B.first_block[j];
   const int d = B.block;
+  const int r_lo = blockIdx.y * kRowsPerCta;
+  if (r_lo >= d) return;
+  const int r_hi = min(d, r_lo + kRowsPerCta);
+  uint16_t* s_w = reinterpret_cast<uint16_t*>(s_raw);                                   // [kRowsPerCta][cols]
+  int32_t* s_idx = reinterpret_cast<int32_t*>(s_raw + static_cast<size_t>(kRowsPerCta) * J.cols * 2);  // [cols]
 
-  // penalty total of the job: block 0 / split 0 adds the per-block partials in a fixed order
-  if (b == 0 && blockIdx.y == 0 && J.penalty != nullptr) {
+  // penalty total of the job: its first CTA adds the per-block partials in a fixed order
+  if (b == 0 && blockIdx.y == 0 && J.penalty != nullptr && J.partial != nullptr) {
     double p = 0.0;
     for (int i = threadIdx.x; i < J.n_blocks; i += blockDim.x) p += J.partial[i];
     p = warp_sum(p);
@@ -110,7 +138,7 @@ fused_compact_plan_kernel(const __grid_constant__ Batch B) {
     __syncthreads();
     if (threadIdx.x == 0) {
       double tot = 0.0;
-      for (int w = 0; w < kThreads / 32; ++w) tot += s_red[w];
+      for (int w = 0; w < (blockDim.x >> 5); ++w) tot += s_red[w];
       *J.penalty = tot;
     }
   }
@@ -133,30 +161,29 @@ fused_compact_plan_kernel(const __grid_constant__ Batch B) {
     }
   }
 
-  const int rows_per = (d + gridDim.y - 1) / gridDim.y;
-  const int r_lo = blockIdx.y * rows_per;
-  const int r_hi = min(d, r_lo + rows_per);
   const uint16_t* wblk = J.W + static_cast<size_t>(b) * d * J.ldw;
   const uint8_t* flags = J.flags + static_cast<size_t>(b) * J.cols;
   const int chunks = J.cols >> 3;
 
-  // execution layout: W with the pruned columns of this row-block zeroed, 16 bytes at a time
-  if (J.plan != nullptr) {
-    for (int e = threadIdx.x; e < (r_hi - r_lo) * chunks; e += blockDim.x) {
-      const int r = r_lo + e / chunks, q = e % chunks;
+  // rows of this CTA: 16-byte loads, kept in shared memory; the execution layout is the same
+  // data with the pruned columns zeroed
+  for (int e = threadIdx.x; e < (r_hi - r_lo) * chunks; e += blockDim.x) {
+    const int rr = e / chunks, q = e - rr * chunks;
+    const uint4 w = __ldg(reinterpret_cast<const uint4*>(wblk + static_cast<size_t>(r_lo + rr) * J.ldw + (q << 3)));
+    *reinterpret_cast<uint4*>(s_w + static_cast<size_t>(rr) * J.cols + (q << 3)) = w;
+    if (J.plan != nullptr) {
       const uint2 f = *reinterpret_cast<const uint2*>(flags + (q << 3));
-      uint4 w = __ldg(reinterpret_cast<const uint4*>(wblk + static_cast<size_t>(r) * J.ldw + (q << 3)));
-      // a flag byte is 0 or 1: (flag * 0xffff) masks the matching 16-bit element
-      w.x &= ((f.x & 0xffu) * 0xffffu) | (((f.x >> 8) & 0xffu) * 0xffff0000u);
-      w.y &= (((f.x >> 16) & 0xffu) * 0xffffu) | (((f.x >> 24) & 0xffu) * 0xffff0000u);
-      w.z &= ((f.y & 0xffu) * 0xffffu) | (((f.y >> 8) & 0xffu) * 0xffff0000u);
-      w.w &= (((f.y >> 16) & 0xffu) * 0xffffu) | (((f.y >> 24) & 0xffu) * 0xffff0000u);
-      *reinterpret_cast<uint4*>(J.plan + (static_cast<size_t>(b) * d + r) * J.cols + (q << 3)) = w;
+      uint4 m;   // a flag byte is 0 or 1: flag * 0xffff masks the matching 16-bit element
+      m.x = w.x & (((f.x & 0xffu) * 0xffffu) | (((f.x >> 8) & 0xffu) * 0xffff0000u));
+      m.y = w.y & ((((f.x >> 16) & 0xffu) * 0xffffu) | (((f.x >> 24) & 0xffu) * 0xffff0000u));
+      m.z = w.z & (((f.y & 0xffu) * 0xffffu) | (((f.y >> 8) & 0xffu) * 0xffff0000u));
+      m.w = w.w & ((((f.y >> 16) & 0xffu) * 0xffffu) | (((f.y >> 24) & 0xffu) * 0xffff0000u));
+      *reinterpret_cast<uint4*>(J.plan + (static_cast<size_t>(b) * d + r_lo + rr) * J.cols + (q << 3)) = m;
     }
   }
   if (kc == 0) return;
 
-  // ascending list of kept columns
+  // ascending list of kept columns: each thread inspects 8 flags per round
   int running = 0;
   for (int q0 = 0; q0 < chunks; q0 += blockDim.x) {
     const int q = q0 + threadIdx.x;
@@ -172,25 +199,92 @@ fused_compact_plan_kernel(const __grid_constant__ Batch B) {
       if (bit) s_idx[p++] = (q << 3) + i;
     }
   }
-  __syncthreads();
+  __syncthreads();   // s_idx and s_w complete
   if (blockIdx.y == 0)
     for (int p = threadIdx.x; p < kc; p += blockDim.x) J.idx[base + p] = s_idx[p];
-  uint16_t* tile = J.vals + static_cast<size_t>(d) * base;
-  for (int p = threadIdx.x; p < kc; p += blockDim.x) {
-    const int col = s_idx[p];
-    int r = r_lo;
-    for (; r + 4 <= r_hi; r += 4) {
-      uint16_t v[4];
-#pragma unroll
-      for (int u = 0; u < 4; ++u) v[u] = __ldg(wblk + static_cast<size_t>(r + u) * J.ldw + col);
-#pragma unroll
-      for (int u = 0; u < 4; ++u) tile[static_cast<size_t>(r + u) * kc + p] = v[u];
+
+  // packed tile rows [r_lo, r_hi): a contiguous run of (r_hi - r_lo) * kc elements of vals
+  const long long tile0 = static_cast<long long>(d) * base;      // element offset of the block's tile
+  const long long e0 = tile0 + static_cast<long long>(r_lo) * kc, e1 = tile0 + static_cast<long long>(r_hi) * kc;
+  if ((reinterpret_cast<uintptr_t>(J.vals) & 15) == 0) {
+    for (long long v = (e0 >> 3) + threadIdx.x; v < ((e1 + 7) >> 3); v += blockDim.x) {
+      const long long first = v << 3;
+      long long e = first < e0 ? e0 : first;
+      const long long stop = first + 8 < e1 ? first + 8 : e1;
+      int rel = static_cast<int>(e - e0);
+      int rr = rel / kc, p = rel - rr * kc;
+      uint32_t out[4] = {0u, 0u, 0u, 0u};
+      for (; e < stop; ++e) {
+        const uint32_t val = s_w[static_cast<size_t>(rr) * J.cols + s_idx[p]];
+        const int slot = static_cast<int>(e - first);
+        out[slot >> 1] |= val << ((slot & 1) * 16);
+        if (++p == kc) { p = 0; ++rr; }
+      }
+      if (first >= e0 && first + 8 <= e1) {
+        *reinterpret_cast<uint4*>(J.vals + first) = make_uint4(out[0], out[1], out[2], out[3]);
+      } else {   // vector shared with a neighbouring CTA's rows: element stores for our part only
+        const long long lo = first < e0 ? e0 : first;
+        for (long long x = lo; x < stop; ++x) {
+          const int slot = static_cast<int>(x - first);
+          J.vals[x] = static_cast<uint16_t>(out[slot >> 1] >> ((slot & 1) * 16));
+        }
+      }
     }
-    for (; r < r_hi; ++r) tile[static_cast<size_t>(r) * kc + p] = __ldg(wblk + static_cast<size_t>(r) * J.ldw + col);
+  } else {
+    for (long long e = e0 + threadIdx.x; e < e1; e += blockDim.x) {
+      const int rel = static_cast<int>(e - e0);
+      const int rr = rel / kc, p = rel - rr * kc;
+      J.vals[e] = s_w[static_cast<size_t>(rr) * J.cols + s_idx[p]];
+    }
   }
 }
 
+template <typename Fill>
+int run_batches(const FusedJob* jobs, int n_jobs, int block, Fill launch) {
+  for (int j0 = 0; j0 < n_jobs; j0 += kFusedMaxJobs) {
+    Batch B;
+    B.n_jobs = n_jobs - j0 < kFusedMaxJobs ? n_jobs - j0 : kFusedMaxJobs;
+    B.block = block;
+    int total = 0, max_cols = 0;
+    for (int i = 0; i < B.n_jobs; ++i) {
+      B.job[i] = jobs[j0 + i];
+      B.first_block[i] = total;
+      total += jobs[j0 + i].n_blocks;
+      if (jobs[j0 + i].cols > max_cols) max_cols = jobs[j0 + i].cols;
+    }
+    B.first_block[B.n_jobs] = total;
+    int st = launch(B, total, max_cols);
+    if (st != BSP_OK) return st;
+  }
+  return BSP_OK;
+}
+
 }  // namespace
+
+int fused_stage1(const FusedJob* jobs, int n_jobs, int block, float eps, int squared, cudaStream_t s) {
+  return run_batches(jobs, n_jobs, block, [&](Batch& B, int total, int max_cols) -> int {
+    B.eps = eps;
+    B.squared = squared;
+    int threads = ((max_cols >> 3) + 31) / 32 * 32;
+    threads = threads > 256 ? 256 : threads;
+    fused_stage1_kernel<<<total, threads, 0, s>>>(B);
+    BSP_LAUNCH_CHECK();
+    return BSP_OK;
+  });
+}
+
+int fused_stage2(const FusedJob* jobs, int n_jobs, int block, cudaStream_t s) {
+  return run_batches(jobs, n_jobs, block, [&](Batch& B, int total, int max_cols) -> int {
+    B.eps = 0.0f;
+    B.squared = 0;
+    const int splits = (block + kRowsPerCta - 1) / kRowsPerCta;
+    const size_t smem = static_cast<size_t>(max_cols) * (kRowsPerCta * 2 + 4);
+    fused_stage2_kernel<<<dim3(total, splits), 256, smem, s>>>(B);
+    BSP_LAUNCH_CHECK();
+    return BSP_OK;
+  });
+}
+
 }  // namespace bsp
 
 extern "C" int bsp_prepare_batched(const bsp_layer_job* jobs, int n_jobs, int block, float eps, int pen,
@@ -199,6 +293,7 @@ extern "C" int bsp_prepare_batched(const bsp_layer_job* jobs, int n_jobs, int bl
   if (jobs == nullptr || n_jobs <= 0 || block <= 0) return BSP_ERR_ARG;
   if (pen != BSP_PEN_L2 && pen != BSP_PEN_L2SQ) return BSP_ERR_ARG;
   if (!(eps >= 0.0f)) return BSP_ERR_ARG;
+  if (n_jobs > 4096) return BSP_ERR_UNSUPPORTED;
   // validate everything before the first launch
   for (int i = 0; i < n_jobs; ++i) {
     const bsp_layer_job& u = jobs[i];
@@ -207,49 +302,32 @@ extern "C" int bsp_prepare_batched(const bsp_layer_job* jobs, int n_jobs, int bl
     if (u.blk_ptr == nullptr || u.idx == nullptr || u.vals == nullptr || u.ws == nullptr) return BSP_ERR_ARG;
     if (!aligned_to(u.ws, 256) || !aligned_to(u.blk_ptr, 4) || !aligned_to(u.idx, 4) || !aligned_to(u.vals, 2)) return BSP_ERR_ARG;
     if (u.threshold != u.threshold) return BSP_ERR_ARG;
-    const int nb = u.rows / block;
-    if (u.ws_bytes < ws_layout(nb, u.cols).total) return BSP_ERR_WORKSPACE;
+    if (u.ws_bytes < ws_layout(u.rows / block, u.cols).total) return BSP_ERR_WORKSPACE;
     if (u.plan != nullptr) {
       if (!aligned_to(u.plan, 256)) return BSP_ERR_ARG;
       if (u.plan_bytes < static_cast<size_t>(u.rows) * u.cols * 2) return BSP_ERR_WORKSPACE;
     }
-    const bool fast = u.cols % 8 == 0 && u.ldw % 8 == 0 && aligned_to(u.W, 16) && u.cols <= 12288 && nb <= 8192 &&
-                      (u.keep == nullptr || aligned_to(u.keep, 8)) &&
-                      (u.norms == nullptr || aligned_to(u.norms, 4)) && (u.gamma_out == nullptr || aligned_to(u.gamma_out, 4));
-    if (!fast) return BSP_ERR_UNSUPPORTED;
+    const bool ok = fused_shape_ok(u.W, u.rows, u.cols, u.ldw, block) && (u.keep == nullptr || aligned_to(u.keep, 8)) &&
+                    (u.norms == nullptr || aligned_to(u.norms, 16)) && (u.gamma_out == nullptr || aligned_to(u.gamma_out, 16)) &&
+                    (u.gamma_in == nullptr || aligned_to(u.gamma_in, 16));
+    if (!ok) return BSP_ERR_UNSUPPORTED;
+  }
+  FusedJob* fj = new (std::nothrow) FusedJob[n_jobs];
+  if (fj == nullptr) return BSP_ERR_ARG;
+  for (int i = 0; i < n_jobs; ++i) {
+    const bsp_layer_job& u = jobs[i];
+    const int nb = u.rows / block;
+    const WsLayout L = ws_layout(nb, u.cols);
+    char* wsb = static_cast<char*>(u.ws);
+    fj[i] = FusedJob{static_cast<const uint16_t*>(u.W), u.rows, u.cols, u.ldw, nb, u.threshold, u.threshold_dev,
+                     u.norms, u.gamma_in, u.gamma_out, u.penalty, reinterpret_cast<double*>(wsb + L.sumsq_off),
+                     u.keep ? u.keep : reinterpret_cast<uint8_t*>(wsb + L.keep_off),
+                     reinterpret_cast<int32_t*>(wsb + L.counts_off), u.blk_ptr, u.idx, static_cast<uint16_t*>(u.vals),
+                     u.kept_weights, static_cast<uint16_t*>(u.plan)};
   }
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  for (int j0 = 0; j0 < n_jobs; j0 += kMaxJobs) {
-    Batch B;
-    B.n_jobs = n_jobs - j0 < kMaxJobs ? n_jobs - j0 : kMaxJobs;
-    B.block = block;
-    int total_blocks = 0, max_cols = 0;
-    for (int i = 0; i < B.n_jobs; ++i) {
-      const bsp_layer_job& u = jobs[j0 + i];
-      Job& J = B.job[i];
-      const int nb = u.rows / block;
-      const WsLayout L = ws_layout(nb, u.cols);
-      char* wsb = static_cast<char*>(u.ws);
-      J.W = static_cast<const uint16_t*>(u.W);
-      J.rows = u.rows; J.cols = u.cols; J.ldw = u.ldw; J.n_blocks = nb;
-      J.threshold = u.threshold; J.threshold_dev = u.threshold_dev;
-      J.out = NormOut{u.norms, u.gamma_in, u.gamma_out, nullptr, eps, pen == BSP_PEN_L2SQ ? 1 : 0};
-      J.penalty = u.penalty;
-      J.flags = u.keep ? u.keep : reinterpret_cast<uint8_t*>(wsb + L.keep_off);
-      J.counts = reinterpret_cast<int32_t*>(wsb + L.counts_off);
-      J.partial = reinterpret_cast<double*>(wsb + L.sumsq_off);
-      J.blk_ptr = u.blk_ptr; J.idx = u.idx; J.vals = static_cast<uint16_t*>(u.vals);
-      J.kept_weights = u.kept_weights; J.plan = static_cast<uint16_t*>(u.plan);
-      B.first_block[i] = total_blocks;
-      total_blocks += nb;
-      if (u.cols > max_cols) max_cols = u.cols;
-    }
-    B.first_block[B.n_jobs] = total_blocks;
-    fused_norms_flags_kernel<<<total_blocks, kThreads, 0, s>>>(B);
-    BSP_LAUNCH_CHECK();
-    const int splits = block >= 4 ? 4 : 1;
-    fused_compact_plan_kernel<<<dim3(total_blocks, splits), kThreads, sizeof(int32_t) * max_cols, s>>>(B);
-    BSP_LAUNCH_CHECK();
-  }
-  return BSP_OK;
+  int st = fused_stage1(fj, n_jobs, block, eps, pen == BSP_PEN_L2SQ ? 1 : 0, s);
+  if (st == BSP_OK) st = fused_stage2(fj, n_jobs, block, s);
+  delete[] fj;
+  return st;
 }

@@ -1,6 +1,8 @@
 // bsp_group_norms: per-group l2 norms, the gamma update and the reweighted group-Lasso penalty
 // (Section 3.2, Eq. 2 and Eq. 3) in a single pass over W.  Bandwidth-bound: every weight is
-// read once, one float is written per group and per requested output.
+// read once, one float is written per group and per requested output.  Orientation C with
+// 8-element alignment runs the vectorised stage-1 kernel of bsp_fused.cu; this file holds the
+// generic kernel (any alignment, orientation R) and the entry point.
 #include "bsp_common.cuh"
 
 namespace bsp {
@@ -16,58 +18,6 @@ __device__ __forceinline__ void add_penalty(const NormOut& o, double local) {
   if (o.penalty == nullptr) return;  // uniform across the grid
   local = warp_sum(local);
   if ((threadIdx.x & 31) == 0 && local != 0.0) atomicAdd(o.penalty, local);
-}
-
-// Orientation C fast path: one thread owns 8 adjacent columns of one row-block and walks its d
-// rows with 16-byte loads (a warp covers 512 contiguous bytes of every row).  The eight sums
-// are independent sequential chains, so each equals the defined float32 decision quantity.
-template <int UNROLL>
-__global__ void __launch_bounds__(256)
-norms_c_vec8_kernel(const uint16_t* __restrict__ W, int n_blocks, int cols, int ldw, int d, NormOut o) {
-  const int chunks = cols >> 3;
-  const long long item = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
-  double local = 0.0;
-  if (item < static_cast<long long>(n_blocks) * chunks) {
-    const int b = static_cast<int>(item / chunks);
-    const int q = static_cast<int>(item - static_cast<long long>(b) * chunks);
-    const uint16_t* p = W + static_cast<size_t>(b) * d * ldw + (q << 3);
-    float acc[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) acc[i] = 0.0f;
-    int r = 0;
-    for (; r + UNROLL <= d; r += UNROLL) {
-      uint4 v[UNROLL];
-#pragma unroll
-      for (int u = 0; u < UNROLL; ++u)
-        v[u] = __ldg(reinterpret_cast<const uint4*>(p + static_cast<size_t>(r + u) * ldw));
-#pragma unroll
-      for (int u = 0; u < UNROLL; ++u) {
-        const uint32_t w32[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const float lo = __uint_as_float(w32[i] << 16);
-          const float hi = __uint_as_float(w32[i] & 0xffff0000u);
-          acc[2 * i] = __fmaf_rn(lo, lo, acc[2 * i]);
-          acc[2 * i + 1] = __fmaf_rn(hi, hi, acc[2 * i + 1]);
-        }
-      }
-    }
-    for (; r < d; ++r) {
-      const uint4 v = __ldg(reinterpret_cast<const uint4*>(p + static_cast<size_t>(r) * ldw));
-      const uint32_t w32[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const float lo = __uint_as_float(w32[i] << 16);
-        const float hi = __uint_as_float(w32[i] & 0xffff0000u);
-        acc[2 * i] = __fmaf_rn(lo, lo, acc[2 * i]);
-        acc[2 * i + 1] = __fmaf_rn(hi, hi, acc[2 * i + 1]);
-      }
-    }
-    const size_t g0 = static_cast<size_t>(b) * cols + (q << 3);
-#pragma unroll
-    for (int i = 0; i < 8; ++i) local += finish_group(o, g0 + i, acc[i]);
-  }
-  add_penalty(o, local);
 }
 
 // Any geometry: one thread per group.  C: lanes run along columns (each row is read
@@ -129,14 +79,14 @@ extern "C" int bsp_group_norms(const void* W, int rows, int cols, int ldw, int b
 
   NormOut o{norms, gamma_in, gamma_out, penalty, eps, pen == BSP_PEN_L2SQ ? 1 : 0};
   const uint16_t* w = static_cast<const uint16_t*>(W);
-  const bool vec_ok = orient == BSP_ORIENT_C && (cols % 8 == 0) && (ldw % 8 == 0) && aligned_to(W, 16);
+  const bool vec_ok = orient == BSP_ORIENT_C && cols % 8 == 0 && ldw % 8 == 0 && aligned_to(W, 16) &&   // stage 1 alone has no size limit
+                      (norms == nullptr || aligned_to(norms, 16)) && (gamma_out == nullptr || aligned_to(gamma_out, 16)) &&
+                      (gamma_in == nullptr || aligned_to(gamma_in, 16));
   if (vec_ok) {
-    const long long items = static_cast<long long>(rows / block) * (cols / 8);
-    const unsigned grid = static_cast<unsigned>((items + 255) / 256);
-    if (block % 8 == 0)
-      norms_c_vec8_kernel<8><<<grid, 256, 0, s>>>(w, rows / block, cols, ldw, block, o);
-    else
-      norms_c_vec8_kernel<4><<<grid, 256, 0, s>>>(w, rows / block, cols, ldw, block, o);
+    // vectorised stage 1 with the keep decision switched off; the penalty is added by atomics
+    FusedJob j{w, rows, cols, ldw, rows / block, 0.0f, nullptr, norms, gamma_in, gamma_out, penalty,
+               nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
+    return fused_stage1(&j, 1, block, eps, o.squared, s);
   } else {
     int nb, ng;
     geometry(rows, cols, block, orient, &nb, &ng);

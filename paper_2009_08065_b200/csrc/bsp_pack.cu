@@ -5,9 +5,10 @@
 // Launches per pack: (1) one CTA per block decides its groups and counts the kept ones,
 // (2) CTAs per block turn the counts before theirs into blk_ptr, list the kept indices in
 // ascending order and gather the dense tile of kept values.  W is read from HBM once by (1);
-// (2) re-reads it from L2.  Orientation C with 8-element alignment runs vectorised kernels
-// (16-byte loads, one thread per 8 columns); everything else runs the generic kernels, which
-// insert a single-CTA scan between (1) and (2).
+// (2) re-reads it from L2.  Orientation C with 8-element alignment runs the vectorised
+// two-stage kernels of bsp_fused.cu; this file holds the generic kernels (any alignment,
+// orientation R, with a single-CTA scan between (1) and (2)), the keep-count and percentile
+// kernels, and the entry points.
 #include "bsp_common.cuh"
 
 namespace bsp {
@@ -141,111 +142,6 @@ compact_kernel(const uint16_t* __restrict__ W, Geometry G, const uint8_t* __rest
 }
 
 
-// ------------------------------------------------------------------------------------------
-// Orientation C fast path (cols, ldw multiples of 8; W 16-byte aligned; keep 8-byte aligned)
-// ------------------------------------------------------------------------------------------
-
-// (1) threshold mode, vectorised: one thread per 8 columns of one row-block.
-__global__ void __launch_bounds__(kPackThreads)
-flags_c_vec8_kernel(const uint16_t* __restrict__ W, Geometry G, float threshold,
-                    const float* __restrict__ threshold_dev, uint8_t* __restrict__ keep,
-                    int32_t* __restrict__ counts) {
-  __shared__ int s_count;
-  if (threadIdx.x == 0) s_count = 0;
-  __syncthreads();
-  const float t = threshold_dev ? *threshold_dev : threshold;
-  const bool keep_all = t < 0.0f;
-  const float t2 = __fmul_rn(t, t);
-  const int b = blockIdx.x;
-  int local = 0;
-  for (int q = threadIdx.x; q < (G.cols >> 3); q += blockDim.x) {
-    float acc[8];
-    sumsq8(W + static_cast<size_t>(b) * G.block * G.ldw + (q << 3), G.block, G.ldw, acc);
-    uint32_t lo = 0, hi = 0;
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const uint32_t k0 = (keep_all || acc[i] > t2) ? 1u : 0u;
-      const uint32_t k1 = (keep_all || acc[4 + i] > t2) ? 1u : 0u;
-      lo |= k0 << (8 * i);
-      hi |= k1 << (8 * i);
-      local += static_cast<int>(k0 + k1);
-    }
-    *reinterpret_cast<uint2*>(keep + static_cast<size_t>(b) * G.cols + (q << 3)) = make_uint2(lo, hi);
-  }
-  local = warp_sum(local);
-  if ((threadIdx.x & 31) == 0 && local) atomicAdd(&s_count, local);
-  __syncthreads();
-  if (threadIdx.x == 0) counts[b] = s_count;
-}
-
-// (2) vectorised compaction.  grid = (row-blocks, row splits).  Every CTA sums the counts of the
-// blocks before its own (at most a few thousand values), rebuilds the block's ascending index
-// list in shared memory from the keep flags, and gathers its share of the block's rows.
-__global__ void __launch_bounds__(kPackThreads)
-compact_c_kernel(const uint16_t* __restrict__ W, Geometry G, const uint8_t* __restrict__ keep,
-                 const int32_t* __restrict__ counts, int32_t* __restrict__ blk_ptr,
-                 int32_t* __restrict__ idx, uint16_t* __restrict__ vals, int64_t* __restrict__ kept_weights) {
-  extern __shared__ int32_t s_idx[];   // kept column indices of this block, ascending
-  __shared__ int s_warp[32];
-  __shared__ int s_base;
-  const int b = blockIdx.x;
-  // blk_ptr[b] = sum of counts[0..b)
-  int part = 0;
-  for (int i = threadIdx.x; i < b; i += blockDim.x) part += counts[i];
-  part = warp_sum(part);
-  if (threadIdx.x == 0) s_base = 0;
-  __syncthreads();
-  if ((threadIdx.x & 31) == 0 && part) atomicAdd(&s_base, part);
-  __syncthreads();
-  const int base = s_base;
-  const int kc = counts[b];
-  if (blockIdx.y == 0 && threadIdx.x == 0) {
-    blk_ptr[b] = base;
-    if (b == G.n_blocks - 1) {
-      blk_ptr[G.n_blocks] = base + kc;
-      if (kept_weights) *kept_weights = static_cast<int64_t>(base + kc) * G.block;
-    }
-  }
-  if (kc == 0) return;
-  // ascending list of kept columns: each thread inspects 8 flags per round
-  int running = 0;
-  for (int q0 = 0; q0 < (G.cols >> 3); q0 += blockDim.x) {
-    const int q = q0 + threadIdx.x;
-    uint2 f = make_uint2(0u, 0u);
-    if (q < (G.cols >> 3)) f = *reinterpret_cast<const uint2*>(keep + static_cast<size_t>(b) * G.cols + (q << 3));
-    const int mine = __popc(f.x) + __popc(f.y);          // flags are 0 or 1 per byte
-    int total;
-    int p = running + block_exclusive_scan(mine, s_warp, &total);
-    running += total;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const uint32_t bit = ((i < 4 ? f.x : f.y) >> (8 * (i & 3))) & 1u;
-      if (bit) s_idx[p++] = (q << 3) + i;
-    }
-  }
-  __syncthreads();
-  if (blockIdx.y == 0)
-    for (int p = threadIdx.x; p < kc; p += blockDim.x) idx[base + p] = s_idx[p];
-  // rows of this CTA's share: tile[r, p] = W[b*d + r, s_idx[p]]
-  const int rows_per = (G.block + gridDim.y - 1) / gridDim.y;
-  const int r_lo = blockIdx.y * rows_per;
-  const int r_hi = min(G.block, r_lo + rows_per);
-  uint16_t* tile = vals + static_cast<size_t>(G.block) * base;
-  const uint16_t* wblk = W + static_cast<size_t>(b) * G.block * G.ldw;
-  for (int p = threadIdx.x; p < kc; p += blockDim.x) {
-    const int col = s_idx[p];
-    int r = r_lo;
-    for (; r + 4 <= r_hi; r += 4) {
-      uint16_t v[4];
-#pragma unroll
-      for (int u = 0; u < 4; ++u) v[u] = __ldg(wblk + static_cast<size_t>(r + u) * G.ldw + col);
-#pragma unroll
-      for (int u = 0; u < 4; ++u) tile[static_cast<size_t>(r + u) * kc + p] = v[u];
-    }
-    for (; r < r_hi; ++r) tile[static_cast<size_t>(r) * kc + p] = __ldg(wblk + static_cast<size_t>(r) * G.ldw + col);
-  }
-}
-
 // Float32 sums of squares of all groups, flattened in per-group-array order.
 __global__ void __launch_bounds__(kPackThreads)
 sumsq_kernel(const uint16_t* __restrict__ W, Geometry G, float* __restrict__ S) {
@@ -353,25 +249,29 @@ extern "C" int bsp_prune_pack(const void* W, int rows, int cols, int ldw, int bl
   uint8_t* flags = keep ? keep : reinterpret_cast<uint8_t*>(wsb + L.keep_off);
   const uint16_t* w = static_cast<const uint16_t*>(W);
 
-  const bool fast = orient == BSP_ORIENT_C && cols % 8 == 0 && ldw % 8 == 0 && aligned_to(W, 16) &&
-                    aligned_to(flags, 8) && cols <= 12288 && G.n_blocks <= 8192;
+  const bool fast = orient == BSP_ORIENT_C && fused_shape_ok(W, rows, cols, ldw, block) && aligned_to(flags, 8);
+  if (fast) {
+    // vectorised kernels of bsp_fused.cu: stage 1 for the flags (unless the keep-count kernel makes them), stage 2
+    FusedJob j{w, rows, cols, ldw, G.n_blocks, threshold, threshold_dev, nullptr, nullptr, nullptr, nullptr, nullptr,
+               flags, counts, blk_ptr, idx, static_cast<uint16_t*>(vals), kept_weights, nullptr};
+    if (keep_per_block >= 0) {
+      flags_topk_kernel<<<G.n_blocks, kPackThreads, sizeof(float) * G.n_groups, s>>>(w, G, keep_per_block, flags, counts);
+      BSP_LAUNCH_CHECK();
+    } else {
+      st = fused_stage1(&j, 1, block, 0.0f, 0, s);
+      if (st != BSP_OK) return st;
+    }
+    return fused_stage2(&j, 1, block, s);
+  }
   if (keep_per_block >= 0) {
     flags_topk_kernel<<<G.n_blocks, kPackThreads, sizeof(float) * G.n_groups, s>>>(w, G, keep_per_block, flags, counts);
-  } else if (fast) {
-    flags_c_vec8_kernel<<<G.n_blocks, kPackThreads, 0, s>>>(w, G, threshold, threshold_dev, flags, counts);
   } else {
     flags_threshold_kernel<<<G.n_blocks, kPackThreads, 0, s>>>(w, G, threshold, threshold_dev, flags, counts);
   }
   BSP_LAUNCH_CHECK();
-  if (fast) {
-    const int splits = block >= 4 ? 4 : 1;
-    compact_c_kernel<<<dim3(G.n_blocks, splits), kPackThreads, sizeof(int32_t) * cols, s>>>(
-        w, G, flags, counts, blk_ptr, idx, static_cast<uint16_t*>(vals), kept_weights);
-  } else {
-    scan_counts_kernel<<<1, 1024, 0, s>>>(counts, G.n_blocks, block, blk_ptr, kept_weights);
-    BSP_LAUNCH_CHECK();
-    compact_kernel<<<G.n_blocks, kPackThreads, 0, s>>>(w, G, flags, blk_ptr, idx, static_cast<uint16_t*>(vals));
-  }
+  scan_counts_kernel<<<1, 1024, 0, s>>>(counts, G.n_blocks, block, blk_ptr, kept_weights);
+  BSP_LAUNCH_CHECK();
+  compact_kernel<<<G.n_blocks, kPackThreads, 0, s>>>(w, G, flags, blk_ptr, idx, static_cast<uint16_t*>(vals));
   BSP_LAUNCH_CHECK();
   return BSP_OK;
 }
