@@ -138,28 +138,14 @@ __device__ __forceinline__ int warp_sum(int v) {
 
 // Float32 sums of squares of 8 adjacent columns over the d rows of a row-block: eight independent
 // sequential chains, each the defined decision quantity of its group.
-__device__ __forceinline__ void sumsq8(const uint16_t* __restrict__ p, int d, int ldw, float (&acc)[8]) {
+template <int ROWS>
+__device__ __forceinline__ void sumsq8_rows(const uint16_t* __restrict__ p, int ldw, float (&acc)[8]) {
+  uint4 v[ROWS];
 #pragma unroll
-  for (int i = 0; i < 8; ++i) acc[i] = 0.0f;
-  int r = 0;
-  for (; r + 8 <= d; r += 8) {
-    uint4 v[8];
+  for (int u = 0; u < ROWS; ++u) v[u] = __ldg(reinterpret_cast<const uint4*>(p + static_cast<size_t>(u) * ldw));
 #pragma unroll
-    for (int u = 0; u < 8; ++u) v[u] = __ldg(reinterpret_cast<const uint4*>(p + static_cast<size_t>(r + u) * ldw));
-#pragma unroll
-    for (int u = 0; u < 8; ++u) {
-      const uint32_t w32[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const float lo = __uint_as_float(w32[i] << 16), hi = __uint_as_float(w32[i] & 0xffff0000u);
-        acc[2 * i] = __fmaf_rn(lo, lo, acc[2 * i]);
-        acc[2 * i + 1] = __fmaf_rn(hi, hi, acc[2 * i + 1]);
-      }
-    }
-  }
-  for (; r < d; ++r) {
-    const uint4 v = __ldg(reinterpret_cast<const uint4*>(p + static_cast<size_t>(r) * ldw));
-    const uint32_t w32[4] = {v.x, v.y, v.z, v.w};
+  for (int u = 0; u < ROWS; ++u) {     // rows in increasing order: the chains stay sequential
+    const uint32_t w32[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const float lo = __uint_as_float(w32[i] << 16), hi = __uint_as_float(w32[i] & 0xffff0000u);
@@ -167,6 +153,14 @@ __device__ __forceinline__ void sumsq8(const uint16_t* __restrict__ p, int d, in
       acc[2 * i + 1] = __fmaf_rn(hi, hi, acc[2 * i + 1]);
     }
   }
+}
+__device__ __forceinline__ void sumsq8(const uint16_t* __restrict__ p, int d, int ldw, float (&acc)[8]) {
+#pragma unroll
+  for (int i = 0; i < 8; ++i) acc[i] = 0.0f;
+  int r = 0;
+  for (; r + 16 <= d; r += 16) sumsq8_rows<16>(p + static_cast<size_t>(r) * ldw, ldw, acc);   // 256 bytes in flight
+  for (; r + 4 <= d; r += 4) sumsq8_rows<4>(p + static_cast<size_t>(r) * ldw, ldw, acc);
+  for (; r < d; ++r) sumsq8_rows<1>(p + static_cast<size_t>(r) * ldw, ldw, acc);
 }
 
 // Block-wide exclusive prefix sum of one int per thread (blockDim.x a multiple of 32, <= 1024).

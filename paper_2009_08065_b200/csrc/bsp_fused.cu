@@ -4,10 +4,11 @@
 //            block's rows (8 rows in flight), eight independent sequential float32 sums of
 //            squares (the defined decision quantity), then any of: norms / gamma (two 16-byte
 //            stores each), penalty partial, keep flags (one 8-byte store) and the block's count.
-//   stage 2  grid (row-blocks, groups of 4 rows): blk_ptr from the counts before the block, the
-//            ascending index list from the flags, the rows staged once in shared memory (16-byte
-//            loads) and from there (a) the zero-expanded execution layout, (b) the packed tile,
-//            written as 16-byte vectors wherever the output is 16-byte aligned.
+//   stage 2  grid (row-blocks, row ranges of about 16K weights): blk_ptr from the counts before
+//            the block, the ascending index list from the flags, then 4 rows at a time staged in
+//            shared memory (16-byte loads) and from there (a) the zero-expanded execution
+//            layout, (b) the packed tile, written as 16-byte vectors wherever the output is
+//            16-byte aligned.
 #include <new>
 
 #include "bsp_common.cuh"
@@ -15,7 +16,7 @@
 namespace bsp {
 namespace {
 
-constexpr int kRowsPerCta = 4;
+constexpr int kRowsPerPass = 4;   // rows staged in shared memory at a time
 
 struct Batch {
   int n_jobs, block, squared;
@@ -113,6 +114,22 @@ fused_stage1_kernel(const __grid_constant__ Batch B) {
   }
 }
 
+// Rows staged in shared memory at a time: up to 24 KB (the whole block for narrow matrices).
+__host__ __device__ inline int rows_per_pass(int cols) {
+  int r = 12288 / cols;
+  r = r < 4 ? 4 : r;
+  return r > 16 ? 16 : r;
+}
+
+// Rows of a row-block that one stage-2 CTA handles: about 16K weights per CTA, a multiple of the
+// 4-row staging pass, so that narrow matrices build their index list once per block and wide ones
+// still spread over several CTAs.
+__host__ __device__ inline int rows_per_cta(int cols, int d) {
+  int r = (16384 / cols) / kRowsPerPass * kRowsPerPass;
+  if (r < kRowsPerPass) r = kRowsPerPass;
+  return r > d ? d : r;
+}
+
 __global__ void __launch_bounds__(256)
 fused_stage2_kernel(const __grid_constant__ Batch B) {
   extern __shared__ __align__(16) uint8_t s_raw[];
@@ -123,11 +140,12 @@ fused_stage2_kernel(const __grid_constant__ Batch B) {
   const FusedJob& J = B.job[j];
   const int b = blockIdx.x - B.first_block[j];
   const int d = B.block;
-  const int r_lo = blockIdx.y * kRowsPerCta;
-  if (r_lo >= d) return;
-  const int r_hi = min(d, r_lo + kRowsPerCta);
-  uint16_t* s_w = reinterpret_cast<uint16_t*>(s_raw);                                   // [kRowsPerCta][cols]
-  int32_t* s_idx = reinterpret_cast<int32_t*>(s_raw + static_cast<size_t>(kRowsPerCta) * J.cols * 2);  // [cols]
+  const int per_cta = rows_per_cta(J.cols, d);
+  const int r_begin = blockIdx.y * per_cta;
+  if (r_begin >= d) return;
+  const int r_end = min(d, r_begin + per_cta);
+  uint16_t* s_w = reinterpret_cast<uint16_t*>(s_raw);                                    // [rows_per_pass][cols]
+  int32_t* s_idx = reinterpret_cast<int32_t*>(s_raw + static_cast<size_t>(rows_per_pass(J.cols)) * J.cols * 2);  // [cols]
 
   // penalty total of the job: its first CTA adds the per-block partials in a fixed order
   if (b == 0 && blockIdx.y == 0 && J.penalty != nullptr && J.partial != nullptr) {
@@ -165,77 +183,96 @@ fused_stage2_kernel(const __grid_constant__ Batch B) {
   const uint8_t* flags = J.flags + static_cast<size_t>(b) * J.cols;
   const int chunks = J.cols >> 3;
 
-  // rows of this CTA: 16-byte loads, kept in shared memory; the execution layout is the same
-  // data with the pruned columns zeroed
-  for (int e = threadIdx.x; e < (r_hi - r_lo) * chunks; e += blockDim.x) {
-    const int rr = e / chunks, q = e - rr * chunks;
-    const uint4 w = __ldg(reinterpret_cast<const uint4*>(wblk + static_cast<size_t>(r_lo + rr) * J.ldw + (q << 3)));
-    *reinterpret_cast<uint4*>(s_w + static_cast<size_t>(rr) * J.cols + (q << 3)) = w;
-    if (J.plan != nullptr) {
-      const uint2 f = *reinterpret_cast<const uint2*>(flags + (q << 3));
-      uint4 m;   // a flag byte is 0 or 1: flag * 0xffff masks the matching 16-bit element
-      m.x = w.x & (((f.x & 0xffu) * 0xffffu) | (((f.x >> 8) & 0xffu) * 0xffff0000u));
-      m.y = w.y & ((((f.x >> 16) & 0xffu) * 0xffffu) | (((f.x >> 24) & 0xffu) * 0xffff0000u));
-      m.z = w.z & (((f.y & 0xffu) * 0xffffu) | (((f.y >> 8) & 0xffu) * 0xffff0000u));
-      m.w = w.w & ((((f.y >> 16) & 0xffu) * 0xffffu) | (((f.y >> 24) & 0xffu) * 0xffff0000u));
-      *reinterpret_cast<uint4*>(J.plan + (static_cast<size_t>(b) * d + r_lo + rr) * J.cols + (q << 3)) = m;
-    }
-  }
-  if (kc == 0) return;
-
   // ascending list of kept columns: each thread inspects 8 flags per round
-  int running = 0;
-  for (int q0 = 0; q0 < chunks; q0 += blockDim.x) {
-    const int q = q0 + threadIdx.x;
-    uint2 f = make_uint2(0u, 0u);
-    if (q < chunks) f = *reinterpret_cast<const uint2*>(flags + (q << 3));
-    const int mine = __popc(f.x) + __popc(f.y);
-    int total;
-    int p = running + block_exclusive_scan(mine, s_warp, &total);
-    running += total;
+  if (kc > 0) {
+    int running = 0;
+    for (int q0 = 0; q0 < chunks; q0 += blockDim.x) {
+      const int q = q0 + threadIdx.x;
+      uint2 f = make_uint2(0u, 0u);
+      if (q < chunks) f = *reinterpret_cast<const uint2*>(flags + (q << 3));
+      const int mine = __popc(f.x) + __popc(f.y);
+      int total;
+      int p = running + block_exclusive_scan(mine, s_warp, &total);
+      running += total;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const uint32_t bit = ((i < 4 ? f.x : f.y) >> (8 * (i & 3))) & 1u;
-      if (bit) s_idx[p++] = (q << 3) + i;
-    }
-  }
-  __syncthreads();   // s_idx and s_w complete
-  if (blockIdx.y == 0)
-    for (int p = threadIdx.x; p < kc; p += blockDim.x) J.idx[base + p] = s_idx[p];
-
-  // packed tile rows [r_lo, r_hi): a contiguous run of (r_hi - r_lo) * kc elements of vals
-  const long long tile0 = static_cast<long long>(d) * base;      // element offset of the block's tile
-  const long long e0 = tile0 + static_cast<long long>(r_lo) * kc, e1 = tile0 + static_cast<long long>(r_hi) * kc;
-  if ((reinterpret_cast<uintptr_t>(J.vals) & 15) == 0) {
-    for (long long v = (e0 >> 3) + threadIdx.x; v < ((e1 + 7) >> 3); v += blockDim.x) {
-      const long long first = v << 3;
-      long long e = first < e0 ? e0 : first;
-      const long long stop = first + 8 < e1 ? first + 8 : e1;
-      int rel = static_cast<int>(e - e0);
-      int rr = rel / kc, p = rel - rr * kc;
-      uint32_t out[4] = {0u, 0u, 0u, 0u};
-      for (; e < stop; ++e) {
-        const uint32_t val = s_w[static_cast<size_t>(rr) * J.cols + s_idx[p]];
-        const int slot = static_cast<int>(e - first);
-        out[slot >> 1] |= val << ((slot & 1) * 16);
-        if (++p == kc) { p = 0; ++rr; }
+      for (int i = 0; i < 8; ++i) {
+        const uint32_t bit = ((i < 4 ? f.x : f.y) >> (8 * (i & 3))) & 1u;
+        if (bit) s_idx[p++] = (q << 3) + i;
       }
-      if (first >= e0 && first + 8 <= e1) {
-        *reinterpret_cast<uint4*>(J.vals + first) = make_uint4(out[0], out[1], out[2], out[3]);
-      } else {   // vector shared with a neighbouring CTA's rows: element stores for our part only
-        const long long lo = first < e0 ? e0 : first;
-        for (long long x = lo; x < stop; ++x) {
-          const int slot = static_cast<int>(x - first);
-          J.vals[x] = static_cast<uint16_t>(out[slot >> 1] >> ((slot & 1) * 16));
+    }
+    __syncthreads();
+    if (blockIdx.y == 0)
+      for (int p = threadIdx.x; p < kc; p += blockDim.x) J.idx[base + p] = s_idx[p];
+  }
+  if (kc == 0 && J.plan == nullptr) return;
+
+  const bool vec_ok = (reinterpret_cast<uintptr_t>(J.vals) & 15) == 0;
+  const long long tile0 = static_cast<long long>(d) * base;      // element offset of the block's tile in vals
+  const int pass_rows = rows_per_pass(J.cols);
+  for (int r_lo = r_begin; r_lo < r_end; r_lo += pass_rows) {
+    const int n_rows = min(pass_rows, r_end - r_lo);
+    // this pass's rows, one warp per row (rows warp, warp + n_warps, ...), lanes along the row:
+    // 16-byte loads kept in shared memory; the execution layout is the same data with the pruned
+    // columns zeroed.  No index arithmetic beyond adds, so the loop stays load-bound.
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, n_warps = blockDim.x >> 5;
+    for (int rr = warp; rr < n_rows; rr += n_warps) {
+      const uint16_t* src = wblk + static_cast<size_t>(r_lo + rr) * J.ldw;
+      uint16_t* dst = s_w + rr * J.cols;
+      uint16_t* pdst = J.plan ? J.plan + (static_cast<size_t>(b) * d + r_lo + rr) * J.cols : nullptr;
+      for (int q0 = lane; q0 < chunks; q0 += 128) {
+        uint4 w[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+          if (q0 + 32 * u < chunks) w[u] = __ldg(reinterpret_cast<const uint4*>(src + ((q0 + 32 * u) << 3)));
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int q = q0 + 32 * u;
+          if (q >= chunks) break;
+          *reinterpret_cast<uint4*>(dst + (q << 3)) = w[u];
+          if (pdst != nullptr) {
+            const uint2 f = *reinterpret_cast<const uint2*>(flags + (q << 3));
+            uint4 m;   // a flag byte is 0 or 1: flag * 0xffff masks the matching 16-bit element
+            m.x = w[u].x & (((f.x & 0xffu) * 0xffffu) | (((f.x >> 8) & 0xffu) * 0xffff0000u));
+            m.y = w[u].y & ((((f.x >> 16) & 0xffu) * 0xffffu) | (((f.x >> 24) & 0xffu) * 0xffff0000u));
+            m.z = w[u].z & (((f.y & 0xffu) * 0xffffu) | (((f.y >> 8) & 0xffu) * 0xffff0000u));
+            m.w = w[u].w & ((((f.y >> 16) & 0xffu) * 0xffffu) | (((f.y >> 24) & 0xffu) * 0xffff0000u));
+            *reinterpret_cast<uint4*>(pdst + (q << 3)) = m;
+          }
         }
       }
     }
-  } else {
-    for (long long e = e0 + threadIdx.x; e < e1; e += blockDim.x) {
-      const int rel = static_cast<int>(e - e0);
-      const int rr = rel / kc, p = rel - rr * kc;
-      J.vals[e] = s_w[static_cast<size_t>(rr) * J.cols + s_idx[p]];
+    __syncthreads();   // s_w (and, on the first pass, s_idx) complete
+    // packed tile rows of this pass, again one warp per row: row r occupies
+    // vals[tile0 + r*kc, tile0 + (r+1)*kc); whole 16-byte vectors in the middle, ragged ends by element
+    if (kc > 0) {
+      for (int rr = warp; rr < n_rows; rr += n_warps) {
+        const uint16_t* srow = s_w + rr * J.cols;
+        const long long e0 = tile0 + static_cast<long long>(r_lo + rr) * kc;
+        uint16_t* out_row = J.vals + e0;                               // element p of the row goes to out_row[p]
+        if (vec_ok) {
+          const int head = static_cast<int>((8 - (e0 & 7)) & 7);       // elements before the first aligned vector
+          const int n_vec = kc > head ? (kc - head) >> 3 : 0;
+          for (int v = lane; v < n_vec; v += 32) {
+            const int p = head + (v << 3);
+            uint32_t o[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+              o[i] = static_cast<uint32_t>(srow[s_idx[p + 2 * i]]) | (static_cast<uint32_t>(srow[s_idx[p + 2 * i + 1]]) << 16);
+            *reinterpret_cast<uint4*>(out_row + p) = make_uint4(o[0], o[1], o[2], o[3]);
+          }
+          const int tail0 = head + (n_vec << 3);
+          if (lane < 8) {
+            if (lane < head && lane < kc) out_row[lane] = srow[s_idx[lane]];
+          } else if (lane < 16) {
+            const int p = tail0 + (lane - 8);
+            if (p >= head && p < kc) out_row[p] = srow[s_idx[p]];
+          }
+        } else {
+          for (int p = lane; p < kc; p += 32) out_row[p] = srow[s_idx[p]];
+        }
+      }
     }
+    __syncthreads();   // s_w is overwritten by the next pass
   }
 }
 
@@ -277,8 +314,17 @@ int fused_stage2(const FusedJob* jobs, int n_jobs, int block, cudaStream_t s) {
   return run_batches(jobs, n_jobs, block, [&](Batch& B, int total, int max_cols) -> int {
     B.eps = 0.0f;
     B.squared = 0;
-    const int splits = (block + kRowsPerCta - 1) / kRowsPerCta;
-    const size_t smem = static_cast<size_t>(max_cols) * (kRowsPerCta * 2 + 4);
+    int splits = 1;
+    for (int i = 0; i < B.n_jobs; ++i) {
+      const int per = rows_per_cta(B.job[i].cols, block);
+      const int need = (block + per - 1) / per;
+      if (need > splits) splits = need;
+    }
+    size_t smem = 0;
+    for (int i = 0; i < B.n_jobs; ++i) {
+      const size_t need = static_cast<size_t>(B.job[i].cols) * (rows_per_pass(B.job[i].cols) * 2 + 4);
+      if (need > smem) smem = need;
+    }
     fused_stage2_kernel<<<dim3(total, splits), 256, smem, s>>>(B);
     BSP_LAUNCH_CHECK();
     return BSP_OK;
