@@ -122,7 +122,7 @@ class LayerOnDevice:
         import paper_2009_08065_b200 as bsp
         self.torch, self.bsp, self.wl, self.device = torch, bsp, wl, device
         self.host = {}          # pinned host copies of the inputs, for the end-to-end leg
-        x = si.make_activations(seed + 1000 * rank, "layer_in", wl.tokens, wl.linears[0].k_in)
+        x = si.make_activations(rank_seed(seed, rank), "layer_in", wl.tokens, wl.linears[0].k_in)
         self.host["x"] = torch.from_numpy(x.view(np.int16)).pin_memory()
         self.x = self.host["x"].to(device)
         self.lin = []
@@ -184,6 +184,27 @@ class LayerOnDevice:
     def nonzero_flops(self):
         self.torch.cuda.synchronize()
         return [2 * self.wl.tokens * int(e["pk"].kept_weights.item()) for e in self.lin]
+
+
+def rank_seed(seed: int, rank: int) -> int:
+    """Seed of a rank's activations: every rank processes its own batch of tokens (weights are replicated)."""
+    return seed + 1000 * rank
+
+
+def reduce_max(values, device, world):
+    """Element-wise maximum over ranks of a list of floats (the job takes as long as its slowest rank)."""
+    if world <= 1:
+        return [float(v) for v in values]
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t.tolist()]
+
+
+def job_throughput(world: int, flops_per_rank_step: int, steps: int, total_ms: float) -> float:
+    """Whole-job TFLOP/s: all ranks' non-zero FLOPs over the slowest rank's time."""
+    return world * flops_per_rank_step * steps / total_ms / 1e9
 
 
 def dense_context(wl, device, iters=20):
@@ -297,10 +318,7 @@ def run_cuda(args):
             e2e_ms.append(e_s.elapsed_time(e_e))
     e2e_total_ms = sum(e2e_ms)
 
-    if world > 1:
-        t = torch.tensor([total_ms, e2e_total_ms], dtype=torch.float64, device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, e2e_total_ms = float(t[0]), float(t[1])
+    total_ms, e2e_total_ms = reduce_max([total_ms, e2e_total_ms], device, world)
 
     if rank == 0:
         peaks, peak_src = measured_peaks()
@@ -308,7 +326,7 @@ def run_cuda(args):
         gemm_total = sum(gemm_mean_ms)
         achieved = step_flops / gemm_total / 1e9          # TFLOP/s over the four GEMM launches of a step
         peak = float(peaks["bf16_tflops"])
-        value = world * step_flops * args.steps / total_ms / 1e9
+        value = job_throughput(world, step_flops, args.steps, total_ms)
         line = {
             "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": round(total_ms / args.steps, 5), "higher_is_better": True,
@@ -323,7 +341,7 @@ def run_cuda(args):
                 "nonzero_gflop_per_step_per_gpu": round(step_flops / 1e9, 3),
             },
             "percent_of_bf16_peak": round(100 * value / world / peak, 2),
-            "e2e": {"value": round(world * step_flops * len(e2e_ms) / e2e_total_ms / 1e9, 3), "unit": UNIT,
+            "e2e": {"value": round(job_throughput(world, step_flops, len(e2e_ms), e2e_total_ms), 3), "unit": UNIT,
                     "h2d_bytes_per_step": layer.h2d_bytes(),
                     "d2h_bytes_per_step": y_host.numel() * 2 + pen_host.numel() * 8},
             "gpu_launches": 2 * layer.kernels_per_step * args.steps,

@@ -114,12 +114,15 @@ fused_stage1_kernel(const __grid_constant__ Batch B) {
   }
 }
 
-// Rows staged in shared memory at a time: up to 24 KB (the whole block for narrow matrices).
+// Rows staged in shared memory at a time: about 24 KB (the whole block for narrow matrices).
+// With the 4-byte index list per column the dynamic shared memory stays under 48 KB for
+// every width up to kFusedMaxCols.
 __host__ __device__ inline int rows_per_pass(int cols) {
   int r = 12288 / cols;
-  r = r < 4 ? 4 : r;
+  r = r < 3 ? 3 : r;
   return r > 16 ? 16 : r;
 }
+static_assert(kFusedMaxCols * (3 * 2 + 4) + 1024 <= 48 * 1024, "stage-2 shared memory must fit the default limit");
 
 // Rows of a row-block that one stage-2 CTA handles: about 16K weights per CTA, a multiple of the
 // 4-row staging pass, so that narrow matrices build their index list once per block and wide ones

@@ -143,7 +143,6 @@ template <int N>
 __device__ __forceinline__ void tma_store_wait_read() {
   asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
 }
-__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 // Named barriers of the epilogue (barrier 0 is __syncthreads): 1 + g among the 128 threads of
 // epilogue group g, 3 among all 256 epilogue threads.
@@ -222,6 +221,9 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
   auto acc_empty_bar = [&](int a) { return bar_base + 8u * (2 * S + 2 + a); };
 
   if (threadIdx.x == 0) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_x)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_w)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_y)) : "memory");
     for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(acc_full_bar(a), 1); mbar_init(acc_empty_bar(a), 8); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -376,7 +378,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
       acc_phase[acc] ^= 1u;
       acc ^= 1;
     }
-    if (issuer) tma_store_wait_all();
+    if (issuer) tma_store_wait_read<0>();   // shared memory must outlive the reads; the writes complete with the grid
     if (!ok && lane == 0) atomicExch(P.status, BSP_ERR_TIMEOUT);
   }
 
