@@ -96,7 +96,7 @@ struct FusedJob {
   int64_t* kept_weights;
   uint16_t* plan;
 };
-constexpr int kFusedMaxJobs = 16;
+constexpr int kFusedMaxJobs = 96;     // per launch; the job table travels as a kernel parameter (about 15 KB)
 constexpr int kFusedMaxCols = 4096;     // stage 2 keeps 12 bytes of shared memory per column
 constexpr int kFusedMaxBlocks = 1024;   // stage 2 sums the counts before its block directly
 // Stage 1: sums of squares -> norms / gamma / penalty and/or keep flags + counts, one pass over W.

@@ -25,10 +25,14 @@ struct Batch {
   FusedJob job[kFusedMaxJobs];
 };
 
+// Job that owns CTA `cta`: the last j with first_block[j] <= cta (binary search).
 __device__ __forceinline__ int find_job(const Batch& B, int cta) {
-  int j = 0;
-  while (j + 1 < B.n_jobs && cta >= B.first_block[j + 1]) ++j;
-  return j;
+  int lo = 0, hi = B.n_jobs - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (B.first_block[mid] <= cta) lo = mid; else hi = mid - 1;
+  }
+  return lo;
 }
 
 __global__ void __launch_bounds__(256)

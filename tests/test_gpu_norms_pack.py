@@ -236,8 +236,8 @@ def test_prepare_batched_optional_outputs_and_many_jobs():
     """More jobs than one launch holds, outputs skipped, the squared-norm penalty, stale gamma."""
     eps, block = 1e-2, 8
     jobs, ws = [], []
-    for n in range(19):
-        w = si.normal_bf16(70 + n, f"many{n}", (64 + 8 * n, 72), 0.02)
+    for n in range(100):
+        w = si.normal_bf16(70 + n, f"many{n}", (64 + 8 * (n % 20), 72), 0.02)
         pk = bsp.PackedMatrix.allocate(w.shape[0], 72, block, bsp.ORIENT_C, DEV)
         stale = (np.abs(si.bf16_bits_to_f32(si.normal_bf16(90 + n, "g", (w.shape[0] // block, 72), 1.0))) + 0.5).astype(np.float32)
         jobs.append(bsp.LayerJob(W=to_dev(w), out=pk, threshold=0.05,
