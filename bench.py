@@ -490,14 +490,41 @@ def run_reference(args):
     }), flush=True)
 
 
+def run_case(args):
+    """A handful of launches of one call on the bench workload, for profilers (no timing, no JSON):
+    --case qkv|attn_out|ffn_up|ffn_down runs that linear's GEMM, --case prepare the batched weight-side call."""
+    import torch
+    torch.cuda.set_device(0)
+    device = torch.device("cuda", 0)
+    layer = LayerOnDevice(workload(), si.DEFAULT_SEED, 0, device)
+    layer.step()
+    torch.cuda.synchronize()
+    bsp = layer.bsp
+    for _ in range(4):
+        if args.case == "prepare":
+            bsp.bsp_prepare_batched(layer.jobs, layer.wl.linears[0].block, EPS, bsp.PEN_L2)
+        else:
+            outs = {"qkv": layer.lin[0]["Y"], "attn_out": layer.lin[1]["Y"], "ffn_up": layer.lin[2]["Y"]}
+            e = next(e for e in layer.lin if e["spec"].name.endswith("." + args.case))
+            spec = e["spec"]
+            bsp.bsp_linear_planned(e["plan"], spec.n_out, spec.k_in, spec.block, layer.source(spec, outs), e["b"],
+                                   int(spec.gelu), e["Y"])
+    bsp.bsp_linear_status()
+    print(f"case {args.case}: 4 launches done")
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["cuda", "reference"], default="cuda")
+    ap.add_argument("--case", choices=["qkv", "attn_out", "ffn_up", "ffn_down", "prepare"], default=None,
+                    help="run a few launches of one call for a profiler and exit")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.case:
+        run_case(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_cuda(args)
