@@ -239,6 +239,13 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
   tcgen05_fence_after();
   const uint32_t tmem_base = *tmem_holder;
 
+  // Programmatic dependent launch: everything above touched only this CTA's shared and tensor
+  // memory and overlaps the tail of the previous kernel in the stream.  From here on the kernel
+  // reads memory that kernel may have written (X, the plan), so wait for it to finish; and let
+  // the next kernel in the stream start its own prologue as soon as SMs become free.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
   const int m_tiles = (P.tokens + kBlockM - 1) / kBlockM;
   const int n_tiles = (P.n_out + BN - 1) / BN;
   const int total_tiles = m_tiles * n_tiles;
@@ -516,8 +523,17 @@ int launch_tc(DeviceInfo* dev, int slot, const void* plan, const void* X, void* 
   const int n_tiles = (P.n_out + BN - 1) / BN;
   const int tiles = m_tiles * n_tiles;
   const int grid = tiles < dev->sms ? tiles : dev->sms;
-  linear_tc_kernel<BN><<<grid, kThreads, Cfg::kSmemBytes, s>>>(map_x, map_w, map_y, P);
-  BSP_LAUNCH_CHECK();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = Cfg::kSmemBytes;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // start while the previous kernel drains
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  BSP_CUDA_TRY(cudaLaunchKernelEx(&cfg, linear_tc_kernel<BN>, map_x, map_w, map_y, P));
   return BSP_OK;
 }
 
