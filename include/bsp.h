@@ -236,6 +236,35 @@ int bsp_linear(const int32_t* blk_ptr, const int32_t* idx, const void* vals,
                void* Y, int ldy, void* ws, size_t ws_bytes, void* stream);
 int bsp_linear_status(void* stream);
 
+/* ---------------------------------------------------------------------------------------------
+ * bsp_linear_chain — several pruned linear layers, each reading the chain input or an earlier
+ * layer's output, in one persistent launch (the paper's deployment target, Sections 3.1 / 4.4, is
+ * the whole encoder; this runs an encoder layer's linears QKV -> attention output -> FFN-up ->
+ * FFN-down back to back).  Every op computes what bsp_linear_planned computes:
+ *   Y_i = act_i( S_i (W_i * Mask_i)^T + b_i ),  S_i = columns [src_col, src_col + k_in) of X
+ *   (src = -1) or of Y_src (0 <= src < i).
+ * Row-tile m of an op needs only row-tile m of its source, so no grid-wide barrier separates the
+ * layers; see csrc/bsp_linear_chain.cu.  Outputs are bit-identical to calling bsp_linear_planned
+ * op by op.
+ *
+ * ops: HOST array of n_ops (1..8) descriptors; plan / bias / Y are device pointers as in
+ * bsp_linear_planned (plan from bsp_linear_plan or bsp_prepare_batched).  ws: device scratch of
+ * bsp_linear_chain_ws_bytes bytes, 256-byte aligned (per-row-tile completion counters; cleared by
+ * the call).  Needs the alignment of the tensor-core path for every op and for src_col
+ * (multiple of 8), else BSP_ERR_UNSUPPORTED; the launch is cooperative (one CTA per SM).
+ * Bounded waits as bsp_linear_planned: check bsp_linear_status.
+ */
+typedef struct bsp_chain_op {
+  const void* plan; int n_out, k_in, block;
+  const void* bias; int act;
+  void* Y; int ldy;
+  int src;       /* -1: the chain input X; i >= 0: the output of op i (must be an earlier op) */
+  int src_col;   /* first column of the source that this op reads */
+} bsp_chain_op;
+int bsp_linear_chain_ws_bytes(int n_ops, int tokens, size_t* bytes);
+int bsp_linear_chain(const bsp_chain_op* ops, int n_ops, const void* X, int tokens, int ldx,
+                     void* ws, size_t ws_bytes, void* stream);
+
 /* bsp_linear_cuda_core — the same layer computed straight from the packed form by a plain
  * CUDA-core kernel (one thread per output, float32 accumulation in index order).  It is what
  * bsp_linear falls back to when the alignment rules above do not hold, and is exported so the

@@ -57,6 +57,16 @@ class _LayerJob(ctypes.Structure):
     ]
 
 
+class _ChainOp(ctypes.Structure):
+    """Mirror of `bsp_chain_op` in bsp.h."""
+    _fields_ = [
+        ("plan", _vp), ("n_out", _i), ("k_in", _i), ("block", _i),
+        ("bias", _vp), ("act", _i),
+        ("Y", _vp), ("ldy", _i),
+        ("src", _i), ("src_col", _i),
+    ]
+
+
 _SIGNATURES = {
     "bsp_status_string": (ctypes.c_char_p, [_i]),
     "bsp_last_cuda_error": (_i, []),
@@ -71,6 +81,8 @@ _SIGNATURES = {
     "bsp_linear_plan": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _sz, _vp]),
     "bsp_linear_planned": (_i, [_vp, _i, _i, _i, _vp, _i, _i, _vp, _i, _vp, _i, _vp]),
     "bsp_linear": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _i, _i, _vp, _i, _vp, _i, _vp, _sz, _vp]),
+    "bsp_linear_chain_ws_bytes": (_i, [_i, _i, _szp]),
+    "bsp_linear_chain": (_i, [ctypes.POINTER(_ChainOp), _i, _vp, _i, _i, _vp, _sz, _vp]),
     "bsp_linear_status": (_i, [_vp]),
     "bsp_linear_cuda_core": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _i, _i, _vp, _i, _vp, _i, _vp]),
 }
@@ -253,6 +265,44 @@ def bsp_linear(packed: PackedMatrix, X: torch.Tensor, bias: Optional[torch.Tenso
     _check(lib.bsp_linear(_ptr(packed.blk_ptr), _ptr(packed.idx), _ptr(packed.vals), packed.rows, packed.cols,
                           packed.block, _ptr(X), X.shape[0], _ld(X), _ptr(bias), act, _ptr(Y), _ld(Y), _ptr(ws),
                           0 if ws is None else ws.numel() * ws.element_size(), _stream(stream)), "bsp_linear")
+
+
+@dataclass
+class ChainOp:
+    """One linear of a bsp_linear_chain call: reads X (src = -1) or the Y of an earlier op, from column src_col."""
+    plan: torch.Tensor
+    n_out: int
+    k_in: int
+    block: int
+    bias: Optional[torch.Tensor]
+    act: int
+    Y: torch.Tensor
+    src: int = -1
+    src_col: int = 0
+
+
+def make_chain_array(ops):
+    """The host descriptor array for bsp_linear_chain; build it once and reuse it for repeated calls."""
+    arr = (_ChainOp * len(ops))()
+    for a, o in zip(arr, ops):
+        a.plan, a.n_out, a.k_in, a.block = _ptr(o.plan), o.n_out, o.k_in, o.block
+        a.bias, a.act = _ptr(o.bias), o.act
+        a.Y, a.ldy = _ptr(o.Y), _ld(o.Y)
+        a.src, a.src_col = o.src, o.src_col
+    return arr
+
+
+def bsp_linear_chain_ws_bytes(n_ops: int, tokens: int) -> int:
+    b = ctypes.c_size_t()
+    _check(lib.bsp_linear_chain_ws_bytes(n_ops, tokens, ctypes.byref(b)), "bsp_linear_chain_ws_bytes")
+    return b.value
+
+
+def bsp_linear_chain(ops, X: torch.Tensor, ws: torch.Tensor, stream=None) -> None:
+    """ops: a list of ChainOp, or an array made by make_chain_array."""
+    arr = ops if isinstance(ops, ctypes.Array) else make_chain_array(ops)
+    _check(lib.bsp_linear_chain(arr, len(arr), _ptr(X), X.shape[0], _ld(X), _ptr(ws), ws.numel() * ws.element_size(),
+                                _stream(stream)), "bsp_linear_chain")
 
 
 def bsp_linear_cuda_core(packed: PackedMatrix, X: torch.Tensor, bias: Optional[torch.Tensor], act: int,

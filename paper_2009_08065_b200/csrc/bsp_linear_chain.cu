@@ -1,0 +1,344 @@
+// bsp_linear_chain: several pruned linear layers whose inputs are earlier layers' outputs (QKV ->
+// attention output -> FFN-up -> FFN-down of an encoder layer), in ONE persistent cooperative
+// launch.  Without attention in between, row-tile m of a layer only needs row-tile m of the layer
+// it reads, so the layers need no grid-wide barrier between them: every CTA walks one global list
+// of 128 x 256 output tiles (all tiles of op 0, then op 1, ...) round-robin, and the TMA producer
+// of a tile first waits until the tiles of the source rows it reads have been stored (a per
+// (op, row-tile) completion counter in global memory, bumped by the epilogue after its TMA stores
+// have completed).  Compared with one launch per layer this removes the launch / prologue / drain
+// of every layer but the first and lets the next layer's tiles fill the SMs that the last,
+// partly filled wave of a layer would leave idle.
+//
+// A tile only ever waits for tiles with a smaller index, and every CTA takes its tiles in
+// increasing order, so the smallest unfinished tile can always proceed; the launch is cooperative
+// so that all CTAs are resident.  The dependency wait, like the mbarrier waits, has a deadline.
+// The pipeline inside a CTA is the one of bsp_linear_tc.cu (TMA producer warp, MMA warp, two
+// epilogue groups of four warps, two TMEM accumulators) with BN fixed at 256.
+#include "bsp_tc.cuh"
+
+namespace bsp {
+using namespace tc;
+
+int check_linear_args(const void* a, const void* b, const void* c, int n_out, int k_in, int block,
+                      const void* X, int tokens, int ldx, int act, const void* Y, int ldy);
+
+namespace {
+
+constexpr int kBN = 256;
+constexpr int kMaxOps = 8;
+using Cfg = TileCfg<kBN>;
+
+struct ChainOp {
+  int n_out, k_blocks, act;
+  int n_tiles;           // output tiles per row-tile (ceil(n_out / 256))
+  int tile_begin;        // global index of this op's first tile
+  int dep;               // op whose output this op reads, or -1 for the chain input
+  int dep_need;          // completions of one source row-tile that make it readable
+  const uint16_t* bias;
+};
+struct ChainParams {
+  int n_ops, m_tiles, total_tiles, tokens;
+  int* done;             // [n_ops][m_tiles] completion counters, zeroed before the launch
+  int* status;
+  ChainOp op[kMaxOps];
+};
+struct ChainMaps {
+  CUtensorMap x[kMaxOps], w[kMaxOps], y[kMaxOps];
+};
+
+struct TileRef {
+  int g, m, n;
+};
+__device__ __forceinline__ TileRef decode_tile(const ChainParams& P, int t) {
+  int g = 0;
+  while (g + 1 < P.n_ops && t >= P.op[g + 1].tile_begin) ++g;
+  const int local = t - P.op[g].tile_begin;
+  const int m = local / P.op[g].n_tiles;
+  return TileRef{g, m, local - m * P.op[g].n_tiles};
+}
+
+// Bounded wait until *counter >= need (acquire at GPU scope).
+__device__ __forceinline__ bool wait_counter(const int* counter, int need) {
+  const unsigned long long start = global_timer_ns();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 64; ++i) {
+      int v;
+      asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(counter) : "memory");
+      if (v >= need) return true;
+    }
+    if (global_timer_ns() - start > kWaitLimitNs) return false;
+  }
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+linear_chain_kernel(const __grid_constant__ ChainMaps M, const __grid_constant__ ChainParams P) {
+  constexpr int S = Cfg::kStages;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+  // [S operand stages][2 epilogue staging buffers][bias, bf16, for two tiles][mbarriers, TMEM base]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S * Cfg::kStage + 2 * kEpiStage + 2 * kBN * 2);
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 2 * S + 4);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t smem_base = smem_u32(smem);
+  const uint32_t bar_base = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (S + s); };
+  auto acc_full_bar = [&](int a) { return bar_base + 8u * (2 * S + a); };
+  auto acc_empty_bar = [&](int a) { return bar_base + 8u * (2 * S + 2 + a); };
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(acc_full_bar(a), 1); mbar_init(acc_empty_bar(a), 8); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_holder)),
+                 "r"(static_cast<uint32_t>(Cfg::kTmemCols)) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tcgen05_fence_before();
+  __syncthreads();
+  tcgen05_fence_after();
+  const uint32_t tmem_base = *tmem_holder;
+
+  if (warp == 0 && lane == 0) {
+    // ---------------------------------------------------------------- TMA producer
+    int stage = 0;
+    uint32_t phase = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < P.total_tiles && ok; tile += gridDim.x) {
+      const TileRef T = decode_tile(P, tile);
+      const ChainOp& op = P.op[T.g];
+      if (op.dep >= 0) {
+        // the rows this tile reads were written by other CTAs' TMA stores
+        if (!wait_counter(P.done + op.dep * P.m_tiles + T.m, op.dep_need)) { ok = false; break; }
+        asm volatile("fence.proxy.async;" ::: "memory");   // order the acquire before the async-proxy reads below
+      }
+      for (int kb = 0; kb < op.k_blocks; ++kb) {
+        if (!mbar_wait(empty_bar(stage), phase ^ 1u)) { ok = false; break; }
+        const uint32_t a_dst = smem_base + stage * Cfg::kStage;
+        const uint32_t b_dst = a_dst + Cfg::kStageA;
+        mbar_arrive_expect_tx(full_bar(stage), Cfg::kStage);
+        tma_load_2d(a_dst, &M.x[T.g], kb * kBlockK, T.m * kBlockM, full_bar(stage));
+        tma_load_2d(b_dst, &M.w[T.g], kb * kBlockK, T.n * kBN, full_bar(stage));
+        if (++stage == S) { stage = 0; phase ^= 1u; }
+      }
+    }
+    if (!ok) {
+      atomicExch(P.status, BSP_ERR_TIMEOUT);
+      for (int s = 0; s < S; ++s) {   // bounded chance for copies already issued to land
+        const int back = (stage - 1 - s + 2 * S) % S;
+        const uint32_t ph = (back < stage) ? phase : (phase ^ 1u);
+        (void)mbar_wait(full_bar(back), ph);
+      }
+    }
+  } else if (warp == 1 && lane == 0) {
+    // ---------------------------------------------------------------- MMA issuer
+    constexpr uint32_t idesc = instr_desc_bf16(kBN);
+    int stage = 0;
+    uint32_t phase = 0;
+    uint32_t acc_phase[2] = {0u, 0u};
+    int acc = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < P.total_tiles && ok; tile += gridDim.x) {
+      const int k_blocks = P.op[decode_tile(P, tile).g].k_blocks;
+      if (!mbar_wait(acc_empty_bar(acc), acc_phase[acc] ^ 1u)) { ok = false; break; }
+      tcgen05_fence_after();
+      const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * kBN);
+      for (int kb = 0; kb < k_blocks; ++kb) {
+        if (!mbar_wait(full_bar(stage), phase)) { ok = false; break; }
+        tcgen05_fence_after();
+        const uint32_t a_addr = smem_base + stage * Cfg::kStage;
+        const uint32_t b_addr = a_addr + Cfg::kStageA;
+#pragma unroll
+        for (int k = 0; k < kBlockK / kUmmaK; ++k)
+          tcgen05_mma_bf16(d_tmem, smem_desc_sw128(a_addr + k * kUmmaK * 2), smem_desc_sw128(b_addr + k * kUmmaK * 2),
+                           idesc, (kb | k) != 0 ? 1u : 0u);
+        tcgen05_commit(empty_bar(stage));
+        if (++stage == S) { stage = 0; phase ^= 1u; }
+      }
+      if (!ok) break;
+      tcgen05_commit(acc_full_bar(acc));
+      acc_phase[acc] ^= 1u;
+      acc ^= 1;
+    }
+    if (!ok) atomicExch(P.status, BSP_ERR_TIMEOUT);
+  } else if (warp >= 2) {
+    // ---------------------------------------------------------------- epilogue (two groups of four warps)
+    const int group = (warp - 2) >> 2;
+    const int quad = warp & 3;
+    const int row = quad * 32 + lane;
+    const int epi_tid = threadIdx.x - 64;
+    const bool issuer = (epi_tid & 127) == 0;
+    const uint32_t buf = smem_base + S * Cfg::kStage + group * kEpiStage;
+    uint16_t* s_bias = reinterpret_cast<uint16_t*>(smem + S * Cfg::kStage + 2 * kEpiStage);   // [2][256] bf16
+    const uint32_t row_off = static_cast<uint32_t>(row) * 128u;
+    const uint32_t row_xor = static_cast<uint32_t>(row & 7);
+    uint32_t acc_phase[2] = {0u, 0u};
+    int acc = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < P.total_tiles && ok; tile += gridDim.x) {
+      const TileRef T = decode_tile(P, tile);
+      const ChainOp& op = P.op[T.g];
+      const int m0 = T.m * kBlockM, n0 = T.n * kBN;
+      for (int c = epi_tid; c < kBN; c += 256)
+        s_bias[acc * kBN + c] = (op.bias != nullptr && n0 + c < op.n_out) ? __ldg(op.bias + n0 + c) : static_cast<uint16_t>(0);
+      epilogue_sync_all();
+      if (!mbar_wait(acc_full_bar(acc), acc_phase[acc])) { ok = false; break; }
+      tcgen05_fence_after();
+      const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + static_cast<uint32_t>(acc * kBN);
+      const int pieces = (min(kBN, op.n_out - n0) + kEpiCols - 1) / kEpiCols;
+      bool released = false;
+#pragma unroll 1
+      for (int pc = group; pc < pieces; pc += 2) {
+        const int c0 = pc * kEpiCols;
+        if (issuer) tma_store_wait_read<0>();
+        group_sync(group);
+        uint32_t v0[32], v1[32];
+        tmem_load_32cols(taddr + c0, v0);
+        tmem_load_32cols(taddr + c0 + 32, v1);
+        tmem_load_wait();
+        if (pc + 2 >= pieces) {
+          tcgen05_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(acc_empty_bar(acc));
+          released = true;
+        }
+        const uint16_t* bias_c = s_bias + acc * kBN + c0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const uint32_t* v = j < 4 ? &v0[j * 8] : &v1[(j - 4) * 8];
+          const uint4 b8 = *reinterpret_cast<const uint4*>(bias_c + j * 8);
+          const uint32_t bw[4] = {b8.x, b8.y, b8.z, b8.w};
+          float f[8];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            f[2 * i] = __uint_as_float(v[2 * i]) + __uint_as_float(bw[i] << 16);
+            f[2 * i + 1] = __uint_as_float(v[2 * i + 1]) + __uint_as_float(bw[i] & 0xffff0000u);
+          }
+          if (op.act == BSP_ACT_GELU) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) f[i] = gelu_erf(f[i]);
+          }
+          st_shared_v4(buf + row_off + ((static_cast<uint32_t>(j) ^ row_xor) << 4), pack_bf16x2(f[0], f[1]),
+                       pack_bf16x2(f[2], f[3]), pack_bf16x2(f[4], f[5]), pack_bf16x2(f[6], f[7]));
+        }
+        fence_async_smem();
+        group_sync(group);
+        if (issuer) {
+          tma_store_2d(&M.y[T.g], n0 + c0, m0, buf);
+          tma_store_commit();
+        }
+      }
+      if (!released) {
+        tcgen05_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(acc_empty_bar(acc));
+      }
+      // publish this group's share of the tile: its stores have to be complete (not merely read out
+      // of shared memory) before a consumer on another SM may load the rows
+      if (issuer) {
+        asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+        asm volatile("fence.proxy.async;" ::: "memory");
+        __threadfence();
+        atomicAdd(P.done + T.g * P.m_tiles + T.m, 1);
+      }
+      acc_phase[acc] ^= 1u;
+      acc ^= 1;
+    }
+    if (!ok && lane == 0) atomicExch(P.status, BSP_ERR_TIMEOUT);
+  }
+
+  tcgen05_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tcgen05_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                 "r"(static_cast<uint32_t>(Cfg::kTmemCols)) : "memory");
+  }
+}
+
+}  // namespace
+}  // namespace bsp
+
+extern "C" int bsp_linear_chain_ws_bytes(int n_ops, int tokens, size_t* bytes) {
+  using namespace bsp;
+  if (n_ops <= 0 || n_ops > kMaxOps || tokens < 0 || bytes == nullptr) return BSP_ERR_ARG;
+  const size_t m_tiles = (static_cast<size_t>(tokens) + kBlockM - 1) / kBlockM;
+  *bytes = round_up(sizeof(int) * n_ops * (m_tiles ? m_tiles : 1), 256);
+  return BSP_OK;
+}
+
+extern "C" int bsp_linear_chain(const bsp_chain_op* ops, int n_ops, const void* X, int tokens, int ldx,
+                                void* ws, size_t ws_bytes, void* stream) {
+  using namespace bsp;
+  if (ops == nullptr || X == nullptr || ws == nullptr) return BSP_ERR_ARG;
+  size_t need = 0;
+  int st = bsp_linear_chain_ws_bytes(n_ops, tokens, &need);
+  if (st != BSP_OK) return st;
+  if (!aligned_to(ws, 256) || !aligned_to(X, 16) || ldx % 8) return BSP_ERR_ARG;
+  if (ws_bytes < need) return BSP_ERR_WORKSPACE;
+  const int m_tiles = (tokens + kBlockM - 1) / kBlockM;
+
+  ChainParams P = {};
+  ChainMaps M;
+  P.n_ops = n_ops;
+  P.m_tiles = m_tiles;
+  P.tokens = tokens;
+  int tile_begin = 0;
+  for (int i = 0; i < n_ops; ++i) {
+    const bsp_chain_op& u = ops[i];
+    const void* src = X;
+    int src_ld = ldx, src_cols = ldx;
+    if (u.src >= i) return BSP_ERR_ARG;                        // a source must be an earlier op
+    if (u.src >= 0) { src = ops[u.src].Y; src_ld = ops[u.src].ldy; src_cols = ops[u.src].n_out; }
+    st = check_linear_args(u.plan, u.plan, u.plan, u.n_out, u.k_in, u.block, src, tokens, src_ld, u.act, u.Y, u.ldy);
+    if (st != BSP_OK) return st;
+    if (u.src_col < 0 || u.src_col % 8 || u.src_col + u.k_in > src_cols) return BSP_ERR_SHAPE;
+    if (!aligned_to(u.plan, 16) || !aligned_to(u.Y, 16) || u.k_in % 8 || u.n_out % 8 || u.ldy % 8 || src_ld % 8)
+      return BSP_ERR_UNSUPPORTED;
+    if (tokens == 0) continue;
+    const uint16_t* src_base = static_cast<const uint16_t*>(src) + u.src_col;
+    if (!make_map(&M.x[i], src_base, u.k_in, tokens, src_ld, kBlockM)) return BSP_ERR_CUDA;
+    if (!make_map(&M.w[i], u.plan, u.k_in, u.n_out, u.k_in, kBN)) return BSP_ERR_CUDA;
+    if (!make_map(&M.y[i], u.Y, u.n_out, tokens, u.ldy, kBlockM)) return BSP_ERR_CUDA;
+    ChainOp& o = P.op[i];
+    o.n_out = u.n_out;
+    o.k_blocks = (u.k_in + kBlockK - 1) / kBlockK;
+    o.act = u.act;
+    o.n_tiles = (u.n_out + kBN - 1) / kBN;
+    o.tile_begin = tile_begin;
+    o.dep = u.src;
+    o.dep_need = u.src >= 0 ? 2 * P.op[u.src].n_tiles : 0;   // each tile is published by its two epilogue groups
+    o.bias = static_cast<const uint16_t*>(u.bias);
+    tile_begin += o.n_tiles * m_tiles;
+  }
+  if (tokens == 0) return BSP_OK;
+  P.total_tiles = tile_begin;
+
+  TcDevice* dev = tc_device();
+  if (dev == nullptr) return BSP_ERR_CUDA;
+  P.status = dev->status;
+  P.done = static_cast<int*>(ws);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  BSP_CUDA_TRY(cudaMemsetAsync(ws, 0, need, s));
+  if (!dev->attr_set[4]) {
+    BSP_CUDA_TRY(cudaFuncSetAttribute(linear_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes));
+    dev->attr_set[4] = true;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(P.total_tiles < dev->sms ? P.total_tiles : dev->sms);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = Cfg::kSmemBytes;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeCooperative;   // all CTAs resident: tiles wait on tiles of other CTAs
+  attr[0].val.cooperative = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  BSP_CUDA_TRY(cudaLaunchKernelEx(&cfg, linear_chain_kernel, M, P));
+  return BSP_OK;
+}
