@@ -230,6 +230,14 @@ int bsp_linear_plan(const int32_t* blk_ptr, const int32_t* idx, const void* vals
 int bsp_linear_planned(const void* plan, int n_out, int k_in, int block,
                        const void* X, int tokens, int ldx, const void* bias, int act,
                        void* Y, int ldy, void* stream);
+/* bsp_linear_planned with the kernel variant chosen by the caller: BSP_LINEAR_AUTO (what
+ * bsp_linear_planned does), BSP_LINEAR_ONE_CTA (128 x BN tiles, one CTA each) or
+ * BSP_LINEAR_CTA_PAIR (256 x 256 tiles shared by a cluster of two CTAs, one third less operand
+ * traffic from L2).  Results are identical up to float32 summation order (the same in both). */
+typedef enum { BSP_LINEAR_AUTO = 0, BSP_LINEAR_ONE_CTA = 1, BSP_LINEAR_CTA_PAIR = 2 } bsp_linear_algo;
+int bsp_linear_planned_ex(const void* plan, int n_out, int k_in, int block,
+                          const void* X, int tokens, int ldx, const void* bias, int act,
+                          void* Y, int ldy, int algo, void* stream);
 int bsp_linear(const int32_t* blk_ptr, const int32_t* idx, const void* vals,
                int n_out, int k_in, int block,
                const void* X, int tokens, int ldx, const void* bias, int act,

@@ -80,6 +80,7 @@ _SIGNATURES = {
     "bsp_linear_plan_bytes": (_i, [_i, _i, _i, _szp]),
     "bsp_linear_plan": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _sz, _vp]),
     "bsp_linear_planned": (_i, [_vp, _i, _i, _i, _vp, _i, _i, _vp, _i, _vp, _i, _vp]),
+    "bsp_linear_planned_ex": (_i, [_vp, _i, _i, _i, _vp, _i, _i, _vp, _i, _vp, _i, _i, _vp]),
     "bsp_linear": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _i, _i, _vp, _i, _vp, _i, _vp, _sz, _vp]),
     "bsp_linear_chain_ws_bytes": (_i, [_i, _i, _szp]),
     "bsp_linear_chain": (_i, [ctypes.POINTER(_ChainOp), _i, _vp, _i, _i, _vp, _sz, _vp]),
@@ -258,6 +259,16 @@ def bsp_linear_planned(plan: torch.Tensor, n_out: int, k_in: int, block: int, X:
                        bias: Optional[torch.Tensor], act: int, Y: torch.Tensor, stream=None) -> None:
     _check(lib.bsp_linear_planned(_ptr(plan), n_out, k_in, block, _ptr(X), X.shape[0], _ld(X), _ptr(bias), act,
                                   _ptr(Y), _ld(Y), _stream(stream)), "bsp_linear_planned")
+
+
+LINEAR_AUTO, LINEAR_ONE_CTA, LINEAR_CTA_PAIR = 0, 1, 2
+
+
+def bsp_linear_planned_ex(plan: torch.Tensor, n_out: int, k_in: int, block: int, X: torch.Tensor,
+                          bias: Optional[torch.Tensor], act: int, Y: torch.Tensor, algo: int = LINEAR_AUTO,
+                          stream=None) -> None:
+    _check(lib.bsp_linear_planned_ex(_ptr(plan), n_out, k_in, block, _ptr(X), X.shape[0], _ld(X), _ptr(bias), act,
+                                     _ptr(Y), _ld(Y), algo, _stream(stream)), "bsp_linear_planned_ex")
 
 
 def bsp_linear(packed: PackedMatrix, X: torch.Tensor, bias: Optional[torch.Tensor], act: int, Y: torch.Tensor,

@@ -31,6 +31,8 @@ namespace bsp {
 
 int check_linear_args(const void* a, const void* b, const void* c, int n_out, int k_in, int block,
                       const void* X, int tokens, int ldx, int act, const void* Y, int ldy);
+int launch_tc_pair(TcDevice* dev, const void* plan, const void* X, void* Y, int tokens, int n_out, int k_in, int act,
+                   const void* bias, int ldx, int ldy, cudaStream_t s);
 
 using namespace tc;
 
@@ -383,23 +385,34 @@ extern "C" int bsp_linear_plan(const int32_t* blk_ptr, const int32_t* idx, const
   return BSP_OK;
 }
 
-extern "C" int bsp_linear_planned(const void* plan, int n_out, int k_in, int block, const void* X, int tokens,
-                                  int ldx, const void* bias, int act, void* Y, int ldy, void* stream) {
+extern "C" int bsp_linear_planned_ex(const void* plan, int n_out, int k_in, int block, const void* X, int tokens,
+                                     int ldx, const void* bias, int act, void* Y, int ldy, int algo, void* stream) {
   using namespace bsp;
   int st = check_linear_args(plan, plan, plan, n_out, k_in, block, X, tokens, ldx, act, Y, ldy);
   if (st != BSP_OK) return st;
+  if (algo < BSP_LINEAR_AUTO || algo > BSP_LINEAR_CTA_PAIR) return BSP_ERR_ARG;
   if (!tc_path_ok(plan, n_out, k_in, X, ldx, Y, ldy)) return BSP_ERR_UNSUPPORTED;
   if (tokens == 0) return BSP_OK;
   TcDevice* dev = tc_device();
   if (dev == nullptr) return BSP_ERR_CUDA;
-  LinearParams P{tokens, n_out, k_in, act, static_cast<const uint16_t*>(bias), dev->status};
   cudaStream_t s = static_cast<cudaStream_t>(stream);
+  // Measured on B200: CTA pairs win (about 5 %) once the problem runs for many waves, where the L2 -> SM
+  // operand traffic binds; for a few waves the one-CTA kernel's shorter start-up wins (about 2 us).
+  const long long pair_tiles = static_cast<long long>((tokens + 255) / 256) * ((n_out + 255) / 256);
+  const bool pair = algo == BSP_LINEAR_CTA_PAIR || (algo == BSP_LINEAR_AUTO && pair_tiles >= 4LL * dev->sms);
+  if (pair) return launch_tc_pair(dev, plan, X, Y, tokens, n_out, k_in, act, bias, ldx, ldy, s);
+  LinearParams P{tokens, n_out, k_in, act, static_cast<const uint16_t*>(bias), dev->status};
   switch (choose_bn(tokens, n_out, dev->sms)) {
     case 256: return launch_tc<256>(dev, 0, plan, X, Y, P, ldx, ldy, s);
     case 192: return launch_tc<192>(dev, 1, plan, X, Y, P, ldx, ldy, s);
     case 128: return launch_tc<128>(dev, 2, plan, X, Y, P, ldx, ldy, s);
     default: return launch_tc<64>(dev, 3, plan, X, Y, P, ldx, ldy, s);
   }
+}
+
+extern "C" int bsp_linear_planned(const void* plan, int n_out, int k_in, int block, const void* X, int tokens,
+                                  int ldx, const void* bias, int act, void* Y, int ldy, void* stream) {
+  return bsp_linear_planned_ex(plan, n_out, k_in, block, X, tokens, ldx, bias, act, Y, ldy, BSP_LINEAR_AUTO, stream);
 }
 
 extern "C" int bsp_linear(const int32_t* blk_ptr, const int32_t* idx, const void* vals, int n_out, int k_in,

@@ -166,3 +166,23 @@ def test_plan_is_reusable():
         assert_linear_close(bits_of(y), y_ref, scales, "planned")
     # the plan is W * Mask laid out densely
     assert np.array_equal(bits_of(plan.view(torch.int16)[: 384 * 256].reshape(384, 256)), wp)
+
+
+@pytest.mark.parametrize("T,N,K,act", [(4096, 2304, 768, 0), (300, 520, 136, 1), (1, 256, 64, 0), (777, 768, 3072, 1)])
+def test_cta_pair_kernel_matches_one_cta_kernel_and_oracle(T, N, K, act):
+    """The two tensor-core variants (one CTA per 128 x BN tile, a CTA pair per 256 x 256 tile) agree bit for bit."""
+    spec, wp, keep, x, b = make_case(14, f"pair{T}x{N}x{K}", T, N, K, 8, 2.0, act)
+    pk = gpu_pack(wp, 8)
+    plan = torch.empty(bsp.bsp_linear_plan_bytes(N, K, 8), dtype=torch.uint8, device=DEV)
+    bsp.bsp_linear_plan(pk, plan)
+    xd, bd = to_dev(x), to_dev(b)
+    ys = []
+    for algo in (bsp.LINEAR_ONE_CTA, bsp.LINEAR_CTA_PAIR):
+        y = torch.full((T, N), 0x7FC0, dtype=torch.int16, device=DEV)
+        bsp.bsp_linear_planned_ex(plan, N, K, 8, xd, bd, act, y, algo)
+        bsp.bsp_linear_status()
+        ys.append(y)
+    assert torch.equal(ys[0], ys[1])
+    if T <= 1024:
+        y_ref, scales = oracle_linear(x, wp, b, act)
+        assert_linear_close(bits_of(ys[1]), y_ref, scales, "pair")
