@@ -4,7 +4,7 @@
 One *step* = one pass of the whole path over one batch of synthetic input, for each of the four
 linears of a BERT-base encoder layer at 4096 tokens (16-row blocks, 3.0x compression):
     norms, gamma, penalty  ->  Algorithm 1 keep flags + packed storage  ->  execution layout
-    (bsp_prepare_batched: one call for the four matrices)  ->  bsp_linear_chain (tcgen05 GEMMs + bias [+ GELU]),
+    (bsp_prepare_batched: one call for the four matrices)  ->  bsp_linear_planned (tcgen05 GEMM + bias [+ GELU]),
 with the layer's outputs chained (attention-output reads the V third of QKV's output, FFN-up
 reads attention-output's result through GELU, FFN-down reads FFN-up's).
 
@@ -142,7 +142,7 @@ class LayerOnDevice:
                 "Y": torch.empty((wl.tokens, spec.n_out), dtype=torch.int16, device=device),
             }
             self.lin.append(e)
-        self.kernels_per_step = 3   # two weight-side launches for the batch, one chained launch for the four linears
+        self.kernels_per_step = 2 + len(self.lin)   # two weight-side launches for the batch, one GEMM per matrix
 
     def source(self, spec, outs):
         if spec.src == "x":
@@ -154,33 +154,23 @@ class LayerOnDevice:
 
     def step(self, gemm_events=None):
         """One pass of the path: one batched weight-side call for the four matrices (norms, gamma, penalty,
-        keep flags, pack, plan: two launches), then the four linears as one chained persistent launch."""
-        bsp = self.bsp
+        keep flags, pack, plan: two launches), then the four GEMMs in order."""
+        bsp, outs = self.bsp, {}
         if not hasattr(self, "jobs"):
             self.jobs = bsp.make_job_array([
                 bsp.LayerJob(W=e["W"], out=e["pk"], threshold=0.0, norms=e["norms"], gamma_out=e["gamma"],
                              penalty=e["penalty"], plan=e["plan"]) for e in self.lin])
-            names = [e["spec"].name.split(".")[1] for e in self.lin]
-            ops = []
-            for e in self.lin:
-                spec = e["spec"]
-                src, col = -1, 0
-                if spec.src == "qkv_v":
-                    src, col = names.index("qkv"), 2 * spec.k_in
-                elif spec.src != "x":
-                    src = names.index(spec.src)
-                ops.append(bsp.ChainOp(plan=e["plan"], n_out=spec.n_out, k_in=spec.k_in, block=spec.block, bias=e["b"],
-                                       act=int(spec.gelu), Y=e["Y"], src=src, src_col=col))
-            self.chain = bsp.make_chain_array(ops)
-            self.chain_ws = self.torch.empty(bsp.bsp_linear_chain_ws_bytes(len(ops), self.wl.tokens),
-                                             dtype=self.torch.uint8, device=self.device)
         bsp.bsp_prepare_batched(self.jobs, self.wl.linears[0].block, EPS, bsp.PEN_L2)
-        if gemm_events is not None:
-            gemm_events[0].record()
-        bsp.bsp_linear_chain(self.chain, self.x, self.chain_ws)
-        if gemm_events is not None:
-            gemm_events[1].record()
-        return {e["spec"].name.split(".")[1]: e["Y"] for e in self.lin}
+        for i, e in enumerate(self.lin):
+            spec = e["spec"]
+            src = self.source(spec, outs)
+            if gemm_events is not None:
+                gemm_events[i][0].record()
+            bsp.bsp_linear_planned(e["plan"], spec.n_out, spec.k_in, spec.block, src, e["b"], int(spec.gelu), e["Y"])
+            if gemm_events is not None:
+                gemm_events[i][1].record()
+            outs[spec.name.split(".")[1]] = e["Y"]
+        return outs
 
     def upload_inputs(self):
         self.x.copy_(self.host["x"], non_blocking=True)
@@ -320,7 +310,7 @@ def run_cuda(args):
     # each, so they are kept out of the step that is timed as a whole).
     ev = lambda: torch.cuda.Event(enable_timing=True, external=True)  # noqa: E731
     ev_step = (ev(), ev())
-    ev_gemm = (ev(), ev())
+    ev_gemm = [(ev(), ev()) for _ in layer.lin]
     graph, graph_k = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
     with torch.cuda.graph(graph):
         ev_step[0].record()
@@ -340,7 +330,7 @@ def run_cuda(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    step_ms, gemm_ms = [], []
+    step_ms, gemm_ms = [], [[] for _ in layer.lin]
     barrier()
     with ClockSampler(local_rank) as clocks:
         for _ in range(args.steps):
@@ -351,7 +341,8 @@ def run_cuda(args):
             flush.zero_()
             graph_k.replay()               # same step again, instrumented per kernel (not part of `value`)
             torch.cuda.synchronize()
-            gemm_ms.append(ev_gemm[0].elapsed_time(ev_gemm[1]))
+            for i, (a, b) in enumerate(ev_gemm):
+                gemm_ms[i].append(a.elapsed_time(b))
     barrier()
     layer.bsp.bsp_linear_status()
     total_ms = sum(step_ms)
@@ -379,8 +370,9 @@ def run_cuda(args):
 
     if rank == 0:
         peaks, peak_src = measured_peaks()
-        gemm_total = statistics.mean(gemm_ms)
-        achieved = step_flops / gemm_total / 1e9          # non-zero TFLOP/s of the chained GEMM launch
+        gemm_mean_ms = [statistics.mean(v) for v in gemm_ms]
+        gemm_total = sum(gemm_mean_ms)
+        achieved = step_flops / gemm_total / 1e9          # TFLOP/s over the four GEMM launches of a step
         peak = float(peaks["bf16_tflops"])
         value = job_throughput(world, step_flops, args.steps, total_ms)
         line = {
@@ -391,7 +383,8 @@ def run_cuda(args):
                 "workload": wl.name + " (one BERT-base encoder layer: QKV, attn-out, FFN-up+GELU, FFN-down; "
                             "tokens per GPU 4096; 16-row blocks; 3.0x compression)",
                 "step": "bsp_prepare_batched (norms+gamma+penalty, keep flags, pack, plan of the 4 matrices: 2 launches) "
-                        "then bsp_linear_chain (the 4 GEMMs in one persistent launch); one CUDA graph",
+                        "then the 4 GEMMs in sequence (bsp_linear_planned; the single chained launch bsp_linear_chain measured "
+                        "8 % slower on this workload); one CUDA graph",
                 "l2": f"flushed between steps by writing {L2_FLUSH_BYTES >> 20} MiB",
                 "parallelism": "token split, replicated weights, no collective" if world > 1 else "single GPU",
                 "nonzero_gflop_per_step_per_gpu": round(step_flops / 1e9, 3),
@@ -403,12 +396,13 @@ def run_cuda(args):
             "gpu_launches": 2 * layer.kernels_per_step * args.steps,
             "clocks": clocks.summary(),
             "roofline": {
-                "kernel": "linear_chain_kernel (bsp_linear_chain): the layer's four linears in one launch",
+                "kernel": "linear_tc_kernel (bsp_linear_planned), the four launches of a step",
                 "bound": "tensor", "achieved": round(achieved, 2), "peak": peak, "unit": "TFLOP/s",
                 "frac": round(achieved / peak, 4), "traffic": None,
                 "peak_source": f"bf16_tflops burst, {peak_src}",
-                "launch_ms": round(gemm_total, 5), "dense_tflops_executed": round(
-                    sum(2 * wl.tokens * sp.n_out * sp.k_in for sp in wl.linears) / gemm_total / 1e9, 1),
+                "per_launch": {e["spec"].name.split(".")[1]: {
+                    "ms": round(gemm_mean_ms[i], 5), "nonzero_tflops": round(flops[i] / gemm_mean_ms[i] / 1e9, 1)}
+                    for i, e in enumerate(layer.lin)},
             },
         }
         if world == 1:
@@ -499,8 +493,7 @@ def run_reference(args):
 
 def run_case(args):
     """A handful of launches of one call on the bench workload, for profilers (no timing, no JSON):
-    --case qkv|attn_out|ffn_up|ffn_down runs that linear's GEMM alone, --case chain the chained launch of all
-    four, --case prepare the batched weight-side call."""
+    --case qkv|attn_out|ffn_up|ffn_down runs that linear's GEMM, --case prepare the batched weight-side call."""
     import torch
     torch.cuda.set_device(0)
     device = torch.device("cuda", 0)
@@ -511,8 +504,6 @@ def run_case(args):
     for _ in range(4):
         if args.case == "prepare":
             bsp.bsp_prepare_batched(layer.jobs, layer.wl.linears[0].block, EPS, bsp.PEN_L2)
-        elif args.case == "chain":
-            bsp.bsp_linear_chain(layer.chain, layer.x, layer.chain_ws)
         else:
             outs = {"qkv": layer.lin[0]["Y"], "attn_out": layer.lin[1]["Y"], "ffn_up": layer.lin[2]["Y"]}
             e = next(e for e in layer.lin if e["spec"].name.endswith("." + args.case))
@@ -529,7 +520,7 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["cuda", "reference"], default="cuda")
-    ap.add_argument("--case", choices=["qkv", "attn_out", "ffn_up", "ffn_down", "prepare", "chain"], default=None,
+    ap.add_argument("--case", choices=["qkv", "attn_out", "ffn_up", "ffn_down", "prepare"], default=None,
                     help="run a few launches of one call for a profiler and exit")
     args = ap.parse_args()
     if args.case:
