@@ -197,35 +197,15 @@ linear_chain_kernel(const __grid_constant__ ChainMaps M, const __grid_constant__
         const int c0 = pc * kEpiCols;
         if (issuer) tma_store_wait_read<0>();
         group_sync(group);
-        uint32_t v0[32], v1[32];
-        tmem_load_32cols(taddr + c0, v0);
-        tmem_load_32cols(taddr + c0 + 32, v1);
-        tmem_load_wait();
+        EpiloguePiece piece;
+        piece_load(taddr + c0, smem_u32(s_bias + acc * kBN + c0), piece);
         if (pc + 2 >= pieces) {
           tcgen05_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(acc_empty_bar(acc));
           released = true;
         }
-        const uint16_t* bias_c = s_bias + acc * kBN + c0;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const uint32_t* v = j < 4 ? &v0[j * 8] : &v1[(j - 4) * 8];
-          const uint4 b8 = *reinterpret_cast<const uint4*>(bias_c + j * 8);
-          const uint32_t bw[4] = {b8.x, b8.y, b8.z, b8.w};
-          float f[8];
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            f[2 * i] = __uint_as_float(v[2 * i]) + __uint_as_float(bw[i] << 16);
-            f[2 * i + 1] = __uint_as_float(v[2 * i + 1]) + __uint_as_float(bw[i] & 0xffff0000u);
-          }
-          if (op.act == BSP_ACT_GELU) {
-#pragma unroll
-            for (int i = 0; i < 8; ++i) f[i] = gelu_erf(f[i]);
-          }
-          st_shared_v4(buf + row_off + ((static_cast<uint32_t>(j) ^ row_xor) << 4), pack_bf16x2(f[0], f[1]),
-                       pack_bf16x2(f[2], f[3]), pack_bf16x2(f[4], f[5]), pack_bf16x2(f[6], f[7]));
-        }
+        piece_store(piece, op.act, buf + row_off, row_xor);
         fence_async_smem();
         group_sync(group);
         if (issuer) {

@@ -125,8 +125,16 @@ __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.a
 // epilogue group g, 3 among all 256 epilogue threads.
 __device__ __forceinline__ void group_sync(int g) { asm volatile("bar.sync %0, 128;" ::"r"(1 + g) : "memory"); }
 __device__ __forceinline__ void epilogue_sync_all() { asm volatile("bar.sync 3, 256;" ::: "memory"); }
+// Shared-memory accesses of the epilogue as volatile asm WITHOUT a memory clobber: they keep their
+// order among themselves and with the fences and barriers around them (all volatile asm), but do
+// not stop the compiler from hoisting the bias loads of a whole piece ahead of its stores.
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d));
+}
+__device__ __forceinline__ uint4 ld_shared_v4(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+  return v;
 }
 __device__ __forceinline__ void tmem_load_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
@@ -164,11 +172,47 @@ __device__ __forceinline__ float gelu_erf(float x) {
 }
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
-  const uint32_t l = __bfloat16_as_ushort(__float2bfloat16_rn(lo));
-  const uint32_t h = __bfloat16_as_ushort(__float2bfloat16_rn(hi));
-  return l | (h << 16);
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));   // upper half <- first source
+  return r;
 }
 
+// One 64-column piece of a thread's accumulator row, with the bias of those columns.
+struct EpiloguePiece {
+  uint32_t v0[32], v1[32];   // float32 accumulators as bits
+  uint4 bias[8];             // 64 bf16 values
+};
+// Issues the TMEM loads and, while they are in flight, the eight shared-memory loads of the
+// bias; returns once the accumulator values are in registers.  Shared memory is also being
+// written by TMA and read by the tensor core all the time, so a shared load takes on the order of
+// 150 cycles here: the loads must be in flight together, not one per use.
+__device__ __forceinline__ void piece_load(uint32_t taddr, uint32_t bias_smem, EpiloguePiece& p) {
+  tmem_load_32cols(taddr, p.v0);
+  tmem_load_32cols(taddr + 32, p.v1);
+#pragma unroll
+  for (int j = 0; j < 8; ++j) p.bias[j] = ld_shared_v4(bias_smem + 16u * j);
+  tmem_load_wait();
+}
+// bias + optional GELU + bf16 rounding, into this thread's row of the swizzled staging buffer.
+__device__ __forceinline__ void piece_store(const EpiloguePiece& p, int act, uint32_t dst_row, uint32_t row_xor) {
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {        // 8 outputs -> one 16-byte chunk of the 128-byte staging row
+    const uint32_t* v = j < 4 ? &p.v0[j * 8] : &p.v1[(j - 4) * 8];
+    const uint32_t bw[4] = {p.bias[j].x, p.bias[j].y, p.bias[j].z, p.bias[j].w};
+    float f[8];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      f[2 * i] = __uint_as_float(v[2 * i]) + __uint_as_float(bw[i] << 16);
+      f[2 * i + 1] = __uint_as_float(v[2 * i + 1]) + __uint_as_float(bw[i] & 0xffff0000u);
+    }
+    if (act == BSP_ACT_GELU) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) f[i] = gelu_erf(f[i]);
+    }
+    st_shared_v4(dst_row + ((static_cast<uint32_t>(j) ^ row_xor) << 4), pack_bf16x2(f[0], f[1]), pack_bf16x2(f[2], f[3]),
+                 pack_bf16x2(f[4], f[5]), pack_bf16x2(f[6], f[7]));
+  }
+}
 #endif  // __CUDACC__
 
 // ------------------------------------------------------------------------------------------
