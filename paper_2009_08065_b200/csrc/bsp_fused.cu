@@ -379,8 +379,29 @@ extern "C" int bsp_prepare_batched(const bsp_layer_job* jobs, int n_jobs, int bl
                      u.kept_weights, static_cast<uint16_t*>(u.plan)};
   }
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  int st = fused_stage1(fj, n_jobs, block, eps, pen == BSP_PEN_L2SQ ? 1 : 0, s);
-  if (st == BSP_OK) st = fused_stage2(fj, n_jobs, block, s);
+  // Small batches (all CTAs resident at once) take the one-launch path; its per-part counts and
+  // penalty partials live in the workspace's S region, which this call does not use otherwise.
+  int st = BSP_OK;
+  bool done = false;
+  if (n_jobs <= 16) {
+    int32_t* pcounts[16];
+    double* ppartial[16];
+    for (int i = 0; i < n_jobs; ++i) {
+      const bsp_layer_job& u = jobs[i];
+      const int nb = u.rows / block;
+      const WsLayout L = ws_layout(nb, u.cols);
+      char* region = static_cast<char*>(u.ws) + L.sumsq_off;          // 4 bytes per group
+      const size_t slots = static_cast<size_t>(nb) * 32;              // at most 32 parts per block
+      pcounts[i] = reinterpret_cast<int32_t*>(region);
+      ppartial[i] = reinterpret_cast<double*>(region + round_up(slots * sizeof(int32_t), 256));
+      if (round_up(slots * 4, 256) + slots * 8 > static_cast<size_t>(nb) * u.cols * 4) { pcounts[0] = nullptr; break; }
+    }
+    if (pcounts[0] != nullptr) st = fused_onepass(fj, n_jobs, block, eps, pen == BSP_PEN_L2SQ ? 1 : 0, pcounts, ppartial, s, &done);
+  }
+  if (st == BSP_OK && !done) {
+    st = fused_stage1(fj, n_jobs, block, eps, pen == BSP_PEN_L2SQ ? 1 : 0, s);
+    if (st == BSP_OK) st = fused_stage2(fj, n_jobs, block, s);
+  }
   delete[] fj;
   return st;
 }
