@@ -398,7 +398,12 @@ def run_cuda(args):
             "roofline": {
                 "kernel": "linear_tc_kernel (bsp_linear_planned), the four launches of a step",
                 "bound": "tensor", "achieved": round(achieved, 2), "peak": peak, "unit": "TFLOP/s",
-                "frac": round(achieved / peak, 4), "traffic": None,
+                "frac": round(achieved / peak, 4),
+                # dram__bytes_read.sum + dram__bytes_write.sum of the four launches, one ncu capture each
+                # (profiles/linear_tc_kernel_bert_base_T4096.md); Y is still in L2 when each kernel ends
+                "traffic": 58.35e6, "algorithmic_bytes": sum(
+                    2 * wl.tokens * sp.k_in + 2 * sp.n_out * sp.k_in + 2 * wl.tokens * sp.n_out + 2 * sp.n_out
+                    for sp in wl.linears),
                 "peak_source": f"bf16_tflops burst, {peak_src}",
                 "per_launch": {e["spec"].name.split(".")[1]: {
                     "ms": round(gemm_mean_ms[i], 5), "nonzero_tflops": round(flops[i] / gemm_mean_ms[i] / 1e9, 1)}
