@@ -72,10 +72,15 @@ def _grouped(a: np.ndarray, block: int, orient: str) -> np.ndarray:
 # ---------------------------------------------------------------------------
 # group norms, gamma, penalty  (Section 3.2)
 # ---------------------------------------------------------------------------
+def group_sumsq_values(w: np.ndarray, block: int, orient: str) -> np.ndarray:
+    """S_g for a matrix given as float64 values (used for bf16 inputs and by the gradient pins)."""
+    g = _grouped(np.asarray(w, dtype=np.float64), block, orient)
+    return (g * g).sum(axis=-1)
+
+
 def group_sumsq(w_bits: np.ndarray, block: int, orient: str) -> np.ndarray:
     """S_g = sum of squares of the group's weights (the quantity under the root in Eq. 2 / Eq. 3)."""
-    g = _grouped(bf16_to_f64(w_bits), block, orient)
-    return (g * g).sum(axis=-1)
+    return group_sumsq_values(bf16_to_f64(w_bits), block, orient)
 
 
 def group_norms(w_bits: np.ndarray, block: int, orient: str) -> np.ndarray:
@@ -112,6 +117,29 @@ def penalty_l2sq(sumsq: np.ndarray, alpha: Optional[np.ndarray]) -> float:
     if alpha is None:
         return float(sumsq.sum())
     return float((alpha * sumsq).sum())
+
+
+def penalty_grad_values(w: np.ndarray, block: int, orient: str, gamma: np.ndarray, squared: bool = False) -> np.ndarray:
+    """Gradient with respect to W of the regulariser with the penalty weights held fixed, as
+    Algorithm 2 holds gamma between milestones while Adam minimises `mixed_loss`.
+
+    Eq. 2 / Eq. 3 form:  d/dW_e [ gamma_g ||W_g||_2 ] = gamma_g * W_e / ||W_g||_2   (0 for an all-zero group,
+    the minimum-norm subgradient).  Squared-norm variant:  d/dW_e [ alpha_g ||W_g||^2 ] = 2 alpha_g W_e.
+    w: float64 values [rows, cols]; gamma: per-group array; result [rows, cols], without the factor lambda.
+    """
+    w = np.asarray(w, dtype=np.float64)
+    full_gamma = _expand(np.asarray(gamma, dtype=np.float64), block, orient)
+    if squared:
+        return 2.0 * full_gamma * w
+    n = _expand(np.sqrt(group_sumsq_values(w, block, orient)), block, orient)
+    with np.errstate(divide="ignore", invalid="ignore"):
+        g = np.where(n > 0, full_gamma * w / n, 0.0)
+    return g
+
+
+def penalty_grad(w_bits: np.ndarray, block: int, orient: str, gamma: np.ndarray, squared: bool = False) -> np.ndarray:
+    """`penalty_grad_values` on bf16 weights."""
+    return penalty_grad_values(bf16_to_f64(w_bits), block, orient, gamma, squared)
 
 
 # ---------------------------------------------------------------------------

@@ -143,6 +143,35 @@ def test_stale_gamma_differs_from_fresh():
     assert abs(O.penalty_l2(n_new, stale) - O.penalty_l2(n_new, O.gamma_update(n_new, 1e-3))) > 1e-3
 
 
+@pytest.mark.parametrize("orient,block,squared", [("C", 3, False), ("R", 4, False), ("C", 2, True), ("R", 3, True)])
+def test_penalty_gradient_against_finite_differences(orient, block, squared):
+    """Central differences of the penalty value (gamma fixed) reproduce the analytic gradient."""
+    g = si.stream(17, 3)
+    w = g.standard_normal((6, 12)) * 0.5
+    shape = (6 // block, 12) if orient == "C" else (6, 12 // block)
+    gamma = g.uniform(0.5, 2.0, size=shape)
+
+    def value(x):
+        s = O.group_sumsq_values(x, block, orient)
+        return O.penalty_l2sq(s, gamma) if squared else O.penalty_l2(np.sqrt(s), gamma)
+
+    grad = O.penalty_grad_values(w, block, orient, gamma, squared)
+    h = 1e-6
+    for i, j in [(0, 0), (1, 5), (5, 11), (3, 7), (2, 2)]:
+        e = np.zeros_like(w)
+        e[i, j] = h
+        fd = (value(w + e) - value(w - e)) / (2 * h)
+        assert grad[i, j] == pytest.approx(fd, rel=1e-6, abs=1e-9)
+    # closed forms: a group (3, 4) with gamma 2 -> 2 * (0.6, 0.8); an all-zero group -> 0
+    wz = np.zeros((2, 2))
+    wz[:, 0] = [3.0, 4.0]
+    gz = O.penalty_grad_values(wz, 2, "C", np.array([[2.0, 5.0]]))
+    assert np.allclose(gz, [[1.2, 0.0], [1.6, 0.0]], rtol=1e-15, atol=0)
+    assert np.array_equal(O.penalty_grad_values(wz, 2, "C", np.array([[2.0, 5.0]]), squared=True), [[12.0, 0.0], [16.0, 0.0]])
+    # Euler: <W, grad> = penalty for the norm form (degree-1 homogeneous), 2 * penalty for the squared form
+    assert (w * grad).sum() == pytest.approx((2.0 if squared else 1.0) * value(w), rel=1e-12)
+
+
 # ----------------------------------------------------------------------------- decision quantity
 def test_decision_sumsq32_is_sequential_float32():
     """A case where summation order matters in float32: 1 + 2^-24 + 2^-24 taken left to right stays 1."""
