@@ -84,6 +84,21 @@ int bsp_group_norms(const void* W, int rows, int cols, int ldw, int block, int o
                     void* stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * bsp_penalty_grad — the regulariser's gradient with respect to W with the penalty weights held
+ * fixed, which is what Algorithm 2's inner loop needs between two gamma updates ("Update model
+ * weight W to minimize mixed_loss using Adam", mixed_loss = l1loss + f(W, b)):
+ *   BSP_PEN_L2   (Eq. 2 / Eq. 3):  G_e = scale * gamma_g * W_e / ||W_g||_2   (0 for an all-zero group)
+ *   BSP_PEN_L2SQ (squared norms):  G_e = scale * 2 * alpha_g * W_e
+ * gamma: float32 per-group array (shape by orientation) from an earlier bsp_group_norms call;
+ * scale: the factor lambda; grad: float32 [rows, cols] with leading dimension ldg, overwritten,
+ * or added to if accumulate != 0 (so that it can be summed onto the task gradient).
+ * Errors: BSP_ERR_ARG, BSP_ERR_SHAPE.
+ */
+int bsp_penalty_grad(const void* W, int rows, int cols, int ldw, int block, int orient, int pen,
+                     const float* gamma, float scale, float* grad, int ldg, int accumulate,
+                     void* stream);
+
+/* ---------------------------------------------------------------------------------------------
  * bsp_pack_bound — host-only size query for bsp_prune_pack (worst case: nothing pruned).
  *   *idx_elems = number of int32 index entries, *val_elems = number of bf16 values,
  *   *ws_bytes  = workspace bytes bsp_prune_pack / bsp_percentile_threshold need for this shape.
@@ -227,6 +242,14 @@ int bsp_prepare_batched(const bsp_layer_job* jobs, int n_jobs, int block, float 
 int bsp_linear_plan_bytes(int n_out, int k_in, int block, size_t* bytes);
 int bsp_linear_plan(const int32_t* blk_ptr, const int32_t* idx, const void* vals,
                     int n_out, int k_in, int block, void* plan, size_t plan_bytes, void* stream);
+/* bsp_linear_plan_r — the execution layout from the orientation-R packed form (Algorithm 1's own
+ * geometry: strips of `block` columns, kept row segments; idx holds row indices, tiles are
+ * [kc, block]).  n_out = rows of W, k_in = cols; plan_bytes >= n_out * k_in * 2 rounded up to 256.
+ * The resulting plan feeds bsp_linear_planned / bsp_linear_chain like any other (their `block`
+ * argument is then only checked to divide n_out: pass 1).
+ * Errors: BSP_ERR_ARG, BSP_ERR_SHAPE (block does not divide k_in), BSP_ERR_WORKSPACE. */
+int bsp_linear_plan_r(const int32_t* blk_ptr, const int32_t* row_idx, const void* vals,
+                      int n_out, int k_in, int block, void* plan, size_t plan_bytes, void* stream);
 int bsp_linear_planned(const void* plan, int n_out, int k_in, int block,
                        const void* X, int tokens, int ldx, const void* bias, int act,
                        void* Y, int ldy, void* stream);

@@ -71,6 +71,7 @@ _SIGNATURES = {
     "bsp_status_string": (ctypes.c_char_p, [_i]),
     "bsp_last_cuda_error": (_i, []),
     "bsp_group_norms": (_i, [_vp, _i, _i, _i, _i, _i, _f, _i, _vp, _vp, _vp, _vp, _vp]),
+    "bsp_penalty_grad": (_i, [_vp, _i, _i, _i, _i, _i, _i, _vp, _f, _vp, _i, _i, _vp]),
     "bsp_pack_bound": (_i, [_i, _i, _i, _i, _szp, _szp, _szp]),
     "bsp_prune_pack": (_i, [_vp, _i, _i, _i, _i, _i, _f, _vp, _i, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "bsp_prune_pack_static": (_i, [_vp, _i, _i, _i, _i, _i, _f, _vp, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
@@ -79,6 +80,7 @@ _SIGNATURES = {
     "bsp_prepare_batched": (_i, [ctypes.POINTER(_LayerJob), _i, _i, _f, _i, _vp]),
     "bsp_linear_plan_bytes": (_i, [_i, _i, _i, _szp]),
     "bsp_linear_plan": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _sz, _vp]),
+    "bsp_linear_plan_r": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _sz, _vp]),
     "bsp_linear_planned": (_i, [_vp, _i, _i, _i, _vp, _i, _i, _vp, _i, _vp, _i, _vp]),
     "bsp_linear_planned_ex": (_i, [_vp, _i, _i, _i, _vp, _i, _i, _vp, _i, _vp, _i, _i, _vp]),
     "bsp_linear": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _i, _i, _vp, _i, _vp, _i, _vp, _sz, _vp]),
@@ -136,6 +138,14 @@ def bsp_group_norms(W: torch.Tensor, block: int, orient: int = ORIENT_C, eps: fl
     rows, cols = W.shape
     _check(lib.bsp_group_norms(_ptr(W), rows, cols, _ld(W), block, orient, eps, pen, _ptr(norms), _ptr(gamma_in),
                                _ptr(gamma_out), _ptr(penalty), _stream(stream)), "bsp_group_norms")
+
+
+def bsp_penalty_grad(W: torch.Tensor, block: int, orient: int, pen: int, gamma: torch.Tensor, scale: float,
+                     grad: torch.Tensor, accumulate: bool = False, stream=None) -> None:
+    """grad: float32 [rows, cols]; gamma: float32 per-group tensor."""
+    rows, cols = W.shape
+    _check(lib.bsp_penalty_grad(_ptr(W), rows, cols, _ld(W), block, orient, pen, _ptr(gamma), scale, _ptr(grad),
+                                _ld(grad), int(accumulate), _stream(stream)), "bsp_penalty_grad")
 
 
 def bsp_pack_bound(rows: int, cols: int, block: int, orient: int = ORIENT_C) -> Tuple[int, int, int]:
@@ -250,6 +260,12 @@ def bsp_linear_plan_bytes(n_out: int, k_in: int, block: int) -> int:
 
 
 def bsp_linear_plan(packed: PackedMatrix, plan: torch.Tensor, stream=None) -> None:
+    """Execution layout of a packed matrix of either orientation."""
+    if packed.orient == ORIENT_R:
+        _check(lib.bsp_linear_plan_r(_ptr(packed.blk_ptr), _ptr(packed.idx), _ptr(packed.vals), packed.rows, packed.cols,
+                                     packed.block, _ptr(plan), plan.numel() * plan.element_size(), _stream(stream)),
+               "bsp_linear_plan_r")
+        return
     _check(lib.bsp_linear_plan(_ptr(packed.blk_ptr), _ptr(packed.idx), _ptr(packed.vals), packed.rows, packed.cols,
                                packed.block, _ptr(plan), plan.numel() * plan.element_size(), _stream(stream)),
            "bsp_linear_plan")

@@ -263,6 +263,20 @@ plan_expand_kernel(const int32_t* __restrict__ blk_ptr, const int32_t* __restric
   }
 }
 
+// Plan from the orientation-R packed form (vertical strips of h columns, kept ROWS per strip,
+// tiles [kc][h]): every kept row segment goes back to its place; the plan is zeroed beforehand.
+__global__ void __launch_bounds__(256)
+plan_expand_r_kernel(const int32_t* __restrict__ blk_ptr, const int32_t* __restrict__ row_idx,
+                     const uint16_t* __restrict__ vals, int k_in, int h, uint16_t* __restrict__ Wx) {
+  const int a = blockIdx.x;                       // strip
+  const int lo = blk_ptr[a], kc = blk_ptr[a + 1] - lo;
+  const uint16_t* tile = vals + static_cast<size_t>(h) * lo;
+  for (int e = threadIdx.x; e < kc * h; e += blockDim.x) {
+    const int p = e / h, c = e - p * h;
+    Wx[static_cast<size_t>(row_idx[lo + p]) * k_in + static_cast<size_t>(a) * h + c] = tile[e];
+  }
+}
+
 // ------------------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------------------
@@ -361,6 +375,23 @@ extern "C" int bsp_linear_plan(const int32_t* blk_ptr, const int32_t* idx, const
   const int splits = block >= 4 ? 4 : 1;
   plan_expand_kernel<<<dim3(n_out / block, splits), 256, sizeof(int16_t) * k_in, static_cast<cudaStream_t>(stream)>>>(
       blk_ptr, idx, static_cast<const uint16_t*>(vals), k_in, block, static_cast<uint16_t*>(plan));
+  BSP_LAUNCH_CHECK();
+  return BSP_OK;
+}
+
+extern "C" int bsp_linear_plan_r(const int32_t* blk_ptr, const int32_t* row_idx, const void* vals, int n_out,
+                                 int k_in, int block, void* plan, size_t plan_bytes, void* stream) {
+  using namespace bsp;
+  if (blk_ptr == nullptr || row_idx == nullptr || vals == nullptr || plan == nullptr) return BSP_ERR_ARG;
+  if (n_out <= 0 || k_in <= 0 || block <= 0) return BSP_ERR_ARG;
+  if (k_in % block) return BSP_ERR_SHAPE;
+  if (!aligned_to(plan, 256)) return BSP_ERR_ARG;
+  const size_t need = round_up(static_cast<size_t>(n_out) * k_in * 2, 256);
+  if (plan_bytes < need) return BSP_ERR_WORKSPACE;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  BSP_CUDA_TRY(cudaMemsetAsync(plan, 0, static_cast<size_t>(n_out) * k_in * 2, s));
+  plan_expand_r_kernel<<<k_in / block, 256, 0, s>>>(blk_ptr, row_idx, static_cast<const uint16_t*>(vals), k_in, block,
+                                                   static_cast<uint16_t*>(plan));
   BSP_LAUNCH_CHECK();
   return BSP_OK;
 }

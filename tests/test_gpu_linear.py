@@ -186,3 +186,28 @@ def test_cta_pair_kernel_matches_one_cta_kernel_and_oracle(T, N, K, act):
     if T <= 1024:
         y_ref, scales = oracle_linear(x, wp, b, act)
         assert_linear_close(bits_of(ys[1]), y_ref, scales, "pair")
+
+
+@pytest.mark.parametrize("h,rate", [(3, 2.0), (12, 1.428), (16, 5.0), (96, 2.0)])
+def test_linear_on_row_pruned_strips(h, rate):
+    """Algorithm 1's own geometry (orientation R): strips of h columns, row segments pruned by threshold.
+    The packed form is expanded to the execution layout by bsp_linear_plan_r; the layer then matches the
+    masked dense product."""
+    T, N, K = 200, 384, 768
+    spec = si.LinearSpec(f"rlin{h}", N, K, True, rate, h)
+    w = si.make_weight(15, spec, "student_t3")
+    b = si.make_bias(15, spec)
+    x = si.make_activations(15, spec.name, T, K)
+    t_b = O.percentile_threshold(w, h, "R", rate)
+    wp = O.prune(w, h, "R", t_b)
+    pk = bsp.PackedMatrix.allocate(N, K, h, bsp.ORIENT_R, DEV)
+    bsp.bsp_prune_pack(to_dev(w), pk, t_b)
+    plan = torch.full((bsp.bsp_linear_plan_bytes(N, K, 1),), 0x5A, dtype=torch.uint8, device=DEV)
+    bsp.bsp_linear_plan(pk, plan)
+    torch.cuda.synchronize()
+    assert np.array_equal(bits_of(plan.view(torch.int16)[: N * K].reshape(N, K)), wp)      # W * Mask, bit for bit
+    y = torch.full((T, N), 0x7FC0, dtype=torch.int16, device=DEV)
+    bsp.bsp_linear_planned(plan, N, K, 1, to_dev(x), to_dev(b), 1, y)
+    bsp.bsp_linear_status()
+    y_ref, scales = oracle_linear(x, wp, b, 1)
+    assert_linear_close(bits_of(y), y_ref, scales, f"orientation R, h={h}")

@@ -260,3 +260,31 @@ def test_prepare_batched_optional_outputs_and_many_jobs():
     with pytest.raises(bsp.BspError) as e:
         bsp.bsp_prepare_batched([jobs[0], bsp.LayerJob(W=to_dev(odd), out=pk)], 8)
     assert e.value.status == -6
+
+
+# ---------------------------------------------------------------------------------------- penalty gradient
+@pytest.mark.parametrize("orient,block,shape", [(0, 16, (768, 768)), (0, 3, (96, 50)), (1, 12, (96, 768)), (1, 5, (33, 50))])
+def test_penalty_gradient(orient, block, shape):
+    """G = lambda * gamma_g * W / ||W_g|| (and the squared-norm variant), gamma fixed; relative 1e-5 in float32."""
+    o = "CR"[orient]
+    rows, cols = shape
+    spec = si.LinearSpec("pg", rows, cols, False, 2.0, block)
+    wp, _ = si.make_pruned_weight(19, spec, orient=o)                  # half of the groups are all-zero
+    gshape = (rows // block, cols) if orient == 0 else (rows, cols // block)
+    gamma = O.gamma_update(O.group_norms(si.make_weight(20, spec), block, o), 1e-3).astype(np.float32)
+    assert gamma.shape == gshape
+    lam = 3e-4                                                          # a penalty factor from the paper's range
+    wd, gd = to_dev(wp), torch.from_numpy(gamma).to(DEV)
+    for pen, squared in ((bsp.PEN_L2, False), (bsp.PEN_L2SQ, True)):
+        ref = lam * O.penalty_grad(wp, block, o, gamma.astype(np.float64), squared)
+        grad = torch.full((rows, cols), 7.0, dtype=torch.float32, device=DEV)
+        bsp.bsp_penalty_grad(wd, block, orient, pen, gd, lam, grad)
+        torch.cuda.synchronize()
+        assert np.allclose(grad.cpu().numpy(), ref, rtol=REL, atol=1e-12)
+        assert (ref[~O.mask_of(wp)] == 0).all() and (grad.cpu().numpy()[~O.mask_of(wp)] == 0).all()
+        # accumulate onto an existing gradient
+        base = torch.from_numpy(si.bf16_bits_to_f32(si.normal_bf16(21, "tg", (rows, cols), 1e-3))).to(DEV)
+        acc = base.clone()
+        bsp.bsp_penalty_grad(wd, block, orient, pen, gd, lam, acc, accumulate=True)
+        torch.cuda.synchronize()
+        assert np.allclose(acc.cpu().numpy(), base.cpu().numpy().astype(np.float64) + ref, rtol=REL, atol=1e-9)
