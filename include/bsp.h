@@ -250,6 +250,14 @@ int bsp_linear_plan(const int32_t* blk_ptr, const int32_t* idx, const void* vals
  * Errors: BSP_ERR_ARG, BSP_ERR_SHAPE (block does not divide k_in), BSP_ERR_WORKSPACE. */
 int bsp_linear_plan_r(const int32_t* blk_ptr, const int32_t* row_idx, const void* vals,
                       int n_out, int k_in, int block, void* plan, size_t plan_bytes, void* stream);
+/* bsp_linear_plan_t — the TRANSPOSED execution layout PT[k, n] = (W * Mask)[n, k] from the
+ * orientation-C packed form.  It is the operand of the backward product with respect to the
+ * activations of the masked layer that Algorithm 2 retrains (W = W * Mask):
+ *   dX = dY (W * Mask)  =  bsp_linear_planned(plan_t, n_out := k_in, k_in := n_out, block := 1,
+ *                                             X := dY [tokens, n_out], bias := NULL, act := none, Y := dX).
+ * plan_bytes as bsp_linear_plan_bytes(n_out, k_in, block).  Errors as bsp_linear_plan. */
+int bsp_linear_plan_t(const int32_t* blk_ptr, const int32_t* idx, const void* vals,
+                      int n_out, int k_in, int block, void* plan_t, size_t plan_bytes, void* stream);
 int bsp_linear_planned(const void* plan, int n_out, int k_in, int block,
                        const void* X, int tokens, int ldx, const void* bias, int act,
                        void* Y, int ldy, void* stream);

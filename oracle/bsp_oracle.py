@@ -375,6 +375,12 @@ def linear_from_packed(x_bits: np.ndarray, blk_ptr: np.ndarray, idx: np.ndarray,
     return gelu(y) if act == 1 else y
 
 
+def linear_backward_input(dy_bits: np.ndarray, w_bits: np.ndarray, mask: np.ndarray) -> np.ndarray:
+    """dX[t, k] = sum_n dY[t, n] * (W[n, k] * Mask[n, k]): the gradient of the masked layer of Algorithm 2's
+    retraining loop (W = W * Mask) with respect to its input, float64."""
+    return bf16_to_f64(dy_bits) @ (bf16_to_f64(w_bits) * mask)
+
+
 def row_scales(x_bits: np.ndarray, w_bits: np.ndarray, mask: np.ndarray,
                bias_bits: Optional[np.ndarray]) -> np.ndarray:
     """||X[t,:]||_2 * ||(W*Mask)[n,:]||_2 + |b[n]|: the magnitude an output's error is judged against."""

@@ -81,6 +81,7 @@ _SIGNATURES = {
     "bsp_linear_plan_bytes": (_i, [_i, _i, _i, _szp]),
     "bsp_linear_plan": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _sz, _vp]),
     "bsp_linear_plan_r": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _sz, _vp]),
+    "bsp_linear_plan_t": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _sz, _vp]),
     "bsp_linear_planned": (_i, [_vp, _i, _i, _i, _vp, _i, _i, _vp, _i, _vp, _i, _vp]),
     "bsp_linear_planned_ex": (_i, [_vp, _i, _i, _i, _vp, _i, _i, _vp, _i, _vp, _i, _i, _vp]),
     "bsp_linear": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _i, _i, _vp, _i, _vp, _i, _vp, _sz, _vp]),
@@ -269,6 +270,13 @@ def bsp_linear_plan(packed: PackedMatrix, plan: torch.Tensor, stream=None) -> No
     _check(lib.bsp_linear_plan(_ptr(packed.blk_ptr), _ptr(packed.idx), _ptr(packed.vals), packed.rows, packed.cols,
                                packed.block, _ptr(plan), plan.numel() * plan.element_size(), _stream(stream)),
            "bsp_linear_plan")
+
+
+def bsp_linear_plan_t(packed: PackedMatrix, plan_t: torch.Tensor, stream=None) -> None:
+    """Transposed execution layout (orientation C): the operand of dX = dY (W * Mask)."""
+    _check(lib.bsp_linear_plan_t(_ptr(packed.blk_ptr), _ptr(packed.idx), _ptr(packed.vals), packed.rows, packed.cols,
+                                 packed.block, _ptr(plan_t), plan_t.numel() * plan_t.element_size(), _stream(stream)),
+           "bsp_linear_plan_t")
 
 
 def bsp_linear_planned(plan: torch.Tensor, n_out: int, k_in: int, block: int, X: torch.Tensor,

@@ -277,6 +277,21 @@ plan_expand_r_kernel(const int32_t* __restrict__ blk_ptr, const int32_t* __restr
   }
 }
 
+// Transposed plan from the orientation-C packed form: PT[k, n] = (W * Mask)[n, k], for the product
+// dX = dY (W * Mask).  One CTA per row-block; consecutive threads take consecutive rows r of the
+// block, so the 2-byte stores of one kept column are contiguous.  The plan is zeroed beforehand.
+__global__ void __launch_bounds__(256)
+plan_expand_t_kernel(const int32_t* __restrict__ blk_ptr, const int32_t* __restrict__ idx,
+                     const uint16_t* __restrict__ vals, int n_out, int block, uint16_t* __restrict__ PT) {
+  const int b = blockIdx.x;
+  const int lo = blk_ptr[b], kc = blk_ptr[b + 1] - lo;
+  const uint16_t* tile = vals + static_cast<size_t>(block) * lo;
+  for (int e = threadIdx.x; e < kc * block; e += blockDim.x) {
+    const int j = e / block, r = e - j * block;
+    PT[static_cast<size_t>(idx[lo + j]) * n_out + static_cast<size_t>(b) * block + r] = tile[static_cast<size_t>(r) * kc + j];
+  }
+}
+
 // ------------------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------------------
@@ -392,6 +407,23 @@ extern "C" int bsp_linear_plan_r(const int32_t* blk_ptr, const int32_t* row_idx,
   BSP_CUDA_TRY(cudaMemsetAsync(plan, 0, static_cast<size_t>(n_out) * k_in * 2, s));
   plan_expand_r_kernel<<<k_in / block, 256, 0, s>>>(blk_ptr, row_idx, static_cast<const uint16_t*>(vals), k_in, block,
                                                    static_cast<uint16_t*>(plan));
+  BSP_LAUNCH_CHECK();
+  return BSP_OK;
+}
+
+extern "C" int bsp_linear_plan_t(const int32_t* blk_ptr, const int32_t* idx, const void* vals, int n_out, int k_in,
+                                 int block, void* plan_t, size_t plan_bytes, void* stream) {
+  using namespace bsp;
+  if (blk_ptr == nullptr || idx == nullptr || vals == nullptr || plan_t == nullptr) return BSP_ERR_ARG;
+  size_t need;
+  int st = bsp_linear_plan_bytes(n_out, k_in, block, &need);
+  if (st != BSP_OK) return st;
+  if (!aligned_to(plan_t, 256)) return BSP_ERR_ARG;
+  if (plan_bytes < need) return BSP_ERR_WORKSPACE;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  BSP_CUDA_TRY(cudaMemsetAsync(plan_t, 0, static_cast<size_t>(n_out) * k_in * 2, s));
+  plan_expand_t_kernel<<<n_out / block, 256, 0, s>>>(blk_ptr, idx, static_cast<const uint16_t*>(vals), n_out, block,
+                                                     static_cast<uint16_t*>(plan_t));
   BSP_LAUNCH_CHECK();
   return BSP_OK;
 }

@@ -211,3 +211,24 @@ def test_linear_on_row_pruned_strips(h, rate):
     bsp.bsp_linear_status()
     y_ref, scales = oracle_linear(x, wp, b, 1)
     assert_linear_close(bits_of(y), y_ref, scales, f"orientation R, h={h}")
+
+
+def test_backward_with_respect_to_activations():
+    """dX = dY (W * Mask) through the transposed plan and the same tensor-core kernel."""
+    T, N, K, d = 640, 768, 384, 16
+    spec = si.LinearSpec("bwd", N, K, False, 3.0, d)
+    wp, keep = si.make_pruned_weight(16, spec)
+    dy = si.make_activations(16, "bwd.dy", T, N)
+    pk = gpu_pack(wp, d)
+    plan_t = torch.full((bsp.bsp_linear_plan_bytes(N, K, d),), 0x33, dtype=torch.uint8, device=DEV)
+    bsp.bsp_linear_plan_t(pk, plan_t)
+    torch.cuda.synchronize()
+    assert np.array_equal(bits_of(plan_t.view(torch.int16)[: N * K].reshape(K, N)), np.ascontiguousarray(wp.T))
+    dx = torch.full((T, K), 0x7FC0, dtype=torch.int16, device=DEV)
+    bsp.bsp_linear_planned(plan_t, K, N, 1, to_dev(dy), None, 0, dx)
+    bsp.bsp_linear_status()
+    m = O.mask_of(wp)
+    ref = O.linear_backward_input(dy, wp, m)
+    # error scale: ||dY[t, :]|| * ||(W * Mask)[:, k]||
+    scales = np.sqrt((O.bf16_to_f64(dy) ** 2).sum(1))[:, None] * np.sqrt(((O.bf16_to_f64(wp) * m) ** 2).sum(0))[None, :]
+    assert_linear_close(bits_of(dx), ref, np.maximum(scales, 1e-30), "dX")

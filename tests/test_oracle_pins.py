@@ -451,3 +451,21 @@ def test_row_scales():
     m = np.array([[True, True], [True, False]])
     s = O.row_scales(x, w, m, b)
     assert s.tolist() == [[5.0 * 1.0 + 0.25, 5.0 * 0.5 + 2.0]]
+
+
+def test_backward_input_is_the_adjoint_of_the_forward_layer():
+    """<dY, X W^T> == <dY W, X> for the masked weight: pins the backward product to the forward one."""
+    T, N, K, d = 6, 12, 16, 4
+    spec = si.LinearSpec("adj", N, K, False, 2.0, d)
+    wp, keep = si.make_pruned_weight(41, spec)
+    x = si.make_activations(41, "adj", T, K)
+    dy = si.make_activations(42, "adj.dy", T, N)
+    m = O.mask_of(wp)
+    y = O.linear_masked_dense(x, wp, m, None, 0)
+    dx = O.linear_backward_input(dy, wp, m)
+    assert (O.bf16_to_f64(dy) * y).sum() == pytest.approx((dx * O.bf16_to_f64(x)).sum(), rel=1e-13)
+    # a pruned column of a row-block passes no gradient from that block's outputs
+    dy1 = np.zeros_like(dy)
+    dy1[:, :d] = dy[:, :d]                      # only row-block 0's outputs carry gradient
+    dx1 = O.linear_backward_input(dy1, wp, m)
+    assert (dx1[:, ~keep[0]] == 0).all() and (dx1[:, keep[0]] != 0).any()
