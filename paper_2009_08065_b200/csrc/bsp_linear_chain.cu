@@ -77,7 +77,7 @@ linear_chain_kernel(const __grid_constant__ ChainMaps M, const __grid_constant__
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
   // [S operand stages][2 epilogue staging buffers][bias, bf16, for two tiles][mbarriers, TMEM base]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S * Cfg::kStage + 2 * kEpiStage + 2 * kBN * 2);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S * Cfg::kStage + kEpiBytes + 2 * kBN * 2);
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 2 * S + 4);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -173,10 +173,11 @@ linear_chain_kernel(const __grid_constant__ ChainMaps M, const __grid_constant__
     const int row = quad * 32 + lane;
     const int epi_tid = threadIdx.x - 64;
     const bool issuer = (epi_tid & 127) == 0;
-    const uint32_t buf = smem_base + S * Cfg::kStage + group * kEpiStage;
-    uint16_t* s_bias = reinterpret_cast<uint16_t*>(smem + S * Cfg::kStage + 2 * kEpiStage);   // [2][256] bf16
-    const uint32_t row_off = static_cast<uint32_t>(row) * 128u;
-    const uint32_t row_xor = static_cast<uint32_t>(row & 7);
+    const uint32_t buf0 = smem_base + S * Cfg::kStage + group * 2 * kEpiStage;   // this group's two staging buffers
+    uint32_t my_piece = 0;                   // pieces staged by this group so far: selects the buffer
+    uint16_t* s_bias = reinterpret_cast<uint16_t*>(smem + S * Cfg::kStage + kEpiBytes);   // [2][256] bf16
+    const uint32_t row_off = static_cast<uint32_t>(row) * 64u;
+    const uint32_t row_xor = static_cast<uint32_t>((row >> 1) & 3);
     uint32_t acc_phase[2] = {0u, 0u};
     int acc = 0;
     bool ok = true;
@@ -195,7 +196,9 @@ linear_chain_kernel(const __grid_constant__ ChainMaps M, const __grid_constant__
 #pragma unroll 1
       for (int pc = group; pc < pieces; pc += 2) {
         const int c0 = pc * kEpiCols;
-        if (issuer) tma_store_wait_read<0>();
+        const uint32_t buf = buf0 + (my_piece & 1u) * kEpiStage;
+        ++my_piece;
+        if (issuer) tma_store_wait_read<1>();   // the store issued two pieces ago has read this buffer
         group_sync(group);
         EpiloguePiece piece;
         piece_load(taddr + c0, smem_u32(s_bias + acc * kBN + c0), piece);
@@ -284,7 +287,7 @@ extern "C" int bsp_linear_chain(const bsp_chain_op* ops, int n_ops, const void* 
     const uint16_t* src_base = static_cast<const uint16_t*>(src) + u.src_col;
     if (!make_map(&M.x[i], src_base, u.k_in, tokens, src_ld, kBlockM)) return BSP_ERR_CUDA;
     if (!make_map(&M.w[i], u.plan, u.k_in, u.n_out, u.k_in, kBN)) return BSP_ERR_CUDA;
-    if (!make_map(&M.y[i], u.Y, u.n_out, tokens, u.ldy, kBlockM)) return BSP_ERR_CUDA;
+    if (!make_map(&M.y[i], u.Y, u.n_out, tokens, u.ldy, kBlockM, kEpiCols)) return BSP_ERR_CUDA;
     ChainOp& o = P.op[i];
     o.n_out = u.n_out;
     o.k_blocks = (u.k_in + kBlockK - 1) / kBlockK;

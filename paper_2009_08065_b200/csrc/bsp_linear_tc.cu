@@ -15,11 +15,11 @@
 //                      (128-byte swizzle), completion on an mbarrier;
 //   warp 1 (one lane): issues tcgen05.mma (M=128, N=BN, K=16) into one of two TMEM accumulators
 //                      and commits stage release / accumulator ready to mbarriers;
-//   warps 2..9       : epilogue, two groups of four warps; group g takes the 64-column pieces of
+//   warps 2..9       : epilogue, two groups of four warps; group g takes the 32-column pieces of
 //                      the tile with index = g (mod 2).  Each warp tcgen05.ld's its 32 TMEM lanes
 //                      (= 32 tokens), adds bias, optional GELU, rounds to bf16, writes its rows
 //                      into the group's swizzled staging buffer, and one thread hands the
-//                      128 x 64 piece to a TMA store (full-line writes, tails clipped by the
+//                      128 x 32 piece to a TMA store (full-line writes, tails clipped by the
 //                      tensor map).  The epilogue runs concurrently with the next tile's main
 //                      loop on the other accumulator.
 // Every wait is bounded by a wall-clock deadline; on expiry the role records BSP_ERR_TIMEOUT in
@@ -57,7 +57,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
   // operand stages need 1024-byte alignment for the 128-byte swizzle pattern
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
   // [S operand stages][2 epilogue staging buffers][bias, bf16, for two tiles][mbarriers, TMEM base]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S * Cfg::kStage + 2 * kEpiStage + 2 * BN * 2);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S * Cfg::kStage + kEpiBytes + 2 * BN * 2);
   // bars[0..S) full, [S..2S) empty, [2S..2S+2) accumulator full, [2S+2..2S+4) accumulator empty
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 2 * S + 4);
 
@@ -165,10 +165,11 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     const int row = quad * 32 + lane;        // token row of this thread inside the tile
     const int epi_tid = threadIdx.x - 64;    // 0..255 among the epilogue threads
     const bool issuer = (epi_tid & 127) == 0;  // the thread of each group that owns its TMA stores
-    const uint32_t buf = smem_base + S * Cfg::kStage + group * kEpiStage;   // this group's staging buffer
-    uint16_t* s_bias = reinterpret_cast<uint16_t*>(smem + S * Cfg::kStage + 2 * kEpiStage);  // [2][BN] bf16
-    const uint32_t row_off = static_cast<uint32_t>(row) * 128u;
-    const uint32_t row_xor = static_cast<uint32_t>(row & 7);
+    const uint32_t buf0 = smem_base + S * Cfg::kStage + group * 2 * kEpiStage;   // this group's two staging buffers
+    uint32_t my_piece = 0;                   // pieces staged by this group so far: selects the buffer
+    uint16_t* s_bias = reinterpret_cast<uint16_t*>(smem + S * Cfg::kStage + kEpiBytes);  // [2][BN] bf16
+    const uint32_t row_off = static_cast<uint32_t>(row) * 64u;
+    const uint32_t row_xor = static_cast<uint32_t>((row >> 1) & 3);
     uint32_t acc_phase[2] = {0u, 0u};
     int acc = 0;
     bool ok = true;
@@ -188,7 +189,9 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
 #pragma unroll 1
       for (int pc = group; pc < pieces; pc += 2) {
         const int c0 = pc * kEpiCols;
-        if (issuer) tma_store_wait_read<0>();   // this group's previous store has read the staging buffer
+        const uint32_t buf = buf0 + (my_piece & 1u) * kEpiStage;
+        ++my_piece;
+        if (issuer) tma_store_wait_read<1>();   // the store issued two pieces ago has read this buffer
         group_sync(group);
         EpiloguePiece piece;
         piece_load(taddr + c0, smem_u32(s_bias + acc * BN + c0), piece);
@@ -320,7 +323,7 @@ int launch_tc(TcDevice* dev, int slot, const void* plan, const void* X, void* Y,
   CUtensorMap map_x, map_w, map_y;
   if (!make_map(&map_x, X, P.k_in, P.tokens, ldx, kBlockM)) return BSP_ERR_CUDA;
   if (!make_map(&map_w, plan, P.k_in, P.n_out, P.k_in, BN)) return BSP_ERR_CUDA;
-  if (!make_map(&map_y, Y, P.n_out, P.tokens, ldy, kBlockM)) return BSP_ERR_CUDA;
+  if (!make_map(&map_y, Y, P.n_out, P.tokens, ldy, kBlockM, kEpiCols)) return BSP_ERR_CUDA;
   if (!dev->attr_set[slot]) {
     BSP_CUDA_TRY(cudaFuncSetAttribute(linear_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes));
     dev->attr_set[slot] = true;

@@ -24,7 +24,7 @@ constexpr int kPairBN = 256;
 constexpr int kPairStageA = kBlockM * kBlockK * 2;         // this CTA's 128 rows of X
 constexpr int kPairStageB = (kPairBN / 2) * kBlockK * 2;   // this CTA's 128 of the 256 weight rows
 constexpr int kPairStage = kPairStageA + kPairStageB;
-constexpr int kPairFixed = 1024 + 2 * kEpiStage + 2 * kPairBN * 2 + 256;
+constexpr int kPairFixed = 1024 + kEpiBytes + 2 * kPairBN * 2 + 256;
 constexpr int kPairStages = (kSmemLimit - kPairFixed) / kPairStage > 8 ? 8 : (kSmemLimit - kPairFixed) / kPairStage;
 constexpr int kPairSmemBytes = kPairStages * kPairStage + kPairFixed;
 constexpr int kPairTmemCols = 512;
@@ -83,7 +83,7 @@ linear_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
   // [S operand stages][2 epilogue staging buffers][bias, bf16, for two tiles][mbarriers, TMEM base]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S * kPairStage + 2 * kEpiStage + 2 * kPairBN * 2);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S * kPairStage + kEpiBytes + 2 * kPairBN * 2);
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 2 * S + 4);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -183,10 +183,11 @@ linear_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
     const int row = quad * 32 + lane;
     const int epi_tid = threadIdx.x - 64;
     const bool issuer = (epi_tid & 127) == 0;
-    const uint32_t buf = smem_base + S * kPairStage + group * kEpiStage;
-    uint16_t* s_bias = reinterpret_cast<uint16_t*>(smem + S * kPairStage + 2 * kEpiStage);
-    const uint32_t row_off = static_cast<uint32_t>(row) * 128u;
-    const uint32_t row_xor = static_cast<uint32_t>(row & 7);
+    const uint32_t buf0 = smem_base + S * kPairStage + group * 2 * kEpiStage;   // this group's two staging buffers
+    uint32_t my_piece = 0;                   // pieces staged by this group so far: selects the buffer
+    uint16_t* s_bias = reinterpret_cast<uint16_t*>(smem + S * kPairStage + kEpiBytes);
+    const uint32_t row_off = static_cast<uint32_t>(row) * 64u;
+    const uint32_t row_xor = static_cast<uint32_t>((row >> 1) & 3);
     uint32_t acc_phase[2] = {0u, 0u};
     int acc = 0;
     bool ok = true;
@@ -204,7 +205,9 @@ linear_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
 #pragma unroll 1
       for (int pc = group; pc < pieces; pc += 2) {
         const int c0 = pc * kEpiCols;
-        if (issuer) tma_store_wait_read<0>();
+        const uint32_t buf = buf0 + (my_piece & 1u) * kEpiStage;
+        ++my_piece;
+        if (issuer) tma_store_wait_read<1>();   // the store issued two pieces ago has read this buffer
         group_sync(group);
         EpiloguePiece piece;
         piece_load(taddr + c0, smem_u32(s_bias + acc * kPairBN + c0), piece);
@@ -252,7 +255,7 @@ int launch_tc_pair(TcDevice* dev, const void* plan, const void* X, void* Y, int 
   CUtensorMap map_x, map_w, map_y;
   if (!make_map(&map_x, X, k_in, tokens, ldx, kBlockM)) return BSP_ERR_CUDA;
   if (!make_map(&map_w, plan, k_in, n_out, k_in, kPairBN / 2)) return BSP_ERR_CUDA;
-  if (!make_map(&map_y, Y, n_out, tokens, ldy, kBlockM)) return BSP_ERR_CUDA;
+  if (!make_map(&map_y, Y, n_out, tokens, ldy, kBlockM, kEpiCols)) return BSP_ERR_CUDA;
   if (!dev->attr_set[5]) {
     BSP_CUDA_TRY(cudaFuncSetAttribute(linear_tc_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPairSmemBytes));
     dev->attr_set[5] = true;

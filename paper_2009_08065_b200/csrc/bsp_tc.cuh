@@ -17,8 +17,10 @@ constexpr int kBlockK = 64;       // bf16 elements per pipeline stage row = 128 
 constexpr int kUmmaK = 16;        // K of one tcgen05.mma for 16-bit inputs
 constexpr int kThreads = 320;     // 10 warps: producer, mma, 2 x 4 epilogue
 constexpr int kSmemLimit = 232448;              // 227 KB of dynamic shared memory per CTA
-constexpr int kEpiCols = 64;                    // columns per epilogue piece = one 128-byte swizzle row of bf16
-constexpr int kEpiStage = kBlockM * kEpiCols * 2;
+constexpr int kEpiCols = 32;                    // columns per epilogue piece = one 64-byte swizzle row of bf16
+constexpr int kEpiStage = kBlockM * kEpiCols * 2;     // one staging buffer: 128 rows x 64 bytes
+constexpr int kEpiBuffers = 4;                  // two per epilogue group, so a store can drain while the next piece is staged
+constexpr int kEpiBytes = kEpiBuffers * kEpiStage;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s per wait
 
 
@@ -29,7 +31,7 @@ struct TileCfg {
   static constexpr int kStageA = kBlockM * kBlockK * 2;
   static constexpr int kStageB = BN * kBlockK * 2;
   static constexpr int kStage = kStageA + kStageB;
-  static constexpr int kFixed = 1024 /*alignment slack*/ + 2 * kEpiStage + 2 * BN * 2 /*bias, two tiles*/ + 256 /*barriers*/;
+  static constexpr int kFixed = 1024 /*alignment slack*/ + kEpiBytes + 2 * BN * 2 /*bias, two tiles*/ + 256 /*barriers*/;
   static constexpr int kStages = ((kSmemLimit - kFixed) / kStage) > 8 ? 8 : ((kSmemLimit - kFixed) / kStage);
   static constexpr int kTmemCols = 2 * BN <= 32 ? 32 : 2 * BN <= 64 ? 64 : 2 * BN <= 128 ? 128 : 2 * BN <= 256 ? 256 : 512;
   static constexpr int kSmemBytes = kStages * kStage + kFixed;
@@ -177,27 +179,27 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return r;
 }
 
-// One 64-column piece of a thread's accumulator row, with the bias of those columns.
+// One 32-column piece of a thread's accumulator row, with the bias of those columns.
 struct EpiloguePiece {
-  uint32_t v0[32], v1[32];   // float32 accumulators as bits
-  uint4 bias[8];             // 64 bf16 values
+  uint32_t v[32];            // float32 accumulators as bits
+  uint4 bias[4];             // 32 bf16 values
 };
-// Issues the TMEM loads and, while they are in flight, the eight shared-memory loads of the
-// bias; returns once the accumulator values are in registers.  Shared memory is also being
-// written by TMA and read by the tensor core all the time, so a shared load takes on the order of
-// 150 cycles here: the loads must be in flight together, not one per use.
+// Issues the TMEM load and, while it is in flight, the four shared-memory loads of the bias;
+// returns once the accumulator values are in registers.  Shared memory is also being written by
+// TMA and read by the tensor core all the time, so a shared load takes on the order of 150 cycles
+// here: the loads must be in flight together, not one per use.
 __device__ __forceinline__ void piece_load(uint32_t taddr, uint32_t bias_smem, EpiloguePiece& p) {
-  tmem_load_32cols(taddr, p.v0);
-  tmem_load_32cols(taddr + 32, p.v1);
+  tmem_load_32cols(taddr, p.v);
 #pragma unroll
-  for (int j = 0; j < 8; ++j) p.bias[j] = ld_shared_v4(bias_smem + 16u * j);
+  for (int j = 0; j < 4; ++j) p.bias[j] = ld_shared_v4(bias_smem + 16u * j);
   tmem_load_wait();
 }
-// bias + optional GELU + bf16 rounding, into this thread's row of the swizzled staging buffer.
+// bias + optional GELU + bf16 rounding, into this thread's 64-byte row of a staging buffer laid out
+// as a TMA store with the 64-byte swizzle expects it (16-byte chunk c of row r at chunk c ^ ((r >> 1) & 3)).
 __device__ __forceinline__ void piece_store(const EpiloguePiece& p, int act, uint32_t dst_row, uint32_t row_xor) {
 #pragma unroll
-  for (int j = 0; j < 8; ++j) {        // 8 outputs -> one 16-byte chunk of the 128-byte staging row
-    const uint32_t* v = j < 4 ? &p.v0[j * 8] : &p.v1[(j - 4) * 8];
+  for (int j = 0; j < 4; ++j) {        // 8 outputs -> one 16-byte chunk
+    const uint32_t* v = &p.v[j * 8];
     const uint32_t bw[4] = {p.bias[j].x, p.bias[j].y, p.bias[j].z, p.bias[j].w};
     float f[8];
 #pragma unroll
@@ -236,17 +238,19 @@ inline EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
-// 2-D bf16 tensor [outer, inner] row-major with leading dimension ld; box [box_outer, 64] with
-// the 128-byte swizzle; out-of-range elements read as zero.
-inline bool make_map(CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer, uint64_t ld, uint32_t box_outer) {
+// 2-D bf16 tensor [outer, inner] row-major with leading dimension ld; box [box_outer, box_inner]:
+// 64 columns with the 128-byte swizzle (operand tiles) or 32 columns with the 64-byte swizzle
+// (epilogue pieces); out-of-range elements read as zero and are not written.
+inline bool make_map(CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer, uint64_t ld, uint32_t box_outer,
+                     uint32_t box_inner = 64) {
   EncodeTiledFn fn = encode_tiled_fn();
   if (!fn) return false;
   const cuuint64_t dims[2] = {inner, outer};
   const cuuint64_t strides[1] = {ld * 2};
-  const cuuint32_t box[2] = {static_cast<cuuint32_t>(kBlockK), box_outer};
+  const cuuint32_t box[2] = {box_inner, box_outer};
   const cuuint32_t elem[2] = {1, 1};
   return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, elem,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, box_inner == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
