@@ -47,8 +47,10 @@ struct LinearParams {
   int* status;
 };
 
+constexpr int kThreadsTc = kThreads + 32;   // 11 warps: a second TMA producer warp for the weight tiles
+
 template <int BN>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreadsTc, 1)
 linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                  const __grid_constant__ CUtensorMap map_y, LinearParams P) {
   using Cfg = TileCfg<BN>;
@@ -73,7 +75,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_x)) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_w)) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_y)) : "memory");
-    for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 2); mbar_init(empty_bar(s), 1); }   // two producers arm a stage
     for (int a = 0; a < 2; ++a) { mbar_init(acc_full_bar(a), 1); mbar_init(acc_empty_bar(a), 8); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -101,19 +103,19 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
   const int k_blocks = (P.k_in + kBlockK - 1) / kBlockK;
 
   if (warp == 0 && lane == 0) {
-    // ---------------------------------------------------------------- TMA producer
+    // ---------------------------------------------------------------- TMA producer of the X tiles
+    // (one thread issues a tensor copy every few hundred cycles at best, so the two operands of a stage
+    // come from two warps: this one and warp 10)
     int stage = 0;
     uint32_t phase = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-      const int m0 = (tile / n_tiles) * kBlockM, n0 = (tile % n_tiles) * BN;
+      const int m0 = (tile / n_tiles) * kBlockM;
       for (int kb = 0; kb < k_blocks; ++kb) {
         if (!mbar_wait(empty_bar(stage), phase ^ 1u)) { ok = false; break; }
         const uint32_t a_dst = smem_base + stage * Cfg::kStage;
-        const uint32_t b_dst = a_dst + Cfg::kStageA;
-        mbar_arrive_expect_tx(full_bar(stage), Cfg::kStage);
+        mbar_arrive_expect_tx(full_bar(stage), Cfg::kStageA);
         tma_load_2d(a_dst, &map_x, kb * kBlockK, m0, full_bar(stage));
-        tma_load_2d(b_dst, &map_w, kb * kBlockK, n0, full_bar(stage));
         if (++stage == S) { stage = 0; phase ^= 1u; }
       }
     }
@@ -126,6 +128,21 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         (void)mbar_wait(full_bar(back), ph);
       }
     }
+  } else if (warp == 10 && lane == 0) {
+    // ---------------------------------------------------------------- TMA producer of the weight tiles
+    int stage = 0;
+    uint32_t phase = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+      const int n0 = (tile % n_tiles) * BN;
+      for (int kb = 0; kb < k_blocks; ++kb) {
+        if (!mbar_wait(empty_bar(stage), phase ^ 1u)) { ok = false; break; }
+        mbar_arrive_expect_tx(full_bar(stage), Cfg::kStageB);
+        tma_load_2d(smem_base + stage * Cfg::kStage + Cfg::kStageA, &map_w, kb * kBlockK, n0, full_bar(stage));
+        if (++stage == S) { stage = 0; phase ^= 1u; }
+      }
+    }
+    if (!ok) atomicExch(P.status, BSP_ERR_TIMEOUT);
   } else if (warp == 1 && lane == 0) {
     // ---------------------------------------------------------------- MMA issuer
     constexpr uint32_t idesc = instr_desc_bf16(BN);
@@ -158,7 +175,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
       acc ^= 1;
     }
     if (!ok) atomicExch(P.status, BSP_ERR_TIMEOUT);
-  } else if (warp >= 2) {
+  } else if (warp >= 2 && warp < 10) {
     // ---------------------------------------------------------------- epilogue
     const int group = (warp - 2) >> 2;       // 0 or 1
     const int quad = warp & 3;               // TMEM lanes [32*quad, 32*quad+32) belong to this warp
@@ -334,7 +351,7 @@ int launch_tc(TcDevice* dev, int slot, const void* plan, const void* X, void* Y,
   const int grid = tiles < dev->sms ? tiles : dev->sms;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(grid);
-  cfg.blockDim = dim3(kThreads);
+  cfg.blockDim = dim3(kThreadsTc);
   cfg.dynamicSmemBytes = Cfg::kSmemBytes;
   cfg.stream = s;
   cudaLaunchAttribute attr[1];
