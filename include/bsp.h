@@ -258,6 +258,15 @@ int bsp_linear_plan_r(const int32_t* blk_ptr, const int32_t* row_idx, const void
  * plan_bytes as bsp_linear_plan_bytes(n_out, k_in, block).  Errors as bsp_linear_plan. */
 int bsp_linear_plan_t(const int32_t* blk_ptr, const int32_t* idx, const void* vals,
                       int n_out, int k_in, int block, void* plan_t, size_t plan_bytes, void* stream);
+/* bsp_linear_backward_weight — the weight gradient of the masked layer that Algorithm 2 retrains
+ * (W = W * Mask after every step):  dW = (dY^T X) * Mask, with dY [tokens, n_out] (ldy) and
+ * X [tokens, k_in] (ldx) bf16, float32 accumulation over the tokens on the tensor cores, dW
+ * [n_out, k_in] (lddw) rounded to bf16.  keep: per-group flags [n_out/block, k_in] as written by
+ * bsp_prune_pack (orientation C); groups with flag 0 are written as +0; NULL = no mask.
+ * Needs 16-byte aligned pointers and n_out, k_in and the leading dimensions multiples of 8
+ * (else BSP_ERR_UNSUPPORTED).  Bounded waits as bsp_linear_planned: check bsp_linear_status. */
+int bsp_linear_backward_weight(const void* dY, int ldy, const void* X, int ldx, int tokens, int n_out, int k_in,
+                               int block, const uint8_t* keep, void* dW, int lddw, void* stream);
 int bsp_linear_planned(const void* plan, int n_out, int k_in, int block,
                        const void* X, int tokens, int ldx, const void* bias, int act,
                        void* Y, int ldy, void* stream);

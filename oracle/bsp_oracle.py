@@ -381,6 +381,12 @@ def linear_backward_input(dy_bits: np.ndarray, w_bits: np.ndarray, mask: np.ndar
     return bf16_to_f64(dy_bits) @ (bf16_to_f64(w_bits) * mask)
 
 
+def linear_backward_weight(dy_bits: np.ndarray, x_bits: np.ndarray, mask: np.ndarray) -> np.ndarray:
+    """dW[n, k] = Mask[n, k] * sum_t dY[t, n] * X[t, k]: the gradient with respect to the weight of the masked
+    layer of Algorithm 2's retraining loop; pruned positions get no gradient (W = W * Mask).  float64."""
+    return (bf16_to_f64(dy_bits).T @ bf16_to_f64(x_bits)) * mask
+
+
 def row_scales(x_bits: np.ndarray, w_bits: np.ndarray, mask: np.ndarray,
                bias_bits: Optional[np.ndarray]) -> np.ndarray:
     """||X[t,:]||_2 * ||(W*Mask)[n,:]||_2 + |b[n]|: the magnitude an output's error is judged against."""

@@ -82,6 +82,7 @@ _SIGNATURES = {
     "bsp_linear_plan": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _sz, _vp]),
     "bsp_linear_plan_r": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _sz, _vp]),
     "bsp_linear_plan_t": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _sz, _vp]),
+    "bsp_linear_backward_weight": (_i, [_vp, _i, _vp, _i, _i, _i, _i, _i, _vp, _vp, _i, _vp]),
     "bsp_linear_planned": (_i, [_vp, _i, _i, _i, _vp, _i, _i, _vp, _i, _vp, _i, _vp]),
     "bsp_linear_planned_ex": (_i, [_vp, _i, _i, _i, _vp, _i, _i, _vp, _i, _vp, _i, _i, _vp]),
     "bsp_linear": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _i, _i, _vp, _i, _vp, _i, _vp, _sz, _vp]),
@@ -277,6 +278,13 @@ def bsp_linear_plan_t(packed: PackedMatrix, plan_t: torch.Tensor, stream=None) -
     _check(lib.bsp_linear_plan_t(_ptr(packed.blk_ptr), _ptr(packed.idx), _ptr(packed.vals), packed.rows, packed.cols,
                                  packed.block, _ptr(plan_t), plan_t.numel() * plan_t.element_size(), _stream(stream)),
            "bsp_linear_plan_t")
+
+
+def bsp_linear_backward_weight(dY: torch.Tensor, X: torch.Tensor, block: int, keep: Optional[torch.Tensor],
+                               dW: torch.Tensor, stream=None) -> None:
+    """dW = (dY^T X) * Mask; dY [tokens, n_out], X [tokens, k_in], dW [n_out, k_in], all bf16."""
+    _check(lib.bsp_linear_backward_weight(_ptr(dY), _ld(dY), _ptr(X), _ld(X), dY.shape[0], dY.shape[1], X.shape[1], block,
+                                          _ptr(keep), _ptr(dW), _ld(dW), _stream(stream)), "bsp_linear_backward_weight")
 
 
 def bsp_linear_planned(plan: torch.Tensor, n_out: int, k_in: int, block: int, X: torch.Tensor,

@@ -104,8 +104,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
 
   if (warp == 0 && lane == 0) {
     // ---------------------------------------------------------------- TMA producer of the X tiles
-    // (one thread issues a tensor copy every few hundred cycles at best, so the two operands of a stage
-    // come from two warps: this one and warp 10)
+    // (the two operands of a stage are issued by two warps, this one and warp 10, so neither waits
+    // behind the other's copy)
     int stage = 0;
     uint32_t phase = 0;
     bool ok = true;

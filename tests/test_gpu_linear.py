@@ -232,3 +232,27 @@ def test_backward_with_respect_to_activations():
     # error scale: ||dY[t, :]|| * ||(W * Mask)[:, k]||
     scales = np.sqrt((O.bf16_to_f64(dy) ** 2).sum(1))[:, None] * np.sqrt(((O.bf16_to_f64(wp) * m) ** 2).sum(0))[None, :]
     assert_linear_close(bits_of(dx), ref, np.maximum(scales, 1e-30), "dX")
+
+
+@pytest.mark.parametrize("T,N,K,d", [(4096, 768, 768, 16), (1000, 520, 264, 8), (130, 136, 72, 8), (50, 256, 3072, 32)])
+def test_backward_with_respect_to_weights(T, N, K, d):
+    """dW = (dY^T X) * Mask on the tensor cores (contraction over tokens, MN-major operand tiles)."""
+    spec = si.LinearSpec(f"bww{T}", N, K, False, 2.0, d)
+    wp, keep = si.make_pruned_weight(17, spec)
+    x = si.make_activations(17, spec.name, T, K)
+    dy = si.make_activations(18, spec.name + ".dy", T, N)
+    keep_dev = torch.from_numpy(keep.astype(np.uint8)).to(DEV)
+    dw = torch.full((N, K), 0x7FC0, dtype=torch.int16, device=DEV)
+    bsp.bsp_linear_backward_weight(to_dev(dy), to_dev(x), d, keep_dev, dw)
+    bsp.bsp_linear_status()
+    torch.cuda.synchronize()
+    m = O.mask_of(wp)
+    ref = O.linear_backward_weight(dy, x, m)
+    got = bits_of(dw)
+    assert not (got[~m] & 0x7FFF).any()                                   # pruned positions carry no gradient
+    scales = np.sqrt((O.bf16_to_f64(dy) ** 2).sum(0))[:, None] * np.sqrt((O.bf16_to_f64(x) ** 2).sum(0))[None, :]
+    assert_linear_close(got, ref, np.maximum(scales, 1e-30), "dW")
+    # without a mask: the plain product
+    bsp.bsp_linear_backward_weight(to_dev(dy), to_dev(x), d, None, dw)
+    bsp.bsp_linear_status()
+    assert_linear_close(bits_of(dw), O.linear_backward_weight(dy, x, np.ones_like(m)), np.maximum(scales, 1e-30), "dW dense")

@@ -469,3 +469,22 @@ def test_backward_input_is_the_adjoint_of_the_forward_layer():
     dy1[:, :d] = dy[:, :d]                      # only row-block 0's outputs carry gradient
     dx1 = O.linear_backward_input(dy1, wp, m)
     assert (dx1[:, ~keep[0]] == 0).all() and (dx1[:, keep[0]] != 0).any()
+
+
+def test_backward_weight_is_the_adjoint_in_w():
+    """<dY, X (V*M)^T> == <(dY^T X)*M, V> for any V: pins the weight gradient to the forward layer; and a
+    brute-force entry."""
+    T, N, K, d = 7, 8, 12, 4
+    spec = si.LinearSpec("adjw", N, K, False, 2.0, d)
+    wp, keep = si.make_pruned_weight(43, spec)
+    v = si.make_weight(44, spec)                       # an arbitrary direction in weight space
+    x = si.make_activations(43, "adjw", T, K)
+    dy = si.make_activations(44, "adjw.dy", T, N)
+    m = O.mask_of(wp)
+    dw = O.linear_backward_weight(dy, x, m)
+    lhs = (O.bf16_to_f64(dy) * O.linear_masked_dense(x, v, m, None, 0)).sum()
+    assert lhs == pytest.approx((dw * O.bf16_to_f64(v)).sum(), rel=1e-13)
+    assert (dw[~m] == 0).all()
+    n, k = [int(a[0]) for a in np.nonzero(m)]
+    brute = sum(float(O.bf16_to_f64(dy)[t, n]) * float(O.bf16_to_f64(x)[t, k]) for t in range(T))
+    assert dw[n, k] == pytest.approx(brute, rel=1e-14)
