@@ -25,6 +25,8 @@
 // Every wait is bounded by a wall-clock deadline; on expiry the role records BSP_ERR_TIMEOUT in
 // the status word and leaves its loop, the other roles then time out on their own waits, and
 // the CTA frees its tensor memory and exits.
+#include <mutex>
+
 #include "bsp_tc.cuh"
 
 namespace bsp {
@@ -372,6 +374,8 @@ bool tc_path_ok(const void* plan, int n_out, int k_in, const void* X, int ldx, c
 
 TcDevice* tc_device() {
   static TcDevice info[64];
+  static std::mutex guard;             // first calls from several host threads must not race on the set-up
+  std::lock_guard<std::mutex> lock(guard);
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
   TcDevice& d = info[dev];

@@ -9,6 +9,8 @@
 // two-stage kernels of bsp_fused.cu; this file holds the generic kernels (any alignment,
 // orientation R, with a single-CTA scan between (1) and (2)), the keep-count and percentile
 // kernels, and the entry points.
+#include <mutex>
+
 #include "bsp_common.cuh"
 
 namespace bsp {
@@ -330,6 +332,8 @@ extern "C" int bsp_prune_pack_static(const void* W, int rows, int cols, int ldw,
   // In host code the array's name is only a handle; the device address has to be asked for,
   // once per device, while that device is current.
   static void* scratch_of_device[64] = {nullptr};
+  static std::mutex guard;
+  std::lock_guard<std::mutex> lock(guard);
   int dev = -1;
   BSP_CUDA_TRY(cudaGetDevice(&dev));
   if (dev < 0 || dev >= 64) return BSP_ERR_UNSUPPORTED;

@@ -96,6 +96,24 @@ def test_argument_errors_are_caught_before_any_launch():
     assert lib.bsp_prepare_batched(ctypes.pointer(job), 1, 16, 1e-3, 0, None) == -1      # W is NULL
     job.W, job.rows, job.cols, job.ldw = 0x1000, 40, 64, 64
     assert lib.bsp_prepare_batched(ctypes.pointer(job), 1, 16, 1e-3, 0, None) == -2      # 16 does not divide 40
+    # penalty gradient, the other plans, the weight gradient, the chain: checked before any launch
+    assert lib.bsp_penalty_grad(p, 8, 8, 8, 3, 0, 0, p, 1.0, p, 8, 0, None) == -2
+    assert lib.bsp_penalty_grad(p, 8, 8, 8, 2, 0, 0, None, 1.0, p, 8, 0, None) == -1
+    assert lib.bsp_penalty_grad(p, 8, 8, 8, 2, 0, 0, p, 1.0, p, 4, 0, None) == -2          # ldg < cols
+    assert lib.bsp_linear_plan_r(p, p, p, 8, 9, 2, ws, 1 << 20, None) == -2                  # h does not divide k_in
+    assert lib.bsp_linear_plan_r(p, p, p, 8, 8, 2, ws, 16, None) == -3
+    assert lib.bsp_linear_plan_t(p, p, p, 10, 8, 4, ws, 1 << 20, None) == -2
+    assert lib.bsp_linear_plan_t(None, p, p, 8, 8, 4, ws, 1 << 20, None) == -1
+    assert lib.bsp_linear_backward_weight(p, 8, p, 8, 4, 10, 8, 4, None, p, 8, None) == -2  # block does not divide n_out
+    assert lib.bsp_linear_backward_weight(p, 8, p, 8, 4, 8, 8, 4, None, None, 8, None) == -1
+    assert lib.bsp_linear_backward_weight(p, 4, p, 8, 4, 8, 8, 4, None, p, 8, None) == -2   # ldy < n_out
+    assert lib.bsp_linear_backward_weight(ctypes.c_void_p(0x1008), 8, p, 8, 4, 8, 8, 4, None, p, 8, None) == -6
+    assert lib.bsp_linear_planned_ex(ws, 8, 8, 4, p, 4, 8, None, 0, p, 8, 9, None) == -1    # unknown variant
+    n = ctypes.c_size_t()
+    assert lib.bsp_linear_chain_ws_bytes(0, 128, ctypes.byref(n)) == -1
+    assert lib.bsp_linear_chain_ws_bytes(9, 128, ctypes.byref(n)) == -1
+    assert lib.bsp_linear_chain_ws_bytes(4, 4096, ctypes.byref(n)) == 0 and n.value == 512
+    assert lib.bsp_linear_chain(None, 1, p, 4, 8, ws, 1 << 20, None) == -1
     # zero tokens is a valid no-op
     assert lib.bsp_linear_cuda_core(p, p, p, 8, 8, 4, p, 0, 8, None, 0, p, 8, None) == 0
 
