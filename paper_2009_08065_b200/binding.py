@@ -35,7 +35,7 @@ def _load() -> ctypes.CDLL:
     path = library_path()
     if not os.path.exists(path):
         raise ImportError(
-            f"{path} is missing: build it with `python -m paper_2009_08065_b200.build` "
+            f"{path} is missing: build it with `python paper_2009_08065_b200/build.py` "
             "(needs nvcc); this package has no fallback path")
     return ctypes.CDLL(path)
 
