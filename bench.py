@@ -272,7 +272,7 @@ def weight_side_bandwidth(device, peaks, iters=10):
     # algorithmic bytes: W read once (2 B/weight); norms + gamma (4 B each) and a flag (1 B) per group;
     # kept values (2 B) and one index (4 B) per kept group; the execution layout (2 B/weight)
     alg = 2 * weights + 9 * groups + 2 * d * kept + 4 * kept + 2 * weights
-    return {"kernels": "fused_stage1_kernel + fused_stage2_kernel (bsp_prepare_batched)",
+    return {"kernels": "fused_stream_kernel (bsp_prepare_batched; W read once) + its clearing kernel",
             "workload": f"72 BERT-base weight matrices in one call, {weights * 2 / 1e6:.1f} MB of bf16 weights, d=16, ~3x",
             "ms": round(t, 4), "algorithmic_mb": round(alg / 1e6, 1), "achieved_gbs": round(alg / t / 1e6, 1),
             "peak_gbs": float(peaks["hbm_gbs"]), "frac": round(alg / t / 1e6 / float(peaks["hbm_gbs"]), 4),
@@ -382,7 +382,7 @@ def run_cuda(args):
             "config": {
                 "workload": wl.name + " (one BERT-base encoder layer: QKV, attn-out, FFN-up+GELU, FFN-down; "
                             "tokens per GPU 4096; 16-row blocks; 3.0x compression)",
-                "step": "bsp_prepare_batched (norms+gamma+penalty, keep flags, pack, plan of the 4 matrices: 2 launches) "
+                "step": "bsp_prepare_batched (norms+gamma+penalty, keep flags, pack, plan of the 4 matrices: a clearing kernel and one kernel that reads W once) "
                         "then the 4 GEMMs in sequence (bsp_linear_planned; the single chained launch bsp_linear_chain measured "
                         "8 % slower on this workload); one CUDA graph",
                 "l2": f"flushed between steps by writing {L2_FLUSH_BYTES >> 20} MiB",

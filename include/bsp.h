@@ -194,9 +194,11 @@ int bsp_apply_mask(void* W, int rows, int cols, int ldw, int block, int orient,
  * bsp_prepare_batched — the weight-side steps of the path for several matrices at once
  * (orientation C): the norms / gamma / penalty of Section 3.2, Algorithm 1's keep decision, the
  * packed storage of Section 3.1 and, optionally, bsp_linear's execution layout, in two launches
- * for the whole batch instead of four or more per matrix.  Results are those of
+ * per 96 matrices (a small clearing kernel and one kernel that reads every weight exactly once)
+ * instead of four or more per matrix.  Results are those of
  * bsp_group_norms + bsp_prune_pack (threshold mode) + bsp_linear_plan called per matrix, bit
  * for bit; the penalty is summed in a fixed order here and is reproducible run to run.
+ * The kernel's bounded waits report through bsp_linear_status (BSP_ERR_TIMEOUT).
  *
  * jobs: HOST array of n_jobs descriptors; the pointers inside are device pointers with the
  * meaning they have in the single-matrix calls.  norms, gamma_in, gamma_out, penalty, keep,

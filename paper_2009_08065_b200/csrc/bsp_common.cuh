@@ -103,9 +103,9 @@ constexpr int kFusedMaxBlocks = 1024;   // stage 2 sums the counts before its bl
 int fused_stage1(const FusedJob* jobs, int n_jobs, int block, float eps, int squared, cudaStream_t s);
 // Stage 2: blk_ptr, index lists, packed tiles, penalty totals, optional execution layout.
 int fused_stage2(const FusedJob* jobs, int n_jobs, int block, cudaStream_t s);
-// One cooperative launch for a small batch (bsp_fused_onepass.cu); *used = false means nothing was launched.
-int fused_onepass(const FusedJob* jobs, int n_jobs, int block, float eps, int squared, int32_t* const* part_counts,
-                  double* const* part_partial, cudaStream_t s, bool* used);
+// Streaming one-pass kernel for batches of any size (bsp_fused_stream.cu); *used = false means nothing was launched.
+int fused_stream(const FusedJob* jobs, int n_jobs, int block, float eps, int squared, int32_t* const* part_counts,
+                 double* const* part_partial, cudaStream_t s, bool* used);
 // Whether a matrix can go through the vectorised kernels.
 inline bool fused_shape_ok(const void* W, int rows, int cols, int ldw, int block) {
   return cols % 8 == 0 && ldw % 8 == 0 && aligned_to(W, 16) && cols <= kFusedMaxCols && rows / block <= kFusedMaxBlocks;

@@ -379,24 +379,28 @@ extern "C" int bsp_prepare_batched(const bsp_layer_job* jobs, int n_jobs, int bl
                      u.kept_weights, static_cast<uint16_t*>(u.plan)};
   }
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  // Small batches (all CTAs resident at once) take the one-launch path; its per-part counts and
-  // penalty partials live in the workspace's S region, which this call does not use otherwise.
+  // The streaming one-pass kernel (W read once) takes the batch when every matrix fits its limits.  Its
+  // per-item counts and penalty partials live in the workspace's S region, which this call does not use otherwise.
   int st = BSP_OK;
   bool done = false;
-  if (n_jobs <= 16) {
-    int32_t* pcounts[16];
-    double* ppartial[16];
-    for (int i = 0; i < n_jobs; ++i) {
+  {
+    int32_t** pcounts = new (std::nothrow) int32_t*[n_jobs];
+    double** ppartial = new (std::nothrow) double*[n_jobs];
+    bool fits = pcounts != nullptr && ppartial != nullptr;
+    for (int i = 0; i < n_jobs && fits; ++i) {
       const bsp_layer_job& u = jobs[i];
       const int nb = u.rows / block;
       const WsLayout L = ws_layout(nb, u.cols);
       char* region = static_cast<char*>(u.ws) + L.sumsq_off;          // 4 bytes per group
-      const size_t slots = static_cast<size_t>(nb) * 32;              // at most 32 parts per block
+      const size_t slots = static_cast<size_t>(nb) * 32;              // at most 31 parts per block, plus two counters
       pcounts[i] = reinterpret_cast<int32_t*>(region);
       ppartial[i] = reinterpret_cast<double*>(region + round_up(slots * sizeof(int32_t), 256));
-      if (round_up(slots * 4, 256) + slots * 8 > static_cast<size_t>(nb) * u.cols * 4) { pcounts[0] = nullptr; break; }
+      if (round_up(slots * 4, 256) + slots * 8 > static_cast<size_t>(nb) * u.cols * 4) fits = false;
     }
-    if (pcounts[0] != nullptr) st = fused_onepass(fj, n_jobs, block, eps, pen == BSP_PEN_L2SQ ? 1 : 0, pcounts, ppartial, s, &done);
+    const int squared = pen == BSP_PEN_L2SQ ? 1 : 0;
+    if (fits) st = fused_stream(fj, n_jobs, block, eps, squared, pcounts, ppartial, s, &done);
+    delete[] pcounts;
+    delete[] ppartial;
   }
   if (st == BSP_OK && !done) {
     st = fused_stage1(fj, n_jobs, block, eps, pen == BSP_PEN_L2SQ ? 1 : 0, s);

@@ -1,0 +1,457 @@
+// Streaming one-pass form of the vectorised weight-side kernels, for batches of any size: W is
+// read from HBM exactly once.
+//
+// A work item is one row-block of one matrix (or a column range of it, so that its rows fit 24 KB
+// of shared memory).  Every CTA takes one item from a ticket counter, so every item with a smaller
+// number has been taken, and is being worked on, before.  The CTA
+//   load     has the item's rows brought into shared memory by bulk asynchronous copies (one per
+//            row, all in flight at once, completion on an mbarrier);
+//   phase A  computes the float32 sums of squares from shared memory (rows in increasing order, the
+//            defined decision quantity), writes norms / gamma / keep flags, and publishes its kept
+//            count (with a "ready" bit) and its penalty partial;
+//   local    lists its kept columns and writes its part of the zero-expanded execution layout,
+//            neither of which depends on other items;
+//   phase B  reads the published counts of the items before it in the same matrix (bounded
+//            relaxed loads), which give blk_ptr and the position of its part of the packed tile,
+//            and writes indices and tile from shared memory.
+// Shared memory per CTA is small (26 KB at 16-row blocks), so eight CTAs share an SM and their
+// phases overlap: the latency of one item's chain is hidden by the other seven.
+// Why this cannot deadlock: a published count depends on nobody, and a taken item is published
+// without waiting.  An item waits for items with a smaller number (all taken) and, when its
+// row-block is split into column ranges, for the later ranges of its own block; at most one block
+// straddles the ticket counter, so fewer than 32 CTAs can wait for items nobody has taken, and the
+// GPU holds more CTAs than that at once.
+// Counts and penalty partials are published as single words that carry their own "ready" bit (the
+// lowest mantissa bit of the float64 partial), read with relaxed loads: a reader needs nothing but
+// the word itself, so no fence is involved.  The last item of a matrix adds the partials in a fixed
+// order.  Masks, indices, tiles, norms and gamma are bit-identical to the two-stage path.
+#include <new>
+
+#include "bsp_tc.cuh"
+
+namespace bsp {
+namespace {
+
+using tc::mbar_init;
+using tc::mbar_arrive_expect_tx;
+using tc::mbar_wait;
+using tc::smem_u32;
+
+constexpr int kStreamMaxJobs = 96;       // per launch; the job table travels as a kernel parameter
+constexpr int kStreamThreads = 128;
+constexpr int kStreamRowBytes = 24 * 1024;   // the row buffer
+constexpr int kReadyBit = 0x40000000;    // set in a published count
+constexpr unsigned long long kSpinLimitNs = 2000000000ull;   // 2 s per wait
+
+struct StreamJob {
+  FusedJob j;
+  int parts, part_cols;      // column ranges per row-block, columns per range (multiple of 8)
+  int first_item;
+  int32_t* part_counts;      // [n_blocks * parts] published counts, then (job 0) the ticket
+  unsigned long long* part_partial;   // [n_blocks * parts] published penalty partials (float64 bits, lowest bit set)
+};
+struct StreamBatch {
+  int n_jobs, block, squared;
+  float eps;
+  int total_items, buf_bytes;
+  int* ticket;
+  int* status;               // receives BSP_ERR_TIMEOUT when a bounded wait expires
+  StreamJob job[kStreamMaxJobs];
+};
+
+struct Item {
+  int jn, local, b, q, c0, pc;
+};
+__device__ __forceinline__ Item locate(const StreamBatch& B, int item) {
+  int lo = 0, hi = B.n_jobs - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (B.job[mid].first_item <= item) lo = mid; else hi = mid - 1;
+  }
+  const StreamJob& O = B.job[lo];
+  Item I;
+  I.jn = lo;
+  I.local = item - O.first_item;
+  I.b = I.local / O.parts;
+  I.q = I.local - I.b * O.parts;
+  I.c0 = I.q * O.part_cols;
+  I.pc = min(O.part_cols, O.j.cols - I.c0);
+  return I;
+}
+
+// Rows of an item into a shared-memory buffer, one bulk copy per row (called by one warp).
+__device__ __forceinline__ void issue_rows(const StreamBatch& B, int item, uint32_t dst, uint32_t bar, int lane) {
+  const Item I = locate(B, item);
+  const FusedJob& J = B.job[I.jn].j;
+  const int d = B.block;
+  const uint32_t row_bytes = static_cast<uint32_t>(I.pc) * 2u;
+  if (lane == 0) mbar_arrive_expect_tx(bar, row_bytes * static_cast<uint32_t>(d));
+  __syncwarp();
+  const uint16_t* wblk = J.W + static_cast<size_t>(I.b) * d * J.ldw + I.c0;
+  for (int r = lane; r < d; r += 32) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst + static_cast<uint32_t>(r) * row_bytes),
+                   "l"(reinterpret_cast<uint64_t>(wblk + static_cast<size_t>(r) * J.ldw)), "r"(row_bytes), "r"(bar)
+                 : "memory");
+  }
+}
+
+// Published count of an item: waits (bounded) for its ready bit.
+__device__ __forceinline__ int wait_count(const int32_t* slot, int* status) {
+  int v;
+  asm volatile("ld.relaxed.gpu.global.b32 %0, [%1];" : "=r"(v) : "l"(slot) : "memory");
+  if (v & kReadyBit) return v & (kReadyBit - 1);
+  const unsigned long long start = tc::global_timer_ns();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 64; ++i) {
+      asm volatile("ld.relaxed.gpu.global.b32 %0, [%1];" : "=r"(v) : "l"(slot) : "memory");
+      if (v & kReadyBit) return v & (kReadyBit - 1);
+      __nanosleep(32);
+    }
+    if (tc::global_timer_ns() - start > kSpinLimitNs) { atomicExch(status, BSP_ERR_TIMEOUT); return 0; }
+  }
+}
+
+// Published penalty partial of an item: waits (bounded) for its ready bit.
+__device__ __forceinline__ double wait_partial(const unsigned long long* slot, int* status) {
+  unsigned long long v;
+  asm volatile("ld.relaxed.gpu.global.b64 %0, [%1];" : "=l"(v) : "l"(slot) : "memory");
+  if (v & 1ull) return __longlong_as_double(static_cast<long long>(v));
+  const unsigned long long start = tc::global_timer_ns();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 64; ++i) {
+      asm volatile("ld.relaxed.gpu.global.b64 %0, [%1];" : "=l"(v) : "l"(slot) : "memory");
+      if (v & 1ull) return __longlong_as_double(static_cast<long long>(v));
+      __nanosleep(32);
+    }
+    if (tc::global_timer_ns() - start > kSpinLimitNs) { atomicExch(status, BSP_ERR_TIMEOUT); return 0.0; }
+  }
+}
+
+__global__ void __launch_bounds__(kStreamThreads, 8)
+fused_stream_kernel(const __grid_constant__ StreamBatch B) {
+  extern __shared__ __align__(128) uint8_t s_raw[];
+  __shared__ __align__(8) uint64_t s_bar;
+  __shared__ int s_item;
+  __shared__ int s_cnt[8];
+  __shared__ double s_pen[8];
+  __shared__ int s_warp[32];
+  __shared__ int s_sum[3];
+  __shared__ int s_kc;
+  const int d = B.block;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, n_warps = blockDim.x >> 5;
+  int32_t* s_idx = reinterpret_cast<int32_t*>(s_raw + static_cast<size_t>(B.buf_bytes));      // [max part columns]
+  const uint32_t bar = smem_u32(&s_bar);
+
+  if (threadIdx.x == 0) {
+    mbar_init(bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    s_item = atomicAdd(B.ticket, 1);
+  }
+  __syncthreads();
+  const int item = s_item;
+  if (item >= B.total_items) return;
+  if (warp == 0) issue_rows(B, item, smem_u32(s_raw), bar, lane);
+  {
+    const Item I = locate(B, item);
+    const StreamJob& O = B.job[I.jn];
+    const FusedJob& J = O.j;
+    const int b = I.b, q = I.q, c0 = I.c0, pc = I.pc, local = I.local;
+    const int chunks = pc >> 3;
+    const uint16_t* s_w = reinterpret_cast<const uint16_t*>(s_raw);                     // [d][pc]
+    uint8_t* s_flag = reinterpret_cast<uint8_t*>(s_idx + O.part_cols);                  // [pc]
+    if (!mbar_wait(bar, 0u)) {
+      atomicExch(B.status, BSP_ERR_TIMEOUT);
+      return;
+    }
+
+    // ---- phase A: sums of squares of 8 adjacent columns per thread, rows in increasing order
+    const bool want_pen = J.penalty != nullptr;
+    const bool want_norms = J.norms != nullptr || J.gamma_out != nullptr || want_pen;
+    const float t = J.threshold_dev ? *J.threshold_dev : J.threshold;
+    const bool keep_all = t < 0.0f;
+    const float t2 = __fmul_rn(t, t);
+    int count = 0;
+    float pen = 0.0f;
+    for (int k = threadIdx.x; k < chunks; k += blockDim.x) {
+      float acc[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) acc[i] = 0.0f;
+      for (int r = 0; r < d; ++r) {
+        const uint4 v = *reinterpret_cast<const uint4*>(s_w + r * pc + (k << 3));
+        const uint32_t w32[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float lo = __uint_as_float(w32[i] << 16), hi = __uint_as_float(w32[i] & 0xffff0000u);
+          acc[2 * i] = __fmaf_rn(lo, lo, acc[2 * i]);
+          acc[2 * i + 1] = __fmaf_rn(hi, hi, acc[2 * i + 1]);
+        }
+      }
+      uint32_t lo = 0, hi = 0;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const uint32_t k0 = (keep_all || acc[i] > t2) ? 1u : 0u;
+        const uint32_t k1 = (keep_all || acc[4 + i] > t2) ? 1u : 0u;
+        lo |= k0 << (8 * i);
+        hi |= k1 << (8 * i);
+        count += static_cast<int>(k0 + k1);
+      }
+      const size_t g0 = static_cast<size_t>(b) * J.cols + c0 + (k << 3);
+      *reinterpret_cast<uint2*>(s_flag + (k << 3)) = make_uint2(lo, hi);
+      *reinterpret_cast<uint2*>(J.flags + g0) = make_uint2(lo, hi);
+      if (want_norms) {
+        float n[8], base[8], fresh[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          n[i] = __fsqrt_rn(acc[i]);
+          base[i] = B.squared ? acc[i] : n[i];
+          fresh[i] = __fdiv_rn(1.0f, base[i] + B.eps);
+        }
+        if (J.norms) {
+          *reinterpret_cast<float4*>(J.norms + g0) = make_float4(n[0], n[1], n[2], n[3]);
+          *reinterpret_cast<float4*>(J.norms + g0 + 4) = make_float4(n[4], n[5], n[6], n[7]);
+        }
+        if (J.gamma_out) {
+          *reinterpret_cast<float4*>(J.gamma_out + g0) = make_float4(fresh[0], fresh[1], fresh[2], fresh[3]);
+          *reinterpret_cast<float4*>(J.gamma_out + g0 + 4) = make_float4(fresh[4], fresh[5], fresh[6], fresh[7]);
+        }
+        if (want_pen) {
+          if (J.gamma_in) {
+            const float4 a = __ldg(reinterpret_cast<const float4*>(J.gamma_in + g0));
+            const float4 c = __ldg(reinterpret_cast<const float4*>(J.gamma_in + g0 + 4));
+            const float w[8] = {a.x, a.y, a.z, a.w, c.x, c.y, c.z, c.w};
+#pragma unroll
+            for (int i = 0; i < 8; ++i) pen = fmaf(w[i], base[i], pen);
+          } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) pen = fmaf(fresh[i], base[i], pen);
+          }
+        }
+      }
+    }
+    count = warp_sum(count);
+    double pd = warp_sum(static_cast<double>(pen));
+    if (lane == 0) { s_cnt[warp] = count; s_pen[warp] = pd; }
+    __syncthreads();
+    const int n_parts = J.n_blocks * O.parts;
+    if (threadIdx.x == 0) {
+      int c = 0;
+      double p = 0.0;
+      for (int w = 0; w < n_warps; ++w) { c += s_cnt[w]; p += s_pen[w]; }
+      asm volatile("st.relaxed.gpu.global.b32 [%0], %1;" ::"l"(O.part_counts + local), "r"(c | kReadyBit) : "memory");
+      if (want_pen)
+        asm volatile("st.relaxed.gpu.global.b64 [%0], %1;" ::"l"(O.part_partial + local),
+                     "l"(static_cast<unsigned long long>(__double_as_longlong(p)) | 1ull) : "memory");
+      s_kc = c;
+      s_sum[0] = 0; s_sum[1] = 0; s_sum[2] = 0;
+    }
+
+    // ---- local work: ascending list of this part's kept columns (local indices in s_idx)
+    int running = 0;
+    for (int k0 = 0; k0 < chunks; k0 += blockDim.x) {
+      const int k = k0 + threadIdx.x;
+      uint2 f = make_uint2(0u, 0u);
+      if (k < chunks) f = *reinterpret_cast<const uint2*>(s_flag + (k << 3));
+      const int mine = __popc(f.x) + __popc(f.y);
+      int total;
+      int p = running + block_exclusive_scan(mine, s_warp, &total);
+      running += total;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const uint32_t bit = ((i < 4 ? f.x : f.y) >> (8 * (i & 3))) & 1u;
+        if (bit) s_idx[p++] = (k << 3) + i;
+      }
+    }
+    // execution layout: the rows with the pruned columns zeroed, one warp per row, 16-byte stores
+    if (J.plan != nullptr) {
+      for (int r = warp; r < d; r += n_warps) {
+        uint16_t* pdst = J.plan + (static_cast<size_t>(b) * d + r) * J.cols + c0;
+        for (int k = lane; k < chunks; k += 32) {
+          const uint4 w = *reinterpret_cast<const uint4*>(s_w + r * pc + (k << 3));
+          const uint2 f = *reinterpret_cast<const uint2*>(s_flag + (k << 3));
+          uint4 m;   // a flag byte is 0 or 1: flag * 0xffff masks the matching 16-bit element
+          m.x = w.x & (((f.x & 0xffu) * 0xffffu) | (((f.x >> 8) & 0xffu) * 0xffff0000u));
+          m.y = w.y & ((((f.x >> 16) & 0xffu) * 0xffffu) | (((f.x >> 24) & 0xffu) * 0xffff0000u));
+          m.z = w.z & (((f.y & 0xffu) * 0xffffu) | (((f.y >> 8) & 0xffu) * 0xffff0000u));
+          m.w = w.w & ((((f.y >> 16) & 0xffu) * 0xffffu) | (((f.y >> 24) & 0xffu) * 0xffff0000u));
+          *reinterpret_cast<uint4*>(pdst + (k << 3)) = m;
+        }
+      }
+    }
+
+    // ---- phase B: offsets from the published counts
+    int before = 0, in_block_before = 0, in_block = 0;
+    for (int i = threadIdx.x; i < local; i += blockDim.x) before += wait_count(O.part_counts + i, B.status);
+    if (O.parts > 1) {
+      for (int i = threadIdx.x; i < O.parts; i += blockDim.x) {
+        const int c = wait_count(O.part_counts + b * O.parts + i, B.status);
+        in_block += c;
+        if (i < q) in_block_before += c;
+      }
+    }
+    before = warp_sum(before);
+    in_block = warp_sum(in_block);
+    in_block_before = warp_sum(in_block_before);
+    __syncthreads();                          // s_sum zeroed, s_kc set, s_idx complete
+    if (lane == 0) {
+      if (before) atomicAdd(&s_sum[0], before);
+      if (in_block) atomicAdd(&s_sum[1], in_block);
+      if (in_block_before) atomicAdd(&s_sum[2], in_block_before);
+    }
+    __syncthreads();
+    const int kc = s_kc;                     // kept groups of this part
+    const int base = s_sum[0];               // kept groups before this item's first one (index into idx)
+    const int kc_block = O.parts > 1 ? s_sum[1] : kc;   // kept groups of the whole row-block
+    const int off_in_block = s_sum[2];       // kept groups of the block's earlier parts
+    const int block_base = base - off_in_block;
+    if (q == 0 && threadIdx.x == 0) {
+      J.blk_ptr[b] = block_base;
+      if (b == J.n_blocks - 1) {
+        J.blk_ptr[J.n_blocks] = block_base + kc_block;
+        if (J.kept_weights) *J.kept_weights = static_cast<int64_t>(block_base + kc_block) * d;
+      }
+    }
+    // penalty total of the matrix, in a fixed order, by its last item (every other item has a smaller number)
+    if (local == n_parts - 1 && want_pen) {
+      double p = 0.0;
+      for (int i = threadIdx.x; i < n_parts; i += blockDim.x) p += wait_partial(O.part_partial + i, B.status);
+      p = warp_sum(p);
+      if (lane == 0) s_pen[warp] = p;
+      __syncthreads();
+      if (threadIdx.x == 0) {
+        double tot = 0.0;
+        for (int w = 0; w < n_warps; ++w) tot += s_pen[w];
+        *J.penalty = tot;
+      }
+    }
+    if (kc > 0) {
+      for (int p = threadIdx.x; p < kc; p += blockDim.x) J.idx[base + p] = c0 + s_idx[p];
+      // packed tile: row r of the block occupies vals[tile0 + r*kc_block, +kc_block); this part fills
+      // positions [off_in_block, off_in_block + kc) of every row.  One warp per row; whole 16-byte
+      // vectors where the destination is aligned, ragged ends by element.
+      const bool vec_ok = (reinterpret_cast<uintptr_t>(J.vals) & 15) == 0;
+      const long long tile0 = static_cast<long long>(d) * block_base;
+      for (int r = warp; r < d; r += n_warps) {
+        const uint16_t* srow = s_w + r * pc;
+        const long long e0 = tile0 + static_cast<long long>(r) * kc_block + off_in_block;
+        uint16_t* out_row = J.vals + e0;
+        if (vec_ok) {
+          const int head = static_cast<int>((8 - (e0 & 7)) & 7);
+          const int n_vec = kc > head ? (kc - head) >> 3 : 0;
+          for (int v = lane; v < n_vec; v += 32) {
+            const int p = head + (v << 3);
+            uint32_t o[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+              o[i] = static_cast<uint32_t>(srow[s_idx[p + 2 * i]]) | (static_cast<uint32_t>(srow[s_idx[p + 2 * i + 1]]) << 16);
+            *reinterpret_cast<uint4*>(out_row + p) = make_uint4(o[0], o[1], o[2], o[3]);
+          }
+          const int tail0 = head + (n_vec << 3);
+          if (lane < 8) {
+            if (lane < head && lane < kc) out_row[lane] = srow[s_idx[lane]];
+          } else if (lane < 16) {
+            const int p = tail0 + (lane - 8);
+            if (p >= head && p < kc) out_row[p] = srow[s_idx[p]];
+          }
+        } else {
+          for (int p = lane; p < kc; p += 32) out_row[p] = srow[s_idx[p]];
+        }
+      }
+    }
+  }
+}
+
+// Zeroes the published counts and partials and the ticket slot of every matrix.
+__global__ void __launch_bounds__(256)
+stream_clear_kernel(const __grid_constant__ StreamBatch B) {
+  const StreamJob& O = B.job[blockIdx.x];
+  const int n = O.j.n_blocks * O.parts;
+  for (int i = threadIdx.x; i < n + 2; i += blockDim.x) O.part_counts[i] = 0;
+  for (int i = threadIdx.x; i < n; i += blockDim.x) O.part_partial[i] = 0ull;
+}
+
+// Fills the job table; false when a matrix does not fit this kernel's limits.
+bool fill_batch(StreamBatch& B, const FusedJob* jobs, int n_jobs, int block, float eps, int squared,
+                int32_t* const* part_counts, double* const* part_partial, size_t* smem_out) {
+  B.n_jobs = n_jobs;
+  B.block = block;
+  B.squared = squared;
+  B.eps = eps;
+  int total = 0, max_part_cols = 0;
+  const int max_cols = (kStreamRowBytes / (2 * block)) / 8 * 8;        // columns whose rows fit a row buffer
+  if (max_cols < 8) return false;
+  for (int i = 0; i < n_jobs; ++i) {
+    StreamJob& O = B.job[i];
+    O.j = jobs[i];
+    const int cols = jobs[i].cols;
+    O.parts = (cols + max_cols - 1) / max_cols;
+    O.part_cols = ((cols + O.parts - 1) / O.parts + 7) / 8 * 8;
+    O.parts = (cols + O.part_cols - 1) / O.part_cols;
+    if (O.parts > 31) return false;
+    if (static_cast<long long>(jobs[i].n_blocks) * O.parts + 2 > static_cast<long long>(jobs[i].n_blocks) * 32) return false;
+    O.first_item = total;
+    O.part_counts = part_counts[i];
+    O.part_partial = reinterpret_cast<unsigned long long*>(part_partial[i]);
+    total += jobs[i].n_blocks * O.parts;
+    if (O.part_cols > max_part_cols) max_part_cols = O.part_cols;
+  }
+  B.total_items = total;
+  B.buf_bytes = static_cast<int>(round_up(static_cast<size_t>(block) * max_part_cols * 2, 128));
+  B.ticket = B.job[0].part_counts + B.job[0].j.n_blocks * B.job[0].parts + 1;
+  *smem_out = static_cast<size_t>(B.buf_bytes) + static_cast<size_t>(max_part_cols) * 5 + 16;
+  return true;
+}
+
+}  // namespace
+
+// Runs the batch through the streaming one-pass kernel (a clearing launch and the kernel, per 96
+// matrices).  *used = false means nothing was launched and the two-stage path should run.
+int fused_stream(const FusedJob* jobs, int n_jobs, int block, float eps, int squared, int32_t* const* part_counts,
+                 double* const* part_partial, cudaStream_t s, bool* used) {
+  *used = false;
+  TcDevice* td = tc_device();
+  if (td == nullptr) return BSP_ERR_CUDA;
+  StreamBatch* B = new (std::nothrow) StreamBatch;
+  if (B == nullptr) return BSP_OK;
+  // every batch is checked before the first launch
+  size_t smem = 0, smem_max = 0;
+  bool ok = true;
+  for (int j0 = 0; j0 < n_jobs && ok; j0 += kStreamMaxJobs) {
+    const int n = n_jobs - j0 < kStreamMaxJobs ? n_jobs - j0 : kStreamMaxJobs;
+    ok = fill_batch(*B, jobs + j0, n, block, eps, squared, part_counts + j0, part_partial + j0, &smem);
+    if (smem > smem_max) smem_max = smem;
+  }
+  constexpr int kSmemCap = 96 * 1024;     // opt-in limit set once per device; a launch asks for what it needs
+  if (ok && smem_max > static_cast<size_t>(kSmemCap)) ok = false;
+  int per_sm = 0;
+  int st = BSP_OK;
+  if (ok) {
+    if (!td->attr_set[7]) {
+      cudaError_t e = cudaFuncSetAttribute(fused_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemCap);
+      if (e != cudaSuccess) { delete B; return cuda_fail(e); }
+      td->attr_set[7] = true;
+    }
+    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fused_stream_kernel, kStreamThreads, smem_max);
+    if (e != cudaSuccess) { delete B; return cuda_fail(e); }
+    if (per_sm * td->sms < 32) ok = false;    // the no-deadlock argument needs 32 CTAs resident at once
+  }
+  for (int j0 = 0; j0 < n_jobs && ok && st == BSP_OK; j0 += kStreamMaxJobs) {
+    const int n = n_jobs - j0 < kStreamMaxJobs ? n_jobs - j0 : kStreamMaxJobs;
+    fill_batch(*B, jobs + j0, n, block, eps, squared, part_counts + j0, part_partial + j0, &smem);
+    B->status = td->status;
+    stream_clear_kernel<<<n, 256, 0, s>>>(*B);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { st = cuda_fail(e); break; }
+    fused_stream_kernel<<<B->total_items, kStreamThreads, smem_max, s>>>(*B);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) { st = cuda_fail(e); break; }
+    *used = true;
+  }
+  delete B;
+  return st;
+}
+
+}  // namespace bsp

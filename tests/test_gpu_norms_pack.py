@@ -262,6 +262,47 @@ def test_prepare_batched_optional_outputs_and_many_jobs():
     assert e.value.status == -6
 
 
+def test_prepare_batched_streaming_batch_larger_than_the_gpu():
+    """More row-blocks than CTAs fit on the GPU at once, with wide matrices split into column ranges:
+    the streaming one-pass kernel (ticket order, published counts) against the oracle, bit for bit."""
+    eps, block = 1e-3, 16
+    shapes = [(768, 768), (3072, 768), (768, 3072)] * 8
+    jobs, refs = [], []
+    for n, (rows, cols) in enumerate(shapes):
+        w = si.student_t_bf16(300 + n, f"stream{n}", (rows, cols), 3.0, 0.02)
+        t_b = float(np.quantile(O.group_norms(w, block, "C"), 0.3 + 0.02 * n))
+        pk = bsp.PackedMatrix.allocate(rows, cols, block, bsp.ORIENT_C, DEV)
+        shape = (rows // block, cols)
+        jobs.append(bsp.LayerJob(
+            W=to_dev(w), out=pk, threshold=t_b,
+            norms=torch.empty(shape, dtype=torch.float32, device=DEV),
+            gamma_out=torch.empty(shape, dtype=torch.float32, device=DEV),
+            penalty=torch.full((1,), -5.0, dtype=torch.float64, device=DEV),
+            plan=torch.empty(bsp.bsp_linear_plan_bytes(rows, cols, block), dtype=torch.uint8, device=DEV)))
+        refs.append((w, t_b))
+    for _ in range(2):                                   # the second call starts from the first one's scratch
+        bsp.bsp_prepare_batched(jobs, block, eps, bsp.PEN_L2)
+        bsp.bsp_linear_status()                          # no bounded wait expired
+        torch.cuda.synchronize()
+        for job, (w, t_b) in zip(jobs, refs):
+            rows, cols = w.shape
+            n_ref = O.group_norms(w, block, "C")
+            g_ref = O.gamma_update(n_ref, eps)
+            assert np.allclose(job.norms.cpu().numpy(), n_ref, rtol=REL, atol=0)
+            assert np.allclose(job.gamma_out.cpu().numpy(), g_ref, rtol=REL, atol=0)
+            assert float(job.penalty.item()) == pytest.approx(O.penalty_l2(n_ref, g_ref), rel=REL)
+            keep_ref = O.keep_flags(w, block, "C", t_b)
+            ref_ptr, ref_idx, ref_vals = O.pack(w, keep_ref, block, "C")
+            blk_ptr, idx, vals, keep, kept = packed_to_host(job.out)
+            assert np.array_equal(keep, keep_ref) and np.array_equal(blk_ptr, ref_ptr)
+            assert np.array_equal(idx, ref_idx) and np.array_equal(vals, ref_vals)
+            assert kept == block * int(keep_ref.sum())
+            plan = bits_of(job.plan.view(torch.int16)[: rows * cols].reshape(rows, cols))
+            assert np.array_equal(plan, O.prune(w, block, "C", t_b))
+            job.out.idx.fill_(-7)
+            job.penalty.fill_(-5.0)
+
+
 # ---------------------------------------------------------------------------------------- penalty gradient
 @pytest.mark.parametrize("orient,block,shape", [(0, 16, (768, 768)), (0, 3, (96, 50)), (1, 12, (96, 768)), (1, 5, (33, 50))])
 def test_penalty_gradient(orient, block, shape):
