@@ -315,6 +315,37 @@ int bsp_linear_chain_ws_bytes(int n_ops, int tokens, size_t* bytes);
 int bsp_linear_chain(const bsp_chain_op* ops, int n_ops, const void* X, int tokens, int ldx,
                      void* ws, size_t ws_bytes, void* stream);
 
+/* ---------------------------------------------------------------------------------------------
+ * bsp_linear_gathered — the same layer, Y = act(X (W * Mask)^T + b), with the pruned work skipped:
+ * for each row-block only the kept columns of X are fetched and multiplied (Section 3.1: only the
+ * non-zero columns of a block take part in the product; Section 4.4: the compact storage is what
+ * saves computation).  Flops executed = 2 * tokens * kept weights (rounded up to 16 kept columns
+ * per block), against 2 * tokens * n_out * k_in for bsp_linear_planned.  Every gathered element
+ * feeds only `block` multiply-adds per token, so this pays off for tall blocks and high
+ * compression; bsp_linear_planned is the better choice for block 16 at 3x.
+ *
+ * XT: the activations TRANSPOSED, bf16 [k_in, tokens] row-major with leading dimension ldxt
+ * (a kept column of X is then a contiguous row); make it with bsp_transpose, or have the producer
+ * of X write it that way.  Y [tokens, n_out] row-major as elsewhere.
+ * gplan: the gather plan, private scratch derived from the packed form by bsp_linear_gather_plan
+ * (per 64 kept columns of a row-block: the weight tile in tensor-core layout, the column numbers,
+ * a stage descriptor), bsp_linear_gather_plan_bytes bytes (worst case: nothing pruned), 256-byte
+ * aligned; built once per pruned matrix and reused for every batch.
+ * Needs block in {16, 32, 64, 128}, k_in < 32768, tokens / ldxt / ldy multiples of 8, 16-byte
+ * aligned XT, Y and bias (else BSP_ERR_UNSUPPORTED).  Bounded waits as bsp_linear_planned: check
+ * bsp_linear_status.  Errors: BSP_ERR_ARG, BSP_ERR_SHAPE, BSP_ERR_WORKSPACE, BSP_ERR_CUDA.
+ *
+ * bsp_transpose — XT[c, r] = X[r, c] for a row-major bf16 matrix [rows, cols] (rows, cols and
+ * both leading dimensions multiples of 8, 16-byte aligned pointers, else BSP_ERR_UNSUPPORTED).
+ */
+int bsp_linear_gather_plan_bytes(int n_out, int k_in, int block, size_t* bytes);   /* host-only */
+int bsp_linear_gather_plan(const int32_t* blk_ptr, const int32_t* idx, const void* vals,
+                           int n_out, int k_in, int block, void* gplan, size_t gplan_bytes, void* stream);
+int bsp_transpose(const void* X, int rows, int cols, int ldx, void* XT, int ldxt, void* stream);
+int bsp_linear_gathered(const void* gplan, int n_out, int k_in, int block,
+                        const void* XT, int tokens, int ldxt, const void* bias, int act,
+                        void* Y, int ldy, void* stream);
+
 /* bsp_linear_cuda_core — the same layer computed straight from the packed form by a plain
  * CUDA-core kernel (one thread per output, float32 accumulation in index order).  It is what
  * bsp_linear falls back to when the alignment rules above do not hold, and is exported so the

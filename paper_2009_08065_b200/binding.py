@@ -77,6 +77,10 @@ _SIGNATURES = {
     "bsp_prune_pack_static": (_i, [_vp, _i, _i, _i, _i, _i, _f, _vp, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
     "bsp_percentile_threshold": (_i, [_vp, _i, _i, _i, _i, _i, _d, _vp, _vp, _sz, _vp]),
     "bsp_apply_mask": (_i, [_vp, _i, _i, _i, _i, _i, _vp, _vp]),
+    "bsp_linear_gather_plan_bytes": (_i, [_i, _i, _i, _szp]),
+    "bsp_linear_gather_plan": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _sz, _vp]),
+    "bsp_transpose": (_i, [_vp, _i, _i, _i, _vp, _i, _vp]),
+    "bsp_linear_gathered": (_i, [_vp, _i, _i, _i, _vp, _i, _i, _vp, _i, _vp, _i, _vp]),
     "bsp_prepare_batched": (_i, [ctypes.POINTER(_LayerJob), _i, _i, _f, _i, _vp]),
     "bsp_linear_plan_bytes": (_i, [_i, _i, _i, _szp]),
     "bsp_linear_plan": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _sz, _vp]),
@@ -308,6 +312,30 @@ def bsp_linear(packed: PackedMatrix, X: torch.Tensor, bias: Optional[torch.Tenso
     _check(lib.bsp_linear(_ptr(packed.blk_ptr), _ptr(packed.idx), _ptr(packed.vals), packed.rows, packed.cols,
                           packed.block, _ptr(X), X.shape[0], _ld(X), _ptr(bias), act, _ptr(Y), _ld(Y), _ptr(ws),
                           0 if ws is None else ws.numel() * ws.element_size(), _stream(stream)), "bsp_linear")
+
+
+def bsp_linear_gather_plan_bytes(n_out: int, k_in: int, block: int) -> int:
+    n = ctypes.c_size_t(0)
+    _check(lib.bsp_linear_gather_plan_bytes(n_out, k_in, block, ctypes.byref(n)), "bsp_linear_gather_plan_bytes")
+    return n.value
+
+
+def bsp_linear_gather_plan(packed: PackedMatrix, gplan: torch.Tensor, stream=None) -> None:
+    _check(lib.bsp_linear_gather_plan(_ptr(packed.blk_ptr), _ptr(packed.idx), _ptr(packed.vals), packed.rows,
+                                      packed.cols, packed.block, _ptr(gplan), gplan.numel() * gplan.element_size(),
+                                      _stream(stream)), "bsp_linear_gather_plan")
+
+
+def bsp_transpose(X: torch.Tensor, XT: torch.Tensor, stream=None) -> None:
+    _check(lib.bsp_transpose(_ptr(X), X.shape[0], X.shape[1], _ld(X), _ptr(XT), _ld(XT), _stream(stream)),
+           "bsp_transpose")
+
+
+def bsp_linear_gathered(gplan: torch.Tensor, n_out: int, k_in: int, block: int, XT: torch.Tensor,
+                        bias: Optional[torch.Tensor], act: int, Y: torch.Tensor, stream=None) -> None:
+    """XT is [k_in, tokens] (the transposed activations); Y is [tokens, n_out]."""
+    _check(lib.bsp_linear_gathered(_ptr(gplan), n_out, k_in, block, _ptr(XT), XT.shape[1], _ld(XT), _ptr(bias), act,
+                                   _ptr(Y), _ld(Y), _stream(stream)), "bsp_linear_gathered")
 
 
 @dataclass

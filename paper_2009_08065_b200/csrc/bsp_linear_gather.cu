@@ -1,0 +1,531 @@
+// bsp_linear_gathered: the pruned linear layer with the pruned work skipped.  For a row-block of
+// d output rows only the kept columns of X are fetched and multiplied (Section 3.1: only the
+// non-zero columns of a block take part; Section 4.4: compact storage saves computation).
+//
+// Operands.  Per row-block the product is  Y[tile, block] = X[tile, kept columns] . vals^T  with
+// 128 tokens as the M side of a tcgen05.mma, the d output rows as its N side and the kept columns
+// as K.  Single columns of a row-major X are 2-byte pieces, useless for 16-byte copies, so the
+// activations are taken TRANSPOSED, XT [k_in, tokens]: a kept column is then a contiguous row of
+// 128 tokens (256 bytes), gathered with 16-byte cp.async copies straight into the tensor core's
+// "MN-major" operand layout (8-row atoms of 64 tokens x 8 columns, 128-byte swizzle).  The weight
+// side comes from a gather plan made once per pruned matrix: per pipeline stage (64 kept columns)
+// the d x 64 tile already in the K-major 128-byte-swizzled layout (one bulk copy lands it), the
+// 64 column numbers, and a byte that says how many 16-column groups are real and whether the stage
+// starts or ends a row-block.
+//
+// Kernel.  Persistent CTAs walk units of (128-token tile) x (run of consecutive row-blocks); the
+// stages of such a run are consecutive in the plan, so the producers just stream them.
+//   warps 0-3 : producers; thread = (16-byte token chunk, row residue mod 8); per stage 8 cp.async
+//               per thread, completion counted on the stage's mbarrier (arrive-on-completion);
+//               thread 0 also issues the bulk copy of the weight tile and hands the stage's byte on;
+//   warp 4    : one lane issues tcgen05.mma (M=128, N=d, K=16) into one of two TMEM accumulators,
+//               commits stage release and, at the end of a row-block, accumulator ready;
+//   warps 5-8 : epilogue; each warp reads its 32 TMEM lanes (tokens), adds bias, optional GELU,
+//               rounds to bf16 and stores its row's d outputs (2 d contiguous bytes).
+// Every wait is bounded; on expiry the role records BSP_ERR_TIMEOUT and leaves its loop.
+//
+// What bounds it: every gathered element crosses L2 -> shared memory once per row-block and feeds
+// only d multiply-adds per token, so the operand traffic per flop is 1/d of a byte: the kernel
+// pays off for tall blocks and high compression, where the zero-expanded dense route spends its
+// time multiplying zeros.
+#include "bsp_tc.cuh"
+
+namespace bsp {
+
+int check_linear_args(const void* a, const void* b, const void* c, int n_out, int k_in, int block,
+                      const void* X, int tokens, int ldx, int act, const void* Y, int ldy);
+
+using namespace tc;
+
+namespace {
+
+constexpr int kGThreads = 288;              // 4 producer warps, MMA warp, 4 epilogue warps
+constexpr int kGProducers = 128;
+constexpr int kGStageK = 64;                // kept columns per pipeline stage
+constexpr int kGStageA = kGStageK * kBlockM * 2;   // 16 KB: 64 rows of 128 tokens
+constexpr int kGPrefetch = 8;               // stages ahead that the column numbers are pulled into L1
+
+template <int D>
+struct GatherCfg {
+  static constexpr int kStageB = D * 128;                       // d rows of 64 bf16
+  static constexpr int kStage = kGStageA + kStageB;
+  static constexpr int kFixed = 1024 /*alignment slack*/ + 512 /*barriers, stage bytes*/;
+  static constexpr int kStagesRaw = (kSmemLimit - kFixed) / kStage;
+  static constexpr int kStages = kStagesRaw > 12 ? 12 : kStagesRaw;
+  static constexpr int kTmemCols = 2 * D < 32 ? 32 : 2 * D;     // 32, 64, 128, 256
+  static constexpr int kSmemBytes = kStages * kStage + kFixed;
+};
+
+// Layout of a gather plan in device memory (all regions 256-byte aligned):
+//   soff  int32 [n_blocks + 1]   first stage of every row-block
+//   meta  uint8 [stages]         bits 0-2: real 16-column groups (1..4), bit 4: first stage of its
+//                                row-block, bit 5: last stage
+//   cols  int16 [stages][64]     column of X for row r of the stage at slot (r & 7) * 8 + (r >> 3)
+//                                (a producer thread's eight rows are adjacent); -1 = zero row,
+//                                -2 = beyond the real groups (not loaded, not multiplied)
+//   tiles bf16  [stages][d][64]  weight tile, row n at byte n*128, 16-byte chunk c at (c ^ (n & 7))
+struct GatherLayout {
+  size_t soff_off, meta_off, cols_off, tiles_off, total;
+  long long max_stages;
+};
+inline GatherLayout gather_layout(int n_out, int k_in, int block) {
+  GatherLayout L;
+  const long long nb = n_out / block;
+  L.max_stages = nb * ((k_in + kGStageK - 1) / kGStageK);      // every row-block has at least one stage
+  if (L.max_stages < nb) L.max_stages = nb;
+  L.soff_off = 0;
+  L.meta_off = round_up(sizeof(int32_t) * static_cast<size_t>(nb + 1), 256);
+  L.cols_off = L.meta_off + round_up(static_cast<size_t>(L.max_stages) + 256, 256);
+  L.tiles_off = L.cols_off + round_up(static_cast<size_t>(L.max_stages + kGPrefetch + 1) * kGStageK * 2, 256);
+  L.total = L.tiles_off + round_up(static_cast<size_t>(L.max_stages) * block * 128, 256);
+  return L;
+}
+
+// ---- plan construction -------------------------------------------------------------------
+// soff[b] = number of stages of the row-blocks before b (one CTA, a running block-wide scan).
+__global__ void __launch_bounds__(1024)
+gather_plan_scan_kernel(const int32_t* __restrict__ blk_ptr, int n_blocks, int32_t* __restrict__ soff) {
+  __shared__ int s_warp[32];
+  int running = 0;
+  for (int b0 = 0; b0 < n_blocks; b0 += blockDim.x) {
+    const int b = b0 + threadIdx.x;
+    int mine = 0;
+    if (b < n_blocks) {
+      const int kc = blk_ptr[b + 1] - blk_ptr[b];
+      mine = kc > 0 ? (kc + kGStageK - 1) / kGStageK : 1;
+    }
+    int total;
+    const int before = running + block_exclusive_scan(mine, s_warp, &total);
+    if (b < n_blocks) soff[b] = before;
+    running += total;
+  }
+  if (threadIdx.x == 0) soff[n_blocks] = running;
+}
+
+// One CTA per row-block: meta bytes, permuted column numbers and swizzled weight tiles of its stages.
+__global__ void __launch_bounds__(256)
+gather_plan_fill_kernel(const int32_t* __restrict__ blk_ptr, const int32_t* __restrict__ idx,
+                        const uint16_t* __restrict__ vals, int block, const int32_t* __restrict__ soff,
+                        uint8_t* __restrict__ meta, int16_t* __restrict__ cols, uint16_t* __restrict__ tiles) {
+  const int b = blockIdx.x;
+  const int lo = blk_ptr[b], kc = blk_ptr[b + 1] - lo;
+  const int g0 = soff[b], n_st = soff[b + 1] - g0;
+  const uint16_t* tile = vals + static_cast<size_t>(block) * lo;        // [block][kc]
+  for (int s = threadIdx.x; s < n_st; s += blockDim.x) {
+    const int left = kc - s * kGStageK;                                  // real columns from this stage on
+    int groups = left <= 0 ? 1 : (left >= kGStageK ? 4 : (left + 15) / 16);
+    meta[g0 + s] = static_cast<uint8_t>(groups | (s == 0 ? 0x10 : 0) | (s == n_st - 1 ? 0x20 : 0));
+  }
+  for (int e = threadIdx.x; e < n_st * kGStageK; e += blockDim.x) {
+    const int s = e / kGStageK, r = e % kGStageK;
+    const int k = s * kGStageK + r;
+    const int left = kc - s * kGStageK;
+    const int groups = left <= 0 ? 1 : (left >= kGStageK ? 4 : (left + 15) / 16);
+    int16_t c = -2;
+    if (r < groups * 16) c = k < kc ? static_cast<int16_t>(idx[lo + k]) : static_cast<int16_t>(-1);
+    cols[static_cast<size_t>(g0 + s) * kGStageK + (r & 7) * 8 + (r >> 3)] = c;
+  }
+  // weight tiles: one thread per 16-byte chunk (8 columns of one row)
+  const int chunks = n_st * block * 8;
+  for (int e = threadIdx.x; e < chunks; e += blockDim.x) {
+    const int s = e / (block * 8), rem = e % (block * 8);
+    const int n = rem >> 3, ch = rem & 7;
+    uint32_t w[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int k0 = s * kGStageK + ch * 8 + 2 * i;
+      const uint32_t v0 = k0 < kc ? tile[static_cast<size_t>(n) * kc + k0] : 0u;
+      const uint32_t v1 = k0 + 1 < kc ? tile[static_cast<size_t>(n) * kc + k0 + 1] : 0u;
+      w[i] = v0 | (v1 << 16);
+    }
+    uint16_t* dst = tiles + (static_cast<size_t>(g0 + s) * block + n) * 64 + ((ch ^ (n & 7)) << 3);
+    *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
+  }
+}
+
+// ---- transposed copy ---------------------------------------------------------------------
+// XT[c, r] = X[r, c] for a row-major bf16 matrix; 64 x 64 tiles through shared memory, 16-byte
+// global accesses on both sides (rows and cols multiples of 8).
+__global__ void __launch_bounds__(256)
+transpose_kernel(const uint16_t* __restrict__ X, int rows, int cols, int ldx, uint16_t* __restrict__ XT, int ldxt) {
+  __shared__ uint16_t s_t[64][66];
+  const int r0 = blockIdx.y * 64, c0 = blockIdx.x * 64;
+  for (int e = threadIdx.x; e < 512; e += 256) {
+    const int r = e >> 3, q = e & 7;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (r0 + r < rows && c0 + q * 8 < cols) v = __ldg(reinterpret_cast<const uint4*>(X + static_cast<size_t>(r0 + r) * ldx + c0 + q * 8));
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      s_t[r][q * 8 + 2 * i] = static_cast<uint16_t>(w[i] & 0xffffu);
+      s_t[r][q * 8 + 2 * i + 1] = static_cast<uint16_t>(w[i] >> 16);
+    }
+  }
+  __syncthreads();
+  for (int e = threadIdx.x; e < 512; e += 256) {
+    const int c = e >> 3, q = e & 7;             // output row c (a column of X), 8 source rows q*8..q*8+7
+    if (c0 + c < cols && r0 + q * 8 < rows) {
+      uint32_t w[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        w[i] = static_cast<uint32_t>(s_t[q * 8 + 2 * i][c]) | (static_cast<uint32_t>(s_t[q * 8 + 2 * i + 1][c]) << 16);
+      *reinterpret_cast<uint4*>(XT + static_cast<size_t>(c0 + c) * ldxt + r0 + q * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+  }
+}
+
+// ---- the kernel --------------------------------------------------------------------------
+struct GatherParams {
+  const uint16_t* XT;
+  int ldxt, tokens, n_out, act;
+  const uint16_t* bias;
+  uint16_t* Y;
+  int ldy;
+  const int32_t* soff;
+  const uint8_t* meta;
+  const int16_t* cols;
+  const uint16_t* tiles;
+  int n_blocks, m_tiles, n_chunks, rb_per_chunk;
+  int* status;
+};
+
+// MN-major operand tile with the 128-byte swizzle: 8-row atoms 1024 bytes apart along the
+// contraction, the two 64-token halves of the tile 8 KB apart.
+__device__ __forceinline__ uint64_t gather_desc_a(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((smem_addr & 0x3ffff) >> 4);
+  d |= static_cast<uint64_t>((kGStageK * 128) >> 4) << 16;      // leading byte offset / 16
+  d |= static_cast<uint64_t>(1024 >> 4) << 32;                   // stride byte offset / 16
+  d |= static_cast<uint64_t>(1) << 46;
+  d |= static_cast<uint64_t>(2) << 61;
+  return d;
+}
+// bf16 x bf16 -> float32, A MN-major (bit 15), B K-major, M = 128, N = d.
+__host__ __device__ constexpr uint32_t gather_idesc(int d) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (static_cast<uint32_t>(d >> 3) << 17) |
+         (static_cast<uint32_t>(kBlockM >> 4) << 24);
+}
+__device__ __forceinline__ void tmem_load_16cols(uint32_t taddr, uint32_t (&v)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+      : "r"(taddr)
+      : "memory");
+}
+
+template <int D>
+__global__ void __launch_bounds__(kGThreads, 1)
+linear_gather_kernel(const __grid_constant__ GatherParams P) {
+  using Cfg = GatherCfg<D>;
+  constexpr int S = Cfg::kStages;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+  // [S stages: A 16 KB, B D*128][mbarriers][stage bytes][TMEM base]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S * Cfg::kStage);
+  // bars[0..S) full, [S..2S) empty, [2S..2S+2) accumulator full, [2S+2..2S+4) accumulator empty
+  uint8_t* s_meta = reinterpret_cast<uint8_t*>(bars + 2 * S + 4);
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(s_meta + 16);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t smem_base = smem_u32(smem);
+  const uint32_t bar_base = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (S + s); };
+  auto acc_full_bar = [&](int a) { return bar_base + 8u * (2 * S + a); };
+  auto acc_empty_bar = [&](int a) { return bar_base + 8u * (2 * S + 2 + a); };
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), kGProducers + 1); mbar_init(empty_bar(s), 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(acc_full_bar(a), 1); mbar_init(acc_empty_bar(a), 4); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 4) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_holder)),
+                 "r"(static_cast<uint32_t>(Cfg::kTmemCols)) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tcgen05_fence_before();
+  __syncthreads();
+  tcgen05_fence_after();
+  const uint32_t tmem_base = *tmem_holder;
+
+  const int total_units = P.m_tiles * P.n_chunks;
+
+  if (warp < 4) {
+    // ---------------------------------------------------------------- producers
+    const int pt = threadIdx.x;                   // 0..127
+    const int chunk = pt & 15, r0 = pt >> 4;      // 16-byte token chunk, row residue mod 8
+    const uint32_t dst_thread = static_cast<uint32_t>((chunk >> 3) * (kGStageK * 128) + r0 * 128 + (((chunk & 7) ^ r0) << 4));
+    int stage = 0;
+    uint32_t phase = 0;
+    bool ok = true;
+    for (int unit = blockIdx.x; unit < total_units && ok; unit += gridDim.x) {
+      const int m = unit / P.n_chunks, ch = unit - m * P.n_chunks;
+      const int rb0 = ch * P.rb_per_chunk, rb1 = min(P.n_blocks, rb0 + P.rb_per_chunk);
+      const int g_begin = __ldg(P.soff + rb0), g_end = __ldg(P.soff + rb1);
+      const int tok = m * kBlockM + chunk * 8;
+      const uint32_t src_bytes = tok < P.tokens ? 16u : 0u;
+      const uint16_t* src_col0 = P.XT + (src_bytes ? tok : 0);
+      if (pt < kGPrefetch)
+        asm volatile("prefetch.global.L1 [%0];" ::"l"(P.cols + static_cast<size_t>(g_begin + pt) * kGStageK));
+      for (int g = g_begin; g < g_end; ++g) {
+        if (!mbar_wait(empty_bar(stage), phase ^ 1u)) { ok = false; break; }
+        const uint32_t a_dst = smem_base + stage * Cfg::kStage;
+        if (pt == 0) {
+          s_meta[stage] = __ldg(P.meta + g);
+          mbar_arrive_expect_tx(full_bar(stage), Cfg::kStageB);
+          asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                       ::"r"(a_dst + kGStageA), "l"(reinterpret_cast<uint64_t>(P.tiles + static_cast<size_t>(g) * D * 64)),
+                         "r"(static_cast<uint32_t>(Cfg::kStageB)), "r"(full_bar(stage))
+                       : "memory");
+          asm volatile("prefetch.global.L1 [%0];" ::"l"(P.cols + static_cast<size_t>(g + kGPrefetch) * kGStageK));
+          asm volatile("prefetch.global.L1 [%0];" ::"l"(P.meta + g + 128));
+        }
+        const uint4 cv = __ldg(reinterpret_cast<const uint4*>(P.cols + static_cast<size_t>(g) * kGStageK + r0 * 8));
+        const uint32_t cw[4] = {cv.x, cv.y, cv.z, cv.w};
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const int col = static_cast<int16_t>((cw[i >> 1] >> (16 * (i & 1))) & 0xffffu);
+          if (col != -2) {
+            const uint16_t* src = col >= 0 ? src_col0 + static_cast<size_t>(col) * P.ldxt : P.XT;
+            const uint32_t sz = col >= 0 ? src_bytes : 0u;
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;"
+                         ::"r"(a_dst + dst_thread + static_cast<uint32_t>(i) * 1024u), "l"(src), "r"(sz) : "memory");
+          }
+        }
+        asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(full_bar(stage)) : "memory");
+        if (++stage == S) { stage = 0; phase ^= 1u; }
+      }
+    }
+    if (!ok) atomicExch(P.status, BSP_ERR_TIMEOUT);
+    asm volatile("cp.async.wait_all;" ::: "memory");
+  } else if (warp == 4) {
+    // ---------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = gather_idesc(D);
+      int stage = 0;
+      uint32_t phase = 0;
+      uint32_t acc_phase[2] = {0u, 0u};
+      int acc = 0;
+      bool ok = true;
+      for (int unit = blockIdx.x; unit < total_units && ok; unit += gridDim.x) {
+        const int m = unit / P.n_chunks, ch = unit - m * P.n_chunks;
+        const int rb0 = ch * P.rb_per_chunk, rb1 = min(P.n_blocks, rb0 + P.rb_per_chunk);
+        const int g_begin = __ldg(P.soff + rb0), g_end = __ldg(P.soff + rb1);
+        for (int g = g_begin; g < g_end; ++g) {
+          if (!mbar_wait(full_bar(stage), phase)) { ok = false; break; }
+          tcgen05_fence_after();
+          const uint32_t mt = s_meta[stage];
+          const int groups = static_cast<int>(mt & 7u);
+          const bool first = (mt & 0x10u) != 0, last = (mt & 0x20u) != 0;
+          if (first) {
+            if (!mbar_wait(acc_empty_bar(acc), acc_phase[acc] ^ 1u)) { ok = false; break; }
+            tcgen05_fence_after();
+          }
+          const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * D);
+          const uint32_t a_addr = smem_base + stage * Cfg::kStage;
+          const uint32_t b_addr = a_addr + kGStageA;
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            if (k < groups)
+              tcgen05_mma_bf16(d_tmem, gather_desc_a(a_addr + k * 2048), smem_desc_sw128(b_addr + k * 32), idesc,
+                               (first && k == 0) ? 0u : 1u);
+          }
+          tcgen05_commit(empty_bar(stage));
+          if (last) {
+            tcgen05_commit(acc_full_bar(acc));
+            acc_phase[acc] ^= 1u;
+            acc ^= 1;
+          }
+          if (++stage == S) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) atomicExch(P.status, BSP_ERR_TIMEOUT);
+    }
+  } else {
+    // ---------------------------------------------------------------- epilogue
+    const int quad = warp & 3;               // TMEM lanes [32*quad, 32*quad+32) belong to this warp
+    uint32_t acc_phase[2] = {0u, 0u};
+    int acc = 0;
+    bool ok = true;
+    for (int unit = blockIdx.x; unit < total_units && ok; unit += gridDim.x) {
+      const int m = unit / P.n_chunks, ch = unit - m * P.n_chunks;
+      const int rb0 = ch * P.rb_per_chunk, rb1 = min(P.n_blocks, rb0 + P.rb_per_chunk);
+      const int t = m * kBlockM + quad * 32 + lane;
+      uint16_t* yrow = P.Y + static_cast<size_t>(t) * P.ldy;
+      for (int rb = rb0; rb < rb1; ++rb) {
+        if (!mbar_wait(acc_full_bar(acc), acc_phase[acc])) { ok = false; break; }
+        tcgen05_fence_after();
+        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + static_cast<uint32_t>(acc * D);
+        constexpr int kPiece = 16;
+#pragma unroll
+        for (int c0 = 0; c0 < D; c0 += kPiece) {
+          uint32_t v[16];
+          tmem_load_16cols(taddr + c0, v);
+          uint4 bv[2] = {make_uint4(0u, 0u, 0u, 0u), make_uint4(0u, 0u, 0u, 0u)};
+          if (P.bias != nullptr) {
+            const uint4* bp = reinterpret_cast<const uint4*>(P.bias + static_cast<size_t>(rb) * D + c0);
+            bv[0] = __ldg(bp);
+            bv[1] = __ldg(bp + 1);
+          }
+          tmem_load_wait();
+          if (c0 + kPiece >= D) {              // this warp's last read of the accumulator
+            tcgen05_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acc_empty_bar(acc));
+          }
+          const uint32_t bw[8] = {bv[0].x, bv[0].y, bv[0].z, bv[0].w, bv[1].x, bv[1].y, bv[1].z, bv[1].w};
+          float f[16];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            f[2 * i] = __uint_as_float(v[2 * i]) + __uint_as_float(bw[i] << 16);
+            f[2 * i + 1] = __uint_as_float(v[2 * i + 1]) + __uint_as_float(bw[i] & 0xffff0000u);
+          }
+          if (P.act == BSP_ACT_GELU) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) f[i] = gelu_erf(f[i]);
+          }
+          if (t < P.tokens) {
+            uint4* out = reinterpret_cast<uint4*>(yrow + static_cast<size_t>(rb) * D + c0);
+            out[0] = make_uint4(pack_bf16x2(f[0], f[1]), pack_bf16x2(f[2], f[3]), pack_bf16x2(f[4], f[5]), pack_bf16x2(f[6], f[7]));
+            out[1] = make_uint4(pack_bf16x2(f[8], f[9]), pack_bf16x2(f[10], f[11]), pack_bf16x2(f[12], f[13]), pack_bf16x2(f[14], f[15]));
+          }
+        }
+        acc_phase[acc] ^= 1u;
+        acc ^= 1;
+      }
+    }
+    if (!ok && lane == 0) atomicExch(P.status, BSP_ERR_TIMEOUT);
+  }
+
+  tcgen05_fence_before();
+  __syncthreads();
+  if (warp == 4) {
+    tcgen05_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                 "r"(static_cast<uint32_t>(Cfg::kTmemCols)) : "memory");
+  }
+}
+
+template <int D>
+int launch_gather(TcDevice* dev, int slot, const GatherParams& P, cudaStream_t s) {
+  using Cfg = GatherCfg<D>;
+  static_assert(Cfg::kStages >= 4, "pipeline too shallow");
+  static bool attr_set[64] = {};
+  int device = 0;
+  BSP_CUDA_TRY(cudaGetDevice(&device));
+  if (device < 0 || device >= 64) return BSP_ERR_CUDA;
+  if (!attr_set[device]) {
+    BSP_CUDA_TRY(cudaFuncSetAttribute(linear_gather_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes));
+    attr_set[device] = true;
+  }
+  (void)slot;
+  const int units = P.m_tiles * P.n_chunks;
+  const int grid = units < dev->sms ? units : dev->sms;
+  linear_gather_kernel<D><<<grid, kGThreads, Cfg::kSmemBytes, s>>>(P);
+  BSP_LAUNCH_CHECK();
+  return BSP_OK;
+}
+
+bool gather_block_ok(int block) { return block == 16 || block == 32 || block == 64 || block == 128; }
+
+}  // namespace
+}  // namespace bsp
+
+extern "C" int bsp_linear_gather_plan_bytes(int n_out, int k_in, int block, size_t* bytes) {
+  using namespace bsp;
+  if (n_out <= 0 || k_in <= 0 || block <= 0 || bytes == nullptr) return BSP_ERR_ARG;
+  if (n_out % block) return BSP_ERR_SHAPE;
+  if (!gather_block_ok(block) || k_in > 32767) return BSP_ERR_UNSUPPORTED;
+  *bytes = gather_layout(n_out, k_in, block).total;
+  return BSP_OK;
+}
+
+extern "C" int bsp_linear_gather_plan(const int32_t* blk_ptr, const int32_t* idx, const void* vals, int n_out,
+                                      int k_in, int block, void* gplan, size_t gplan_bytes, void* stream) {
+  using namespace bsp;
+  if (blk_ptr == nullptr || idx == nullptr || vals == nullptr || gplan == nullptr) return BSP_ERR_ARG;
+  size_t need;
+  int st = bsp_linear_gather_plan_bytes(n_out, k_in, block, &need);
+  if (st != BSP_OK) return st;
+  if (!aligned_to(gplan, 256)) return BSP_ERR_ARG;
+  if (gplan_bytes < need) return BSP_ERR_WORKSPACE;
+  const GatherLayout L = gather_layout(n_out, k_in, block);
+  char* base = static_cast<char*>(gplan);
+  const int nb = n_out / block;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int32_t* soff = reinterpret_cast<int32_t*>(base + L.soff_off);
+  gather_plan_scan_kernel<<<1, 1024, 0, s>>>(blk_ptr, nb, soff);
+  BSP_LAUNCH_CHECK();
+  gather_plan_fill_kernel<<<nb, 256, 0, s>>>(blk_ptr, idx, static_cast<const uint16_t*>(vals), block, soff,
+                                             reinterpret_cast<uint8_t*>(base + L.meta_off),
+                                             reinterpret_cast<int16_t*>(base + L.cols_off),
+                                             reinterpret_cast<uint16_t*>(base + L.tiles_off));
+  BSP_LAUNCH_CHECK();
+  return BSP_OK;
+}
+
+extern "C" int bsp_transpose(const void* X, int rows, int cols, int ldx, void* XT, int ldxt, void* stream) {
+  using namespace bsp;
+  if (X == nullptr || XT == nullptr || rows < 0 || cols <= 0) return BSP_ERR_ARG;
+  if (ldx < cols || ldxt < rows) return BSP_ERR_SHAPE;
+  if (rows % 8 || cols % 8 || ldx % 8 || ldxt % 8 || !aligned_to(X, 16) || !aligned_to(XT, 16)) return BSP_ERR_UNSUPPORTED;
+  if (rows == 0) return BSP_OK;
+  const dim3 grid((cols + 63) / 64, (rows + 63) / 64);
+  if (grid.y > 65535) return BSP_ERR_UNSUPPORTED;
+  transpose_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<const uint16_t*>(X), rows, cols, ldx,
+                                                                        static_cast<uint16_t*>(XT), ldxt);
+  BSP_LAUNCH_CHECK();
+  return BSP_OK;
+}
+
+extern "C" int bsp_linear_gathered(const void* gplan, int n_out, int k_in, int block, const void* XT, int tokens,
+                                   int ldxt, const void* bias, int act, void* Y, int ldy, void* stream) {
+  using namespace bsp;
+  if (gplan == nullptr || XT == nullptr || Y == nullptr) return BSP_ERR_ARG;
+  if (n_out <= 0 || k_in <= 0 || block <= 0 || tokens < 0) return BSP_ERR_ARG;
+  if (act != BSP_ACT_NONE && act != BSP_ACT_GELU) return BSP_ERR_ARG;
+  if (n_out % block) return BSP_ERR_SHAPE;
+  if (ldxt < tokens || ldy < n_out) return BSP_ERR_SHAPE;
+  if (!gather_block_ok(block) || k_in > 32767) return BSP_ERR_UNSUPPORTED;
+  if (!aligned_to(gplan, 256) || !aligned_to(XT, 16) || !aligned_to(Y, 16) || (bias != nullptr && !aligned_to(bias, 16)) ||
+      tokens % 8 || ldxt % 8 || ldy % 8)
+    return BSP_ERR_UNSUPPORTED;
+  if (tokens == 0) return BSP_OK;
+  TcDevice* dev = tc_device();
+  if (dev == nullptr) return BSP_ERR_CUDA;
+  const GatherLayout L = gather_layout(n_out, k_in, block);
+  const char* base = static_cast<const char*>(gplan);
+  GatherParams P;
+  P.XT = static_cast<const uint16_t*>(XT);
+  P.ldxt = ldxt;
+  P.tokens = tokens;
+  P.n_out = n_out;
+  P.act = act;
+  P.bias = static_cast<const uint16_t*>(bias);
+  P.Y = static_cast<uint16_t*>(Y);
+  P.ldy = ldy;
+  P.soff = reinterpret_cast<const int32_t*>(base + L.soff_off);
+  P.meta = reinterpret_cast<const uint8_t*>(base + L.meta_off);
+  P.cols = reinterpret_cast<const int16_t*>(base + L.cols_off);
+  P.tiles = reinterpret_cast<const uint16_t*>(base + L.tiles_off);
+  P.n_blocks = n_out / block;
+  P.m_tiles = (tokens + kBlockM - 1) / kBlockM;
+  // runs of consecutive row-blocks: enough units for about six per SM, runs as long as that allows
+  int n_chunks = (6 * dev->sms + P.m_tiles - 1) / P.m_tiles;
+  if (n_chunks < 1) n_chunks = 1;
+  if (n_chunks > P.n_blocks) n_chunks = P.n_blocks;
+  P.rb_per_chunk = (P.n_blocks + n_chunks - 1) / n_chunks;
+  P.n_chunks = (P.n_blocks + P.rb_per_chunk - 1) / P.rb_per_chunk;
+  P.status = dev->status;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  switch (block) {
+    case 16: return launch_gather<16>(dev, 0, P, s);
+    case 32: return launch_gather<32>(dev, 1, P, s);
+    case 64: return launch_gather<64>(dev, 2, P, s);
+    default: return launch_gather<128>(dev, 3, P, s);
+  }
+}

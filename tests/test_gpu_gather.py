@@ -1,0 +1,131 @@
+"""GPU parity of the gathering linear layer (bsp_linear_gathered: only the kept columns of X are fetched
+and multiplied) and of bsp_transpose, against the oracle's masked dense product (float64).
+
+Tolerances as for the other linear kernels (gpu_util): max |err| / (||x|| ||w|| + |b|) <= 2e-2 and
+sum|err| / sum|ref| <= 5e-3; the transposed copy is bit-exact.
+"""
+import numpy as np
+import pytest
+import torch
+
+import paper_2009_08065_b200 as bsp
+import synth_inputs as si
+from oracle import bsp_oracle as O
+from gpu_util import DEV, assert_linear_close, bits_of, to_dev, upload_packed
+
+pytestmark = pytest.mark.gpu
+
+
+def oracle_linear(x, wp, b, act):
+    m = O.mask_of(wp)
+    return O.linear_masked_dense(x, wp, m, b, act), O.row_scales(x, wp, m, b)
+
+
+def run_gathered(wp, d, x, b, act):
+    """prune/pack on the GPU -> gather plan -> transposed activations -> bsp_linear_gathered."""
+    N, K = wp.shape
+    T = x.shape[0]
+    pk = bsp.PackedMatrix.allocate(N, K, d, bsp.ORIENT_C, DEV)
+    bsp.bsp_prune_pack(to_dev(wp), pk, 0.0)
+    gplan = torch.empty(bsp.bsp_linear_gather_plan_bytes(N, K, d), dtype=torch.uint8, device=DEV)
+    bsp.bsp_linear_gather_plan(pk, gplan)
+    xd = to_dev(x)
+    xt = torch.full((K, T), 0x7FC0, dtype=torch.int16, device=DEV)
+    bsp.bsp_transpose(xd, xt)
+    y = torch.full((T, N), 0x7FC0, dtype=torch.int16, device=DEV)          # NaN pattern: every output must be written
+    bsp.bsp_linear_gathered(gplan, N, K, d, xt, None if b is None else to_dev(b), act, y)
+    bsp.bsp_linear_status()
+    torch.cuda.synchronize()
+    return bits_of(y), bits_of(xt)
+
+
+@pytest.mark.parametrize("rows,cols", [(8, 8), (200, 72), (136, 320), (1024, 768)])
+def test_transpose_is_bit_exact(rows, cols):
+    x = si.make_activations(31, f"tr{rows}x{cols}", rows, cols)
+    xt = torch.zeros((cols, rows), dtype=torch.int16, device=DEV)
+    bsp.bsp_transpose(to_dev(x), xt)
+    torch.cuda.synchronize()
+    assert np.array_equal(bits_of(xt), np.ascontiguousarray(x.T))
+
+
+@pytest.mark.parametrize("act", [0, 1])
+@pytest.mark.parametrize("d,rate", [(16, 2.0), (32, 3.0), (64, 5.0), (128, 8.0)])
+def test_gathered_linear_fixed_keep_count(d, rate, act):
+    """Several token tiles with a ragged last one, several row-blocks per run, kept counts that are not
+    multiples of the 16-column step (K = 712: 356, 237, 142, 89 kept columns per block)."""
+    T, N, K = 328, 512, 712
+    spec = si.LinearSpec(f"gath{d}", N, K, bool(act), rate, d)
+    wp, _ = si.make_pruned_weight(41, spec)
+    x = si.make_activations(41, spec.name, T, K)
+    b = si.make_bias(41, spec)
+    y_ref, scales = oracle_linear(x, wp, b, act)
+    y, xt = run_gathered(wp, d, x, b, act)
+    assert np.array_equal(xt, np.ascontiguousarray(x.T))
+    assert_linear_close(y, y_ref, scales, f"gathered d={d} rate={rate} act={act}")
+
+
+def test_gathered_linear_uneven_blocks_and_empty_blocks():
+    """Threshold pruning of heavy-tailed weights: every row-block keeps a different number of columns;
+    two blocks keep nothing (their outputs are act(b)), one keeps everything, one keeps a single column."""
+    T, N, K, d = 136, 384, 456, 32
+    spec = si.LinearSpec("gath_uneven", N, K, True, 2.0, d)
+    w = si.make_weight(43, spec, "student_t3")
+    t_b = float(np.quantile(O.group_norms(w, d, "C"), 0.6))
+    keep = O.keep_flags(w, d, "C", t_b)
+    keep[1, :] = False
+    keep[7, :] = False
+    keep[4, :] = True
+    keep[9, :] = False
+    keep[9, 100] = True
+    wp = si.zero_groups(w, keep, d, "C")
+    x = si.make_activations(43, spec.name, T, K)
+    b = si.make_bias(43, spec)
+    for act in (0, 1):
+        y_ref, scales = oracle_linear(x, wp, b, act)
+        y, _ = run_gathered(wp, d, x, b, act)
+        assert_linear_close(y, y_ref, scales, f"gathered uneven act={act}")
+    # nothing kept at all and no bias: exact zeros
+    y, _ = run_gathered(np.zeros_like(wp), d, x, None, 0)
+    assert not (y & 0x7FFF).any()
+
+
+def test_gathered_linear_oracle_made_pack_and_dense_route_agree():
+    """The packed form is the contract: a pack made by the oracle drives the gather plan, and the result
+    agrees with the zero-expanded dense route on the same inputs."""
+    T, N, K, d = 256, 256, 512, 64
+    spec = si.LinearSpec("gath_opk", N, K, False, 3.0, d)
+    wp, keep = si.make_pruned_weight(44, spec)
+    x = si.make_activations(44, spec.name, T, K)
+    b = si.make_bias(44, spec)
+    blk_ptr, idx, vals = O.pack(wp, keep, d, "C")
+    pk = upload_packed(blk_ptr, idx, vals, N, K, d)
+    gplan = torch.empty(bsp.bsp_linear_gather_plan_bytes(N, K, d), dtype=torch.uint8, device=DEV)
+    bsp.bsp_linear_gather_plan(pk, gplan)
+    xd, bd = to_dev(x), to_dev(b)
+    xt = torch.empty((K, T), dtype=torch.int16, device=DEV)
+    bsp.bsp_transpose(xd, xt)
+    y = torch.full((T, N), 0x7FC0, dtype=torch.int16, device=DEV)
+    bsp.bsp_linear_gathered(gplan, N, K, d, xt, bd, 0, y)
+    y2 = torch.full((T, N), 0x7FC0, dtype=torch.int16, device=DEV)
+    ws = torch.empty(bsp.bsp_linear_plan_bytes(N, K, d), dtype=torch.uint8, device=DEV)
+    bsp.bsp_linear(pk, xd, bd, 0, y2, ws)
+    bsp.bsp_linear_status()
+    torch.cuda.synchronize()
+    y_ref, scales = oracle_linear(x, wp, b, 0)
+    assert_linear_close(bits_of(y), y_ref, scales, "gathered, oracle pack")
+    assert_linear_close(bits_of(y2), y_ref, scales, "dense route, oracle pack")
+
+
+def test_gathered_linear_bert_large_shape_sampled_rows():
+    """A sweep point of the BERT-large workload at full width (hidden 1024 -> 4096, 64-row blocks, 5x) with
+    4096 tokens: many units per CTA, long runs of row-blocks; the oracle checks a sample of token rows."""
+    T, N, K, d, rate = 4096, 4096, 1024, 64, 5.0
+    spec = si.LinearSpec("gath_large", N, K, True, rate, d)
+    wp, _ = si.make_pruned_weight(45, spec)
+    x = si.make_activations(45, spec.name, T, K)
+    b = si.make_bias(45, spec)
+    y, _ = run_gathered(wp, d, x, b, 1)
+    rows = np.sort(np.random.default_rng(45).choice(T, size=48, replace=False))
+    y_ref, scales = oracle_linear(x[rows], wp, b, 1)
+    assert_linear_close(y[rows], y_ref, scales, "gathered BERT-large FFN-up sample")
+    assert np.isfinite(O.bf16_to_f64(y)).all()
