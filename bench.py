@@ -519,6 +519,83 @@ def run_case(args):
     print(f"case {args.case}: 4 launches done")
 
 
+def run_sweep(args):
+    """The BERT-large sweep (hidden 1024, FFN 4096, tokens 32768 by default): compression 1.5/2/3/5/8 x block height
+    8/16/32/64 on the four linear shapes.  For every point: the zero-expanded dense route (bsp_linear_planned), the
+    gathering kernel (bsp_linear_gathered, block heights it takes; X transposed beforehand, that copy timed
+    separately once per input width), and torch.matmul on the dense shape as context.  L2 is flushed (256 MiB
+    written) before every timed launch; medians of `--steps` launches.  One JSON line per point."""
+    import torch
+    import paper_2009_08065_b200 as bsp
+    torch.cuda.set_device(0)
+    device = torch.device("cuda", 0)
+    peaks, _ = measured_peaks()
+    peak = float(peaks["bf16_tflops"])
+    T = args.sweep_tokens
+    iters = max(3, min(args.steps, 20))
+    shapes = [("qkv", 3072, 1024, 0), ("attn_out", 1024, 1024, 0), ("ffn_up", 4096, 1024, 1), ("ffn_down", 1024, 4096, 0)]
+    if args.sweep_shapes:
+        shapes = [sh for sh in shapes if sh[0] in args.sweep_shapes.split(",")]
+    gen = torch.Generator(device=device)
+    gen.manual_seed(si.DEFAULT_SEED)
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=device)
+
+    def timed(fn):
+        ms = []
+        for i in range(iters + 2):
+            flush.zero_()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            fn()
+            b.record()
+            torch.cuda.synchronize()
+            if i >= 2:
+                ms.append(a.elapsed_time(b))
+        return statistics.median(ms)
+
+    for name, N, K, act in shapes:
+        X = torch.randn(T, K, device=device, generator=gen).to(torch.bfloat16)
+        XT = torch.empty(K, T, dtype=torch.bfloat16, device=device)
+        t_tr = timed(lambda: bsp.bsp_transpose(X, XT))
+        bias = (torch.randn(N, device=device, generator=gen) * 0.02).to(torch.bfloat16)
+        Y = torch.empty(T, N, dtype=torch.bfloat16, device=device)
+        Yg = torch.empty(T, N, dtype=torch.bfloat16, device=device)
+        Wd = (torch.randn(N, K, device=device, generator=gen) * 0.02).to(torch.bfloat16)
+        t_dense = timed(lambda: torch.matmul(X, Wd.t()))
+        for d in (8, 16, 32, 64):
+            for c in (1.5, 2.0, 3.0, 5.0, 8.0):
+                kc = int(round(K / c))
+                scores = torch.rand(N // d, K, device=device, generator=gen)
+                keep = torch.zeros(N // d, K, dtype=torch.bool, device=device)
+                keep.scatter_(1, scores.topk(kc, dim=1).indices, True)
+                W = (Wd.view(N // d, d, K) * keep[:, None, :]).view(N, K).contiguous()
+                pk = bsp.PackedMatrix.allocate(N, K, d, bsp.ORIENT_C, device)
+                bsp.bsp_prune_pack(W, pk, 0.0)
+                plan = torch.empty(bsp.bsp_linear_plan_bytes(N, K, d), dtype=torch.uint8, device=device)
+                bsp.bsp_linear_plan(pk, plan)
+                nz = 2.0 * T * d * kc * (N // d)
+                t_plan = timed(lambda: bsp.bsp_linear_planned(plan, N, K, d, X, bias, act, Y))
+                point = {"sweep": "bert_large", "shape": name, "tokens": T, "n_out": N, "k_in": K, "block": d,
+                         "compression": c, "kept_per_block": kc, "nonzero_gflop": round(nz / 1e9, 2),
+                         "dense_route_ms": round(t_plan, 4), "dense_route_nonzero_tflops": round(nz / t_plan / 1e9, 1),
+                         "torch_dense_ms": round(t_dense, 4), "torch_dense_tflops": round(2.0 * T * N * K / t_dense / 1e9, 1),
+                         "transpose_ms": round(t_tr, 4)}
+                best = nz / t_plan / 1e9
+                if d in (16, 32, 64, 128):
+                    gplan = torch.empty(bsp.bsp_linear_gather_plan_bytes(N, K, d), dtype=torch.uint8, device=device)
+                    bsp.bsp_linear_gather_plan(pk, gplan)
+                    t_g = timed(lambda: bsp.bsp_linear_gathered(gplan, N, K, d, XT, bias, act, Yg))
+                    diff = (Y.float() - Yg.float()).abs().max().item()
+                    point.update({"gather_ms": round(t_g, 4), "gather_nonzero_tflops": round(nz / t_g / 1e9, 1),
+                                  "gather_vs_dense_route": round(t_plan / t_g, 3), "max_abs_diff_between_routes": diff})
+                    best = max(best, nz / t_g / 1e9)
+                    del gplan
+                point["best_percent_of_bf16_peak"] = round(100.0 * best / peak, 2)
+                bsp.bsp_linear_status()
+                print(json.dumps(point), flush=True)
+                del plan, pk, W, keep, scores
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -527,8 +604,14 @@ def main():
     ap.add_argument("--impl", choices=["cuda", "reference"], default="cuda")
     ap.add_argument("--case", choices=["qkv", "attn_out", "ffn_up", "ffn_down", "prepare"], default=None,
                     help="run a few launches of one call for a profiler and exit")
+    ap.add_argument("--sweep", choices=["bert_large"], default=None,
+                    help="time the BERT-large compression x block-height grid and print one JSON line per point")
+    ap.add_argument("--sweep-tokens", type=int, default=32768)
+    ap.add_argument("--sweep-shapes", default=None, help="comma-separated subset of qkv,attn_out,ffn_up,ffn_down")
     args = ap.parse_args()
-    if args.case:
+    if args.sweep:
+        run_sweep(args)
+    elif args.case:
         run_case(args)
     elif args.impl == "reference":
         run_reference(args)

@@ -6,8 +6,11 @@
 // 128 tokens as the M side of a tcgen05.mma, the d output rows as its N side and the kept columns
 // as K.  Single columns of a row-major X are 2-byte pieces, useless for 16-byte copies, so the
 // activations are taken TRANSPOSED, XT [k_in, tokens]: a kept column is then a contiguous row of
-// 128 tokens (256 bytes), gathered with 16-byte cp.async copies straight into the tensor core's
-// "MN-major" operand layout (8-row atoms of 64 tokens x 8 columns, 128-byte swizzle).  The weight
+// 128 tokens (256 bytes), and TMA row gathers (tile::gather4: four rows of a 2-D tensor per
+// instruction, box one row high) bring the kept rows straight into the tensor core's "MN-major"
+// operand layout (8-row atoms of 64 tokens x 8 columns, 128-byte swizzle).  (A first version
+// gathered with 16-byte cp.async copies; the load/store unit's limit on requests in flight held
+// it to about 13 bytes per clock per SM.)  The weight
 // side comes from a gather plan made once per pruned matrix: per pipeline stage (64 kept columns)
 // the d x 64 tile already in the K-major 128-byte-swizzled layout (one bulk copy lands it), the
 // 64 column numbers, and a byte that says how many 16-column groups are real and whether the stage
@@ -15,9 +18,9 @@
 //
 // Kernel.  Persistent CTAs walk units of (128-token tile) x (run of consecutive row-blocks); the
 // stages of such a run are consecutive in the plan, so the producers just stream them.
-//   warps 0-3 : producers; thread = (16-byte token chunk, row residue mod 8); per stage 8 cp.async
-//               per thread, completion counted on the stage's mbarrier (arrive-on-completion);
-//               thread 0 also issues the bulk copy of the weight tile and hands the stage's byte on;
+//   warps 0-3 : producers, warp w filling every fourth stage; lane = (64-token half, four rows): one
+//               gather4 per lane per stage, completion bytes counted on the stage's mbarrier;
+//               lane 0 also issues the bulk copy of the weight tile and hands the stage's byte on;
 //   warp 4    : one lane issues tcgen05.mma (M=128, N=d, K=16) into one of two TMEM accumulators,
 //               commits stage release and, at the end of a row-block, accumulator ready;
 //   warps 5-8 : epilogue; each warp reads its 32 TMEM lanes (tokens), adds bias, optional GELU,
@@ -40,10 +43,10 @@ using namespace tc;
 namespace {
 
 constexpr int kGThreads = 288;              // 4 producer warps, MMA warp, 4 epilogue warps
-constexpr int kGProducers = 128;
 constexpr int kGStageK = 64;                // kept columns per pipeline stage
 constexpr int kGStageA = kGStageK * kBlockM * 2;   // 16 KB: 64 rows of 128 tokens
-constexpr int kGPrefetch = 8;               // stages ahead that the column numbers are pulled into L1
+constexpr int kGQueue = 12;                 // a producer warp loads its column numbers up to this many stages ahead
+constexpr int kGPrefetch = kGQueue;         // the plan's column array is padded by this many stages
 
 template <int D>
 struct GatherCfg {
@@ -60,9 +63,8 @@ struct GatherCfg {
 //   soff  int32 [n_blocks + 1]   first stage of every row-block
 //   meta  uint8 [stages]         bits 0-2: real 16-column groups (1..4), bit 4: first stage of its
 //                                row-block, bit 5: last stage
-//   cols  int16 [stages][64]     column of X for row r of the stage at slot (r & 7) * 8 + (r >> 3)
-//                                (a producer thread's eight rows are adjacent); -1 = zero row,
-//                                -2 = beyond the real groups (not loaded, not multiplied)
+//   cols  int16 [stages][64]     column of X for row r of the stage; -1 = zero row (padding inside a
+//                                real group), -2 = beyond the real groups (not loaded, not multiplied)
 //   tiles bf16  [stages][d][64]  weight tile, row n at byte n*128, 16-byte chunk c at (c ^ (n & 7))
 struct GatherLayout {
   size_t soff_off, meta_off, cols_off, tiles_off, total;
@@ -123,7 +125,7 @@ gather_plan_fill_kernel(const int32_t* __restrict__ blk_ptr, const int32_t* __re
     const int groups = left <= 0 ? 1 : (left >= kGStageK ? 4 : (left + 15) / 16);
     int16_t c = -2;
     if (r < groups * 16) c = k < kc ? static_cast<int16_t>(idx[lo + k]) : static_cast<int16_t>(-1);
-    cols[static_cast<size_t>(g0 + s) * kGStageK + (r & 7) * 8 + (r >> 3)] = c;
+    cols[static_cast<size_t>(g0 + s) * kGStageK + r] = c;
   }
   // weight tiles: one thread per 16-byte chunk (8 columns of one row)
   const int chunks = n_st * block * 8;
@@ -177,7 +179,7 @@ transpose_kernel(const uint16_t* __restrict__ X, int rows, int cols, int ldx, ui
 // ---- the kernel --------------------------------------------------------------------------
 struct GatherParams {
   const uint16_t* XT;
-  int ldxt, tokens, n_out, act;
+  int ldxt, tokens, n_out, k_in, act;
   const uint16_t* bias;
   uint16_t* Y;
   int ldy;
@@ -217,7 +219,7 @@ __device__ __forceinline__ void tmem_load_16cols(uint32_t taddr, uint32_t (&v)[1
 
 template <int D>
 __global__ void __launch_bounds__(kGThreads, 1)
-linear_gather_kernel(const __grid_constant__ GatherParams P) {
+linear_gather_kernel(const __grid_constant__ CUtensorMap map_xt, const __grid_constant__ GatherParams P) {
   using Cfg = GatherCfg<D>;
   constexpr int S = Cfg::kStages;
   extern __shared__ uint8_t smem_raw[];
@@ -237,7 +239,8 @@ linear_gather_kernel(const __grid_constant__ GatherParams P) {
   auto acc_empty_bar = [&](int a) { return bar_base + 8u * (2 * S + 2 + a); };
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), kGProducers + 1); mbar_init(empty_bar(s), 1); }
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_xt)) : "memory");
+    for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(acc_full_bar(a), 1); mbar_init(acc_empty_bar(a), 4); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -256,52 +259,75 @@ linear_gather_kernel(const __grid_constant__ GatherParams P) {
 
   if (warp < 4) {
     // ---------------------------------------------------------------- producers
-    const int pt = threadIdx.x;                   // 0..127
-    const int chunk = pt & 15, r0 = pt >> 4;      // 16-byte token chunk, row residue mod 8
-    const uint32_t dst_thread = static_cast<uint32_t>((chunk >> 3) * (kGStageK * 128) + r0 * 128 + (((chunk & 7) ^ r0) << 4));
-    int stage = 0;
-    uint32_t phase = 0;
+    // Warp w fills the stages whose running number is w (mod 4).  Lane = (64-token half, group of
+    // four consecutive rows): one TMA gather4 per lane brings four kept columns (rows of XT) x 64
+    // tokens into the stage with the 128-byte swizzle.  A row number equal to k_in is out of range
+    // and reads as zeros (padding rows); tokens beyond the end read as zeros too.
+    const int half = lane >> 4, quad4 = lane & 15;
+    const uint32_t dst_lane = static_cast<uint32_t>(half * (kGStageK * 128) + quad4 * 512);
+    long long n0 = 0;                                // stages before this unit, over all units of this CTA
     bool ok = true;
     for (int unit = blockIdx.x; unit < total_units && ok; unit += gridDim.x) {
       const int m = unit / P.n_chunks, ch = unit - m * P.n_chunks;
       const int rb0 = ch * P.rb_per_chunk, rb1 = min(P.n_blocks, rb0 + P.rb_per_chunk);
       const int g_begin = __ldg(P.soff + rb0), g_end = __ldg(P.soff + rb1);
-      const int tok = m * kBlockM + chunk * 8;
-      const uint32_t src_bytes = tok < P.tokens ? 16u : 0u;
-      const uint16_t* src_col0 = P.XT + (src_bytes ? tok : 0);
-      if (pt < kGPrefetch)
-        asm volatile("prefetch.global.L1 [%0];" ::"l"(P.cols + static_cast<size_t>(g_begin + pt) * kGStageK));
-      for (int g = g_begin; g < g_end; ++g) {
-        if (!mbar_wait(empty_bar(stage), phase ^ 1u)) { ok = false; break; }
-        const uint32_t a_dst = smem_base + stage * Cfg::kStage;
-        if (pt == 0) {
-          s_meta[stage] = __ldg(P.meta + g);
-          mbar_arrive_expect_tx(full_bar(stage), Cfg::kStageB);
-          asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                       ::"r"(a_dst + kGStageA), "l"(reinterpret_cast<uint64_t>(P.tiles + static_cast<size_t>(g) * D * 64)),
-                         "r"(static_cast<uint32_t>(Cfg::kStageB)), "r"(full_bar(stage))
-                       : "memory");
-          asm volatile("prefetch.global.L1 [%0];" ::"l"(P.cols + static_cast<size_t>(g + kGPrefetch) * kGStageK));
-          asm volatile("prefetch.global.L1 [%0];" ::"l"(P.meta + g + 128));
-        }
-        const uint4 cv = __ldg(reinterpret_cast<const uint4*>(P.cols + static_cast<size_t>(g) * kGStageK + r0 * 8));
-        const uint32_t cw[4] = {cv.x, cv.y, cv.z, cv.w};
+      const int x = m * kBlockM + half * 64;
+      const int first = g_begin + static_cast<int>(((warp - n0) % 4 + 4) % 4);   // this warp's first stage of the unit
+      // column numbers and stage bytes are loaded two of the warp's stages (eight stages) ahead
+      uint2 cq[2];
+      uint32_t mq[2];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const int col = static_cast<int16_t>((cw[i >> 1] >> (16 * (i & 1))) & 0xffffu);
-          if (col != -2) {
-            const uint16_t* src = col >= 0 ? src_col0 + static_cast<size_t>(col) * P.ldxt : P.XT;
-            const uint32_t sz = col >= 0 ? src_bytes : 0u;
-            asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;"
-                         ::"r"(a_dst + dst_thread + static_cast<uint32_t>(i) * 1024u), "l"(src), "r"(sz) : "memory");
+      for (int q = 0; q < 2; ++q) {
+        cq[q] = __ldg(reinterpret_cast<const uint2*>(P.cols + static_cast<size_t>(first + 4 * q) * kGStageK + quad4 * 4));
+        mq[q] = __ldg(P.meta + first + 4 * q);
+      }
+      for (int g0 = first; g0 < g_end && ok; g0 += 8) {
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+          const int g = g0 + 4 * q;
+          if (g < g_end && ok) {
+            const long long n = n0 + (g - g_begin);
+            const int stage = static_cast<int>(n % S);
+            const uint32_t phase = static_cast<uint32_t>((n / S) & 1);
+            if (!mbar_wait(empty_bar(stage), phase ^ 1u)) { ok = false; }
+            if (ok) {
+              const uint2 cv = cq[q];
+              const uint32_t mt = mq[q];
+              cq[q] = __ldg(reinterpret_cast<const uint2*>(P.cols + static_cast<size_t>(g + 8) * kGStageK + quad4 * 4));
+              mq[q] = __ldg(P.meta + g + 8);
+              const uint32_t a_dst = smem_base + stage * Cfg::kStage;
+              const int groups = static_cast<int>(mt & 7u);
+              if (lane == 0) {
+                s_meta[stage] = static_cast<uint8_t>(mt);
+                mbar_arrive_expect_tx(full_bar(stage), static_cast<uint32_t>(groups * 16 * kBlockM * 2 + Cfg::kStageB));
+                asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                             ::"r"(a_dst + kGStageA), "l"(reinterpret_cast<uint64_t>(P.tiles + static_cast<size_t>(g) * D * 64)),
+                               "r"(static_cast<uint32_t>(Cfg::kStageB)), "r"(full_bar(stage))
+                             : "memory");
+              }
+              __syncwarp();
+              if (quad4 * 4 < groups * 16) {
+                int r[4];
+                r[0] = static_cast<int16_t>(cv.x & 0xffffu);
+                r[1] = static_cast<int16_t>(cv.x >> 16);
+                r[2] = static_cast<int16_t>(cv.y & 0xffffu);
+                r[3] = static_cast<int16_t>(cv.y >> 16);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) r[i] = r[i] < 0 ? P.k_in : r[i];
+                asm volatile(
+                    "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes "
+                    "[%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+                    ::"r"(a_dst + dst_lane), "l"(reinterpret_cast<uint64_t>(&map_xt)), "r"(x), "r"(r[0]), "r"(r[1]),
+                      "r"(r[2]), "r"(r[3]), "r"(full_bar(stage))
+                    : "memory");
+              }
+            }
           }
         }
-        asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(full_bar(stage)) : "memory");
-        if (++stage == S) { stage = 0; phase ^= 1u; }
       }
+      n0 += g_end - g_begin;
     }
-    if (!ok) atomicExch(P.status, BSP_ERR_TIMEOUT);
-    asm volatile("cp.async.wait_all;" ::: "memory");
+    if (!ok && lane == 0) atomicExch(P.status, BSP_ERR_TIMEOUT);
   } else if (warp == 4) {
     // ---------------------------------------------------------------- MMA issuer
     if (lane == 0) {
@@ -357,6 +383,15 @@ linear_gather_kernel(const __grid_constant__ GatherParams P) {
       const int t = m * kBlockM + quad * 32 + lane;
       uint16_t* yrow = P.Y + static_cast<size_t>(t) * P.ldy;
       for (int rb = rb0; rb < rb1; ++rb) {
+        // the bias of this row-block first, so that its latency overlaps the wait for the accumulator
+        uint4 bv[D / 8];
+#pragma unroll
+        for (int j = 0; j < D / 8; ++j) bv[j] = make_uint4(0u, 0u, 0u, 0u);
+        if (P.bias != nullptr) {
+          const uint4* bp = reinterpret_cast<const uint4*>(P.bias + static_cast<size_t>(rb) * D);
+#pragma unroll
+          for (int j = 0; j < D / 8; ++j) bv[j] = __ldg(bp + j);
+        }
         if (!mbar_wait(acc_full_bar(acc), acc_phase[acc])) { ok = false; break; }
         tcgen05_fence_after();
         const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + static_cast<uint32_t>(acc * D);
@@ -365,19 +400,14 @@ linear_gather_kernel(const __grid_constant__ GatherParams P) {
         for (int c0 = 0; c0 < D; c0 += kPiece) {
           uint32_t v[16];
           tmem_load_16cols(taddr + c0, v);
-          uint4 bv[2] = {make_uint4(0u, 0u, 0u, 0u), make_uint4(0u, 0u, 0u, 0u)};
-          if (P.bias != nullptr) {
-            const uint4* bp = reinterpret_cast<const uint4*>(P.bias + static_cast<size_t>(rb) * D + c0);
-            bv[0] = __ldg(bp);
-            bv[1] = __ldg(bp + 1);
-          }
           tmem_load_wait();
           if (c0 + kPiece >= D) {              // this warp's last read of the accumulator
             tcgen05_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(acc_empty_bar(acc));
           }
-          const uint32_t bw[8] = {bv[0].x, bv[0].y, bv[0].z, bv[0].w, bv[1].x, bv[1].y, bv[1].z, bv[1].w};
+          const uint4 b0 = bv[c0 / 8], b1 = bv[c0 / 8 + 1];
+          const uint32_t bw[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
           float f[16];
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
@@ -423,9 +453,12 @@ int launch_gather(TcDevice* dev, int slot, const GatherParams& P, cudaStream_t s
     attr_set[device] = true;
   }
   (void)slot;
+  CUtensorMap map_xt;      // XT as [k_in rows, tokens]; box = one row of 64 tokens, 128-byte swizzle, zeros out of range
+  // (no L2 promotion: a gathered row is 128 bytes, and fetching 256 would read every line twice)
+  if (!make_map(&map_xt, P.XT, P.tokens, P.k_in, P.ldxt, 1, 64, CU_TENSOR_MAP_L2_PROMOTION_L2_128B)) return BSP_ERR_CUDA;
   const int units = P.m_tiles * P.n_chunks;
   const int grid = units < dev->sms ? units : dev->sms;
-  linear_gather_kernel<D><<<grid, kGThreads, Cfg::kSmemBytes, s>>>(P);
+  linear_gather_kernel<D><<<grid, kGThreads, Cfg::kSmemBytes, s>>>(map_xt, P);
   BSP_LAUNCH_CHECK();
   return BSP_OK;
 }
@@ -504,6 +537,7 @@ extern "C" int bsp_linear_gathered(const void* gplan, int n_out, int k_in, int b
   P.ldxt = ldxt;
   P.tokens = tokens;
   P.n_out = n_out;
+  P.k_in = k_in;
   P.act = act;
   P.bias = static_cast<const uint16_t*>(bias);
   P.Y = static_cast<uint16_t*>(Y);
