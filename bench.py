@@ -231,10 +231,9 @@ def dense_context(wl, device, iters=20):
     return out
 
 
-def weight_side_bandwidth(device, peaks, iters=10):
-    """Achieved HBM GB/s of the weight-side kernels (bsp_prepare_batched: norms, gamma, penalty, keep flags,
-    pack, plan) on the 72 weight matrices of a BERT-base encoder stack in one call, L2 flushed before each
-    run.  A single 768x768 matrix is 1.2 MB, far too small to time against HBM on its own."""
+def stack_jobs(device):
+    """The 72 weight matrices of a BERT-base encoder stack (d=16, about 3x) as one bsp_prepare_batched job array:
+    (array, block height, weights, groups, kept groups, the LayerJob objects that own the buffers)."""
     import torch
     import paper_2009_08065_b200 as bsp
     d, rate = 16, 3.0
@@ -256,7 +255,16 @@ def weight_side_bandwidth(device, peaks, iters=10):
         weights += rows * cols
         groups += shape[0] * shape[1]
         kept += int(keep.sum().item())
-    arr = bsp.make_job_array(jobs)
+    return bsp.make_job_array(jobs), d, weights, groups, kept, jobs
+
+
+def weight_side_bandwidth(device, peaks, iters=10):
+    """Achieved HBM GB/s of the weight-side kernels (bsp_prepare_batched: norms, gamma, penalty, keep flags,
+    pack, plan) on the 72 weight matrices of a BERT-base encoder stack in one call, L2 flushed before each
+    run.  A single 768x768 matrix is 1.2 MB, far too small to time against HBM on its own."""
+    import torch
+    import paper_2009_08065_b200 as bsp
+    arr, d, weights, groups, kept, _keepalive = stack_jobs(device)
     flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=device)
     ms = []
     for i in range(iters + 3):
@@ -497,11 +505,46 @@ def run_reference(args):
 
 
 def run_case(args):
-    """A handful of launches of one call on the bench workload, for profilers (no timing, no JSON):
-    --case qkv|attn_out|ffn_up|ffn_down runs that linear's GEMM, --case prepare the batched weight-side call."""
+    """A handful of launches of one call, for profilers (no timing, no JSON):
+    --case qkv|attn_out|ffn_up|ffn_down runs that linear's GEMM on the bench workload, --case prepare the batched
+    weight-side call on its four matrices, --case prepare_stack the same call on the 72 matrices of a BERT-base
+    stack (inputs larger than L2), --case gather the gathering linear kernel on a BERT-large FFN-up point
+    (16384 tokens, 1024 -> 4096, 64-row blocks, 5x)."""
     import torch
     torch.cuda.set_device(0)
     device = torch.device("cuda", 0)
+    if args.case == "prepare_stack":
+        import paper_2009_08065_b200 as bsp
+        stack = stack_jobs(device)          # keeps the buffers alive
+        arr, d = stack[0], stack[1]
+        for _ in range(3):
+            bsp.bsp_prepare_batched(arr, d, EPS, bsp.PEN_L2)
+        bsp.bsp_linear_status()
+        print("case prepare_stack: 3 calls done")
+        return
+    if args.case == "gather":
+        import paper_2009_08065_b200 as bsp
+        T, N, K, d, c = 16384, 4096, 1024, 64, 5.0
+        gen = torch.Generator(device=device)
+        gen.manual_seed(si.DEFAULT_SEED)
+        X = torch.randn(T, K, device=device, generator=gen).to(torch.bfloat16)
+        XT = torch.empty(K, T, dtype=torch.bfloat16, device=device)
+        bsp.bsp_transpose(X, XT)
+        Wd = (torch.randn(N, K, device=device, generator=gen) * 0.02).to(torch.bfloat16)
+        keep = torch.zeros(N // d, K, dtype=torch.bool, device=device)
+        keep.scatter_(1, torch.rand(N // d, K, device=device, generator=gen).topk(int(round(K / c)), dim=1).indices, True)
+        W = (Wd.view(N // d, d, K) * keep[:, None, :]).view(N, K).contiguous()
+        pk = bsp.PackedMatrix.allocate(N, K, d, bsp.ORIENT_C, device)
+        bsp.bsp_prune_pack(W, pk, 0.0)
+        gplan = torch.empty(bsp.bsp_linear_gather_plan_bytes(N, K, d), dtype=torch.uint8, device=device)
+        bsp.bsp_linear_gather_plan(pk, gplan)
+        bias = (torch.randn(N, device=device, generator=gen) * 0.02).to(torch.bfloat16)
+        Y = torch.empty(T, N, dtype=torch.bfloat16, device=device)
+        for _ in range(3):
+            bsp.bsp_linear_gathered(gplan, N, K, d, XT, bias, 1, Y)
+        bsp.bsp_linear_status()
+        print("case gather: 3 launches done")
+        return
     layer = LayerOnDevice(workload(), si.DEFAULT_SEED, 0, device)
     layer.step()
     torch.cuda.synchronize()
@@ -521,7 +564,7 @@ def run_case(args):
 
 def run_sweep(args):
     """The BERT-large sweep (hidden 1024, FFN 4096, tokens 32768 by default): compression 1.5/2/3/5/8 x block height
-    8/16/32/64 on the four linear shapes.  For every point: the zero-expanded dense route (bsp_linear_planned), the
+    8/16/32/64 (and 128) on the four linear shapes.  For every point: the zero-expanded dense route (bsp_linear_planned), the
     gathering kernel (bsp_linear_gathered, block heights it takes; X transposed beforehand, that copy timed
     separately once per input width), and torch.matmul on the dense shape as context.  L2 is flushed (256 MiB
     written) before every timed launch; medians of `--steps` launches.  One JSON line per point."""
@@ -562,7 +605,7 @@ def run_sweep(args):
         Yg = torch.empty(T, N, dtype=torch.bfloat16, device=device)
         Wd = (torch.randn(N, K, device=device, generator=gen) * 0.02).to(torch.bfloat16)
         t_dense = timed(lambda: torch.matmul(X, Wd.t()))
-        for d in (8, 16, 32, 64):
+        for d in (8, 16, 32, 64, 128):        # 128 is beyond the named grid: it shows where the gathering kernel is heading
             for c in (1.5, 2.0, 3.0, 5.0, 8.0):
                 kc = int(round(K / c))
                 scores = torch.rand(N // d, K, device=device, generator=gen)
@@ -602,7 +645,7 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["cuda", "reference"], default="cuda")
-    ap.add_argument("--case", choices=["qkv", "attn_out", "ffn_up", "ffn_down", "prepare"], default=None,
+    ap.add_argument("--case", choices=["qkv", "attn_out", "ffn_up", "ffn_down", "prepare", "prepare_stack", "gather"], default=None,
                     help="run a few launches of one call for a profiler and exit")
     ap.add_argument("--sweep", choices=["bert_large"], default=None,
                     help="time the BERT-large compression x block-height grid and print one JSON line per point")
