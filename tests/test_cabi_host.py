@@ -118,6 +118,35 @@ def test_argument_errors_are_caught_before_any_launch():
     assert lib.bsp_linear_cuda_core(p, p, p, 8, 8, 4, p, 0, 8, None, 0, p, 8, None) == 0
 
 
+def test_gather_entry_points_reject_bad_arguments_without_a_gpu():
+    lib = bsp.lib
+    p, ws = ctypes.c_void_p(0x10000), ctypes.c_void_p(0x20000)
+    n = ctypes.c_size_t()
+    assert lib.bsp_linear_gather_plan_bytes(4096, 1024, 64, ctypes.byref(n)) == 0
+    # stage tables, two column arrays and one d x 64 tile per stage: above the weights themselves, below twice that
+    assert 4096 * 1024 * 2 < n.value < 2 * 4096 * 1024 * 2 and n.value % 256 == 0
+    assert bsp.bsp_linear_gather_plan_bytes(4096, 1024, 64) == n.value
+    assert lib.bsp_linear_gather_plan_bytes(4096, 1024, 48, ctypes.byref(n)) == -2           # 48 does not divide 4096
+    assert lib.bsp_linear_gather_plan_bytes(96, 1024, 48, ctypes.byref(n)) == -6             # block height not taken
+    assert lib.bsp_linear_gather_plan_bytes(128, 40000, 64, ctypes.byref(n)) == -6           # columns do not fit int16
+    assert lib.bsp_linear_gather_plan_bytes(128, 64, 64, None) == -1
+    assert lib.bsp_linear_gather_plan(None, p, p, 128, 64, 64, ws, 1 << 20, None) == -1
+    assert lib.bsp_linear_gather_plan(p, p, p, 128, 64, 64, ws, 16, None) == -3
+    assert lib.bsp_linear_gather_plan(p, p, p, 128, 64, 64, ctypes.c_void_p(0x20010), 1 << 20, None) == -1
+    assert lib.bsp_transpose(None, 8, 8, 8, p, 8, None) == -1
+    assert lib.bsp_transpose(p, 8, 16, 8, ws, 8, None) == -2                                 # ldx < cols
+    assert lib.bsp_transpose(p, 8, 12, 16, ws, 8, None) == -6                                # cols not a multiple of 8
+    assert lib.bsp_transpose(p, 0, 8, 8, ws, 8, None) == 0
+    assert lib.bsp_linear_gathered(None, 128, 64, 64, p, 8, 8, None, 0, p, 128, None) == -1
+    assert lib.bsp_linear_gathered(ws, 128, 64, 64, p, 8, 8, None, 7, p, 128, None) == -1    # unknown activation
+    assert lib.bsp_linear_gathered(ws, 100, 64, 64, p, 8, 8, None, 0, p, 128, None) == -2
+    assert lib.bsp_linear_gathered(ws, 128, 64, 64, p, 16, 8, None, 0, p, 128, None) == -2   # ldxt < tokens
+    assert lib.bsp_linear_gathered(ws, 128, 64, 24, p, 8, 8, None, 0, p, 128, None) == -2    # 24 does not divide 128
+    assert lib.bsp_linear_gathered(ws, 96, 64, 48, p, 8, 8, None, 0, p, 96, None) == -6      # block height not taken
+    assert lib.bsp_linear_gathered(ws, 128, 64, 64, p, 12, 16, None, 0, p, 128, None) == -6  # tokens not a multiple of 8
+    assert lib.bsp_linear_gathered(ws, 128, 64, 64, p, 0, 8, None, 0, p, 128, None) == 0     # zero tokens: no-op
+
+
 def test_product_code_does_not_touch_the_oracle():
     pkg = os.path.join(ROOT, "paper_2009_08065_b200")
     for dirpath, _, files in os.walk(pkg):
