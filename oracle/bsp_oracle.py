@@ -266,6 +266,49 @@ def keep_topk_per_block(w_bits: np.ndarray, block: int, orient: str, keep_count:
 
 
 # ---------------------------------------------------------------------------
+# Algorithm 2, retraining loop: "Update W using Adam", then W = W * Mask
+# ---------------------------------------------------------------------------
+def adam_step_masked(w: np.ndarray, g: np.ndarray, m: np.ndarray, v: np.ndarray, step: int, lr: float,
+                     beta1: float, beta2: float, eps: float, weight_decay: float,
+                     mask: Optional[np.ndarray]) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+    """One iteration of Algorithm 2's retraining loop on one weight matrix, in float64.
+
+    The algorithm says only "update W ... using Adam" and then "W = W * Mask".  Adam is taken as
+    published (Kingma & Ba, 2015, Algorithm 1, with bias correction), `step` counting from 1:
+        m <- beta1 m + (1 - beta1) g          v <- beta2 v + (1 - beta2) g^2
+        mhat = m / (1 - beta1^step)           vhat = v / (1 - beta2^step)
+        W <- W - lr * mhat / (sqrt(vhat) + eps)
+    A weight decay, which the paper does not mention, is the decoupled one (W <- W - lr * wd * W, taken
+    on the old W) and is 0 unless asked for.  The moments are updated for every weight, pruned or not,
+    as the algorithm's order of operations implies; then the mask is applied to W only.
+    mask None = the reweighted-training loop's plain update (no mask yet).
+    Returns (W, m, v).
+    """
+    w = np.asarray(w, dtype=np.float64)
+    g = np.asarray(g, dtype=np.float64)
+    m_new = beta1 * np.asarray(m, dtype=np.float64) + (1.0 - beta1) * g
+    v_new = beta2 * np.asarray(v, dtype=np.float64) + (1.0 - beta2) * g * g
+    mhat = m_new / (1.0 - beta1 ** step)
+    vhat = v_new / (1.0 - beta2 ** step)
+    w_new = w - lr * mhat / (np.sqrt(vhat) + eps) - lr * weight_decay * w
+    if mask is not None:
+        w_new = w_new * np.asarray(mask, dtype=np.float64)
+    return w_new, m_new, v_new
+
+
+def repack_values(w_bits: np.ndarray, blk_ptr: np.ndarray, idx: np.ndarray, block: int) -> np.ndarray:
+    """Packed tiles of an UPDATED W under a fixed set of kept columns (orientation C): Algorithm 2 fixes the
+    mask before retraining, so the storage of Section 3.1 keeps its indices and only its values change.
+    Tile of row-block b: rows [b*block, (b+1)*block) restricted to idx[blk_ptr[b]:blk_ptr[b+1]], row-major."""
+    rows = w_bits.shape[0]
+    out = []
+    for b in range(rows // block):
+        cols = idx[blk_ptr[b]:blk_ptr[b + 1]]
+        out.append(np.ascontiguousarray(w_bits[b * block:(b + 1) * block][:, cols]).reshape(-1))
+    return np.concatenate(out) if out else np.zeros(0, dtype=np.uint16)
+
+
+# ---------------------------------------------------------------------------
 # compressed storage  (Section 3.1: only non-zero rows/columns at block level are indexed)
 # ---------------------------------------------------------------------------
 def pack(w_bits: np.ndarray, keep: np.ndarray, block: int, orient: str

@@ -488,3 +488,72 @@ def test_backward_weight_is_the_adjoint_in_w():
     n, k = [int(a[0]) for a in np.nonzero(m)]
     brute = sum(float(O.bf16_to_f64(dy)[t, n]) * float(O.bf16_to_f64(x)[t, k]) for t in range(T))
     assert dw[n, k] == pytest.approx(brute, rel=1e-14)
+
+
+# ---------------------------------------------------------------------------------------- Algorithm 2's retraining update
+def _adam_scalar_loop(w, g_seq, lr, b1, b2, eps):
+    """Adam as printed by Kingma & Ba (Algorithm 1), one scalar at a time, plain Python floats."""
+    m = v = 0.0
+    out = []
+    for t, g in enumerate(g_seq, start=1):
+        m = b1 * m + (1 - b1) * g
+        v = b2 * v + (1 - b2) * g * g
+        w = w - lr * (m / (1 - b1 ** t)) / (math.sqrt(v / (1 - b2 ** t)) + eps)
+        out.append(w)
+    return out
+
+
+def test_adam_step_first_step_moves_by_lr_against_the_gradient_sign():
+    """With zero moments the bias-corrected first step is lr * g / (|g| + eps): a step of (almost) lr."""
+    w = np.array([[0.5, -0.25, 0.125, 1.0]])
+    g = np.array([[3.0, -7.0, 1e-3, 0.0]])
+    z = np.zeros_like(w)
+    w1, m1, v1 = O.adam_step_masked(w, g, z, z, 1, 1e-2, 0.9, 0.999, 1e-8, 0.0, None)
+    assert np.allclose(w1[0, :3], w[0, :3] - 1e-2 * np.sign(g[0, :3]), rtol=0, atol=1e-6)
+    assert w1[0, 3] == 1.0                                    # zero gradient, no decay: unchanged
+    assert np.allclose(m1, 0.1 * g) and np.allclose(v1, 0.001 * g * g)
+
+
+def test_adam_step_constant_gradient_closed_form_and_scalar_loop():
+    """A constant gradient gives mhat = g and vhat = g^2 at every step, so W_t = W_0 - t lr g / (|g| + eps);
+    a changing gradient is checked against the published algorithm written as a scalar loop."""
+    lr, b1, b2, eps = 3e-5, 0.9, 0.999, 1e-8
+    w = np.array([[0.02, -0.01]])
+    g = np.array([[0.3, -0.004]])
+    m = v = np.zeros_like(w)
+    for t in range(1, 8):
+        w, m, v = O.adam_step_masked(w, g, m, v, t, lr, b1, b2, eps, 0.0, None)
+    assert np.allclose(w, np.array([[0.02, -0.01]]) - 7 * lr * g / (np.abs(g) + eps), rtol=1e-12, atol=0)
+    g_seq = [0.5, -0.2, 0.05, 0.9, -1.5]
+    w = np.array([[0.1]])
+    m = v = np.zeros((1, 1))
+    for t, gt in enumerate(g_seq, start=1):
+        w, m, v = O.adam_step_masked(w, np.array([[gt]]), m, v, t, 1e-3, b1, b2, eps, 0.0, None)
+    assert w[0, 0] == pytest.approx(_adam_scalar_loop(0.1, g_seq, 1e-3, b1, b2, eps)[-1], rel=1e-13)
+
+
+def test_adam_step_mask_and_decoupled_weight_decay():
+    """W = W * Mask after the update: pruned weights are exactly zero, their moments still move; the
+    decay term is lr * wd * W_old, independent of the gradient."""
+    w = np.array([[0.5, -0.25], [0.125, 1.0]])
+    g = np.array([[1.0, 2.0], [3.0, 4.0]])
+    mask = np.array([[True, False], [False, True]])
+    z = np.zeros_like(w)
+    w1, m1, v1 = O.adam_step_masked(w, g, z, z, 1, 1e-2, 0.9, 0.999, 1e-8, 0.0, mask)
+    assert w1[0, 1] == 0.0 and w1[1, 0] == 0.0 and w1[0, 0] != 0.0
+    assert (m1 != 0).all() and (v1 != 0).all()
+    wd0, _, _ = O.adam_step_masked(w, np.zeros_like(g), z, z, 1, 1e-2, 0.9, 0.999, 1e-8, 0.1, None)
+    assert np.allclose(wd0, w * (1 - 1e-2 * 0.1), rtol=1e-15)
+
+
+def test_repack_values_equals_pack_of_the_updated_matrix():
+    """With the kept sets fixed, re-packing the values of an updated W gives what a fresh pack of
+    W * Mask gives, and leaves the indices alone."""
+    spec = si.LinearSpec("repack", 96, 80, False, 2.0, 12)
+    wp, keep = si.make_pruned_weight(5, spec)
+    blk_ptr, idx, vals = O.pack(wp, keep, 12, "C")
+    w2 = si.zero_groups(si.make_weight(6, spec), keep, 12, "C")          # new values, same mask
+    ptr2, idx2, vals2 = O.pack(w2, keep, 12, "C")
+    assert np.array_equal(ptr2, blk_ptr) and np.array_equal(idx2, idx)
+    assert np.array_equal(O.repack_values(w2, blk_ptr, idx, 12), vals2)
+    assert np.array_equal(O.repack_values(wp, blk_ptr, idx, 12), vals)
