@@ -191,6 +191,38 @@ int bsp_apply_mask(void* W, int rows, int cols, int ldw, int block, int orient,
                    const uint8_t* keep, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * bsp_masked_adam_step — one iteration of Algorithm 2's retraining loop on one weight matrix:
+ * "update W ... using Adam", then "W = W * Mask", in one pass.  Adam as published (Kingma & Ba 2015,
+ * bias-corrected; the paper names no hyper-parameters beyond the learning rate, so all are the
+ * caller's):
+ *   m = beta1 m + (1 - beta1) g,   v = beta2 v + (1 - beta2) g^2,
+ *   W = W - lr ( (m / (1 - beta1^step)) / (sqrt(v / (1 - beta2^step)) + eps) + weight_decay W ),
+ *   then every weight of a group whose keep flag is 0 is set to +0 (the moments are updated for
+ *   every weight, pruned or not, as the algorithm's order implies).
+ * W, m, v: float32 [rows, cols] with leading dimension ldw, updated in place (the optimiser's
+ * weights are float32: a bf16 weight cannot absorb steps of the paper's size); grad float32 with
+ * leading dimension ldg (task gradient, plus bsp_penalty_grad's term during reweighted training).
+ * keep: per-group flags as written by bsp_prune_pack for (block, orient), or NULL = no mask (the
+ * reweighted-training loop's plain update; block and orient are then ignored).  step >= 1.
+ * W_bf16: nullable bf16 [rows, cols] (ldb) output, the updated masked weights rounded to nearest
+ * even: with ldb = cols it is the execution layout that bsp_linear_planned reads.
+ * Needs cols and the leading dimensions multiples of 4 and 16-byte aligned float arrays (else
+ * BSP_ERR_UNSUPPORTED).  Errors: BSP_ERR_ARG (NULL, step < 1, beta outside [0, 1), eps < 0),
+ * BSP_ERR_SHAPE.
+ *
+ * bsp_repack_values — the packed values of an UPDATED W under fixed kept sets (orientation C):
+ * Algorithm 2 fixes the mask before retraining, so Section 3.1's storage keeps blk_ptr and idx
+ * and only vals changes: tile of block b = rows of the block restricted to its kept columns.
+ * W: bf16 [rows, cols] (ldw); blk_ptr / idx as written by bsp_prune_pack; vals is overwritten.
+ */
+int bsp_masked_adam_step(float* W, const float* grad, float* m, float* v, int rows, int cols, int ldw, int ldg,
+                         const uint8_t* keep, int block, int orient,
+                         float lr, float beta1, float beta2, float eps, float weight_decay, int step,
+                         void* W_bf16, int ldb, void* stream);
+int bsp_repack_values(const void* W, int rows, int cols, int ldw, int block,
+                      const int32_t* blk_ptr, const int32_t* idx, void* vals, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
  * bsp_prepare_batched — the weight-side steps of the path for several matrices at once
  * (orientation C): the norms / gamma / penalty of Section 3.2, Algorithm 1's keep decision, the
  * packed storage of Section 3.1 and, optionally, bsp_linear's execution layout, in two launches

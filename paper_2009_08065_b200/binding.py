@@ -81,6 +81,8 @@ _SIGNATURES = {
     "bsp_linear_gather_plan": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _sz, _vp]),
     "bsp_transpose": (_i, [_vp, _i, _i, _i, _vp, _i, _vp]),
     "bsp_linear_gathered": (_i, [_vp, _i, _i, _i, _vp, _i, _i, _vp, _i, _vp, _i, _vp]),
+    "bsp_masked_adam_step": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _vp, _i, _i, _f, _f, _f, _f, _f, _i, _vp, _i, _vp]),
+    "bsp_repack_values": (_i, [_vp, _i, _i, _i, _i, _vp, _vp, _vp, _vp]),
     "bsp_prepare_batched": (_i, [ctypes.POINTER(_LayerJob), _i, _i, _f, _i, _vp]),
     "bsp_linear_plan_bytes": (_i, [_i, _i, _i, _szp]),
     "bsp_linear_plan": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _sz, _vp]),
@@ -312,6 +314,23 @@ def bsp_linear(packed: PackedMatrix, X: torch.Tensor, bias: Optional[torch.Tenso
     _check(lib.bsp_linear(_ptr(packed.blk_ptr), _ptr(packed.idx), _ptr(packed.vals), packed.rows, packed.cols,
                           packed.block, _ptr(X), X.shape[0], _ld(X), _ptr(bias), act, _ptr(Y), _ld(Y), _ptr(ws),
                           0 if ws is None else ws.numel() * ws.element_size(), _stream(stream)), "bsp_linear")
+
+
+def bsp_masked_adam_step(W: torch.Tensor, grad: torch.Tensor, m: torch.Tensor, v: torch.Tensor,
+                         keep: Optional[torch.Tensor], block: int, orient: int, lr: float, beta1: float, beta2: float,
+                         eps: float, weight_decay: float, step: int, W_bf16: Optional[torch.Tensor] = None,
+                         stream=None) -> None:
+    """W, m, v, grad: float32 [rows, cols]; keep: per-group uint8 flags or None; W_bf16: optional bf16 output."""
+    rows, cols = W.shape
+    _check(lib.bsp_masked_adam_step(_ptr(W), _ptr(grad), _ptr(m), _ptr(v), rows, cols, _ld(W), _ld(grad), _ptr(keep),
+                                    block, orient, lr, beta1, beta2, eps, weight_decay, step, _ptr(W_bf16),
+                                    0 if W_bf16 is None else _ld(W_bf16), _stream(stream)), "bsp_masked_adam_step")
+
+
+def bsp_repack_values(W: torch.Tensor, packed: PackedMatrix, stream=None) -> None:
+    """Refreshes packed.vals from an updated bf16 W; blk_ptr and idx stay as they are."""
+    _check(lib.bsp_repack_values(_ptr(W), W.shape[0], W.shape[1], _ld(W), packed.block, _ptr(packed.blk_ptr),
+                                 _ptr(packed.idx), _ptr(packed.vals), _stream(stream)), "bsp_repack_values")
 
 
 def bsp_linear_gather_plan_bytes(n_out: int, k_in: int, block: int) -> int:

@@ -147,6 +147,22 @@ def test_gather_entry_points_reject_bad_arguments_without_a_gpu():
     assert lib.bsp_linear_gathered(ws, 128, 64, 64, p, 0, 8, None, 0, p, 128, None) == 0     # zero tokens: no-op
 
 
+def test_retraining_entry_points_reject_bad_arguments_without_a_gpu():
+    lib = bsp.lib
+    p = ctypes.c_void_p(0x10000)
+    args = lambda **kw: [kw.get("W", p), p, p, p, kw.get("rows", 8), kw.get("cols", 8), kw.get("ldw", 8), 8,      # noqa: E731
+                         kw.get("keep", None), kw.get("block", 4), 0, 1e-3, kw.get("beta1", 0.9), 0.999, 1e-8, 0.0,
+                         kw.get("step", 1), None, 0, None]
+    assert lib.bsp_masked_adam_step(*args(W=None)) == -1
+    assert lib.bsp_masked_adam_step(*args(step=0)) == -1
+    assert lib.bsp_masked_adam_step(*args(beta1=1.0)) == -1
+    assert lib.bsp_masked_adam_step(*args(ldw=4)) == -2
+    assert lib.bsp_masked_adam_step(*args(keep=p, block=3)) == -2                            # 3 does not divide 8
+    assert lib.bsp_masked_adam_step(*args(cols=6, ldw=8)) == -6                              # cols not a multiple of 4
+    assert lib.bsp_repack_values(p, 8, 8, 8, 4, None, p, p, None) == -1
+    assert lib.bsp_repack_values(p, 8, 8, 8, 3, p, p, p, None) == -2
+
+
 def test_product_code_does_not_touch_the_oracle():
     pkg = os.path.join(ROOT, "paper_2009_08065_b200")
     for dirpath, _, files in os.walk(pkg):
