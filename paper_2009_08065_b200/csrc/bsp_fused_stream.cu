@@ -142,7 +142,7 @@ fused_stream_kernel(const __grid_constant__ StreamBatch B) {
   __shared__ int s_kc;
   const int d = B.block;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, n_warps = blockDim.x >> 5;
-  int32_t* s_idx = reinterpret_cast<int32_t*>(s_raw + static_cast<size_t>(B.buf_bytes));      // [max part columns]
+  uint16_t* s_idx = reinterpret_cast<uint16_t*>(s_raw + static_cast<size_t>(B.buf_bytes));    // [max part columns], local column numbers
   const uint32_t bar = smem_u32(&s_bar);
 
   if (threadIdx.x == 0) {
@@ -262,7 +262,7 @@ fused_stream_kernel(const __grid_constant__ StreamBatch B) {
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
         const uint32_t bit = ((i < 4 ? f.x : f.y) >> (8 * (i & 3))) & 1u;
-        if (bit) s_idx[p++] = (k << 3) + i;
+        if (bit) s_idx[p++] = static_cast<uint16_t>((k << 3) + i);
       }
     }
     // execution layout: the rows with the pruned columns zeroed, one warp per row, 16-byte stores
@@ -401,7 +401,7 @@ bool fill_batch(StreamBatch& B, const FusedJob* jobs, int n_jobs, int block, flo
   B.total_items = total;
   B.buf_bytes = static_cast<int>(round_up(static_cast<size_t>(block) * max_part_cols * 2, 128));
   B.ticket = B.job[0].part_counts + B.job[0].j.n_blocks * B.job[0].parts + 1;
-  *smem_out = static_cast<size_t>(B.buf_bytes) + static_cast<size_t>(max_part_cols) * 5 + 16;
+  *smem_out = static_cast<size_t>(B.buf_bytes) + static_cast<size_t>(max_part_cols) * 3 + 16;   // rows, 2-byte list, flags
   return true;
 }
 
