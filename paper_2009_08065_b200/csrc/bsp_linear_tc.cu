@@ -466,7 +466,10 @@ extern "C" int bsp_linear_planned_ex(const void* plan, int n_out, int k_in, int 
   // Measured on B200: CTA pairs win (about 5 %) once the problem runs for many waves, where the L2 -> SM
   // operand traffic binds; for a few waves the one-CTA kernel's shorter start-up wins (about 2 us).
   const long long pair_tiles = static_cast<long long>((tokens + 255) / 256) * ((n_out + 255) / 256);
-  const bool pair = algo == BSP_LINEAR_CTA_PAIR || (algo == BSP_LINEAR_AUTO && pair_tiles >= 4LL * dev->sms);
+  // With GELU the epilogue is the longer side of a tile and the one-CTA kernel's slower main loop hides
+  // more of it: 202 us against 209 us at 32768 x 4096 x 1024.
+  const bool pair = algo == BSP_LINEAR_CTA_PAIR ||
+                    (algo == BSP_LINEAR_AUTO && pair_tiles >= 4LL * dev->sms && act == BSP_ACT_NONE);
   if (pair) return launch_tc_pair(dev, plan, X, Y, tokens, n_out, k_in, act, bias, ldx, ldy, s);
   LinearParams P{tokens, n_out, k_in, act, static_cast<const uint16_t*>(bias), dev->status};
   switch (choose_bn(tokens, n_out, dev->sms)) {
