@@ -303,6 +303,47 @@ def test_prepare_batched_streaming_batch_larger_than_the_gpu():
             job.penalty.fill_(-5.0)
 
 
+def test_prepare_batched_with_device_side_percentile_thresholds():
+    """The heavy-tailed workload's recipe in batched form (32-row blocks, 1.79x): every matrix's threshold is
+    found on the device (bsp_percentile_threshold) and read from there by the one batched call; kept counts
+    differ from block to block, and the wide matrix is split into column ranges."""
+    eps, block, rate = 1e-3, 32, 1.79
+    shapes = [(768, 768), (3072, 768), (768, 3072), (768, 768), (768, 3072), (3072, 768)]
+    jobs, refs = [], []
+    for n, (rows, cols) in enumerate(shapes):
+        w = si.student_t_bf16(400 + n, f"distil_batched{n}", (rows, cols), 3.0, 0.02)
+        wd = to_dev(w)
+        pk = bsp.PackedMatrix.allocate(rows, cols, block, bsp.ORIENT_C, DEV)
+        t_dev = torch.zeros(1, dtype=torch.float32, device=DEV)
+        bsp.bsp_percentile_threshold(wd, block, bsp.ORIENT_C, rate, t_dev, pk.ws)
+        shape = (rows // block, cols)
+        jobs.append(bsp.LayerJob(W=wd, out=pk, threshold=123.0, threshold_dev=t_dev,       # the host value must be ignored
+                                 norms=torch.empty(shape, dtype=torch.float32, device=DEV),
+                                 penalty=torch.zeros(1, dtype=torch.float64, device=DEV),
+                                 plan=torch.empty(bsp.bsp_linear_plan_bytes(rows, cols, block), dtype=torch.uint8, device=DEV)))
+        refs.append(w)
+    bsp.bsp_prepare_batched(jobs, block, eps, bsp.PEN_L2)
+    bsp.bsp_linear_status()
+    torch.cuda.synchronize()
+    for job, w in zip(jobs, refs):
+        rows, cols = w.shape
+        t_ref = O.percentile_threshold(w, block, "C", rate)
+        assert np.float32(job.threshold_dev.item()) == np.float32(t_ref)
+        n_ref = O.group_norms(w, block, "C")
+        assert np.allclose(job.norms.cpu().numpy(), n_ref, rtol=REL, atol=0)
+        assert float(job.penalty.item()) == pytest.approx(O.penalty_l2(n_ref, O.gamma_update(n_ref, eps)), rel=REL)
+        keep_ref = O.keep_flags(w, block, "C", t_ref)
+        ref_ptr, ref_idx, ref_vals = O.pack(w, keep_ref, block, "C")
+        blk_ptr, idx, vals, keep, kept = packed_to_host(job.out)
+        assert np.array_equal(keep, keep_ref) and np.array_equal(blk_ptr, ref_ptr)
+        assert np.array_equal(idx, ref_idx) and np.array_equal(vals, ref_vals)
+        counts = np.diff(blk_ptr)
+        assert counts.min() < counts.max()
+        assert abs(float(O.compression_rate(rows, cols, kept)) - rate) < 1e-3 * rate
+        plan = bits_of(job.plan.view(torch.int16)[: rows * cols].reshape(rows, cols))
+        assert np.array_equal(plan, O.prune(w, block, "C", t_ref))
+
+
 # ---------------------------------------------------------------------------------------- penalty gradient
 @pytest.mark.parametrize("orient,block,shape", [(0, 16, (768, 768)), (0, 3, (96, 50)), (1, 12, (96, 768)), (1, 5, (33, 50))])
 def test_penalty_gradient(orient, block, shape):
