@@ -493,7 +493,7 @@ def run_cuda(args):
                 "frac": round(achieved / peak, 4),
                 # dram__bytes_read.sum + dram__bytes_write.sum of the four launches, one ncu capture each
                 # (profiles/linear_tc_kernel_bert_base_T4096.md); Y is still in L2 when each kernel ends
-                "traffic": 58.32e6, "algorithmic_bytes": sum(
+                "traffic": 58.31e6, "algorithmic_bytes": sum(
                     2 * wl.tokens * sp.k_in + 2 * sp.n_out * sp.k_in + 2 * wl.tokens * sp.n_out + 2 * sp.n_out
                     for sp in wl.linears),
                 "peak_source": f"bf16_tflops burst, {peak_src}",
