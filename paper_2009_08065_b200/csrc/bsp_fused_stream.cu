@@ -149,6 +149,9 @@ fused_stream_kernel(const __grid_constant__ StreamBatch B) {
     mbar_init(bar, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    // launched with programmatic stream serialization: everything above overlapped the clearing
+    // kernel; the ticket and the slots it zeroes are touched only from here on
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     s_item = atomicAdd(B.ticket, 1);
   }
   __syncthreads();
@@ -367,6 +370,7 @@ fused_stream_kernel(const __grid_constant__ StreamBatch B) {
 // Zeroes the published counts and partials and the ticket slot of every matrix.
 __global__ void __launch_bounds__(256)
 stream_clear_kernel(const __grid_constant__ StreamBatch B) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the main kernel may take its seats now; it waits for this grid
   const StreamJob& O = B.job[blockIdx.x];
   const int n = O.j.n_blocks * O.parts;
   for (int i = threadIdx.x; i < n + 2; i += blockDim.x) O.part_counts[i] = 0;
@@ -445,8 +449,17 @@ int fused_stream(const FusedJob* jobs, int n_jobs, int block, float eps, int squ
     stream_clear_kernel<<<n, 256, 0, s>>>(*B);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { st = cuda_fail(e); break; }
-    fused_stream_kernel<<<B->total_items, kStreamThreads, smem_max, s>>>(*B);
-    e = cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(B->total_items);
+    cfg.blockDim = dim3(kStreamThreads);
+    cfg.dynamicSmemBytes = smem_max;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // start while the clearing kernel drains
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    e = cudaLaunchKernelEx(&cfg, fused_stream_kernel, *B);
     if (e != cudaSuccess) { st = cuda_fail(e); break; }
     *used = true;
   }
