@@ -121,19 +121,29 @@ class LayerOnDevice:
         import torch
         import paper_2009_08065_b200 as bsp
         self.torch, self.bsp, self.wl, self.device = torch, bsp, wl, device
-        self.host = {}          # pinned host copies of the inputs, for the end-to-end leg
+        # The step's inputs (X, the four W, the four biases) live in ONE device buffer and one pinned host
+        # buffer, each tensor a 256-byte-aligned view: the end-to-end leg uploads them with a single copy.
         x = si.make_activations(rank_seed(seed, rank), "layer_in", wl.tokens, wl.linears[0].k_in)
-        self.host["x"] = torch.from_numpy(x.view(np.int16)).pin_memory()
-        self.x = self.host["x"].to(device)
-        self.lin = []
+        parts = [("x", x.view(np.int16))]
         for spec in wl.linears:
             wp, _ = si.make_pruned_weight(seed, spec)          # weights are replicated across ranks
-            b = si.make_bias(seed, spec)
-            hw = torch.from_numpy(wp.view(np.int16)).pin_memory()
-            hb = torch.from_numpy(b.view(np.int16)).pin_memory()
+            parts.append((spec.name + ".W", wp.view(np.int16)))
+            parts.append((spec.name + ".b", si.make_bias(seed, spec).view(np.int16)))
+        offs, total = {}, 0
+        for name, a in parts:
+            offs[name] = total
+            total += (a.size + 127) // 128 * 128
+        self.host_all = torch.zeros(total, dtype=torch.int16).pin_memory()
+        for name, a in parts:
+            self.host_all[offs[name]: offs[name] + a.size].copy_(torch.from_numpy(np.ascontiguousarray(a).reshape(-1)))
+        self.dev_all = self.host_all.to(device)
+        view = lambda name, a: self.dev_all[offs[name]: offs[name] + a.size].view(a.shape)  # noqa: E731
+        self.x = view("x", parts[0][1])
+        self.lin = []
+        for i, spec in enumerate(wl.linears):
             n_blocks = spec.n_out // spec.block
             e = {
-                "spec": spec, "hW": hw, "hb": hb, "W": hw.to(device), "b": hb.to(device),
+                "spec": spec, "W": view(*parts[1 + 2 * i]), "b": view(*parts[2 + 2 * i]),
                 "norms": torch.empty((n_blocks, spec.k_in), dtype=torch.float32, device=device),
                 "gamma": torch.empty((n_blocks, spec.k_in), dtype=torch.float32, device=device),
                 "penalty": torch.zeros(1, dtype=torch.float64, device=device),
@@ -173,13 +183,10 @@ class LayerOnDevice:
         return outs
 
     def upload_inputs(self):
-        self.x.copy_(self.host["x"], non_blocking=True)
-        for e in self.lin:
-            e["W"].copy_(e["hW"], non_blocking=True)
-            e["b"].copy_(e["hb"], non_blocking=True)
+        self.dev_all.copy_(self.host_all, non_blocking=True)
 
     def h2d_bytes(self):
-        return self.host["x"].numel() * 2 + sum(e["hW"].numel() * 2 + e["hb"].numel() * 2 for e in self.lin)
+        return self.host_all.numel() * 2
 
     def nonzero_flops(self):
         self.torch.cuda.synchronize()
