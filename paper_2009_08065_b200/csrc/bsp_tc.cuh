@@ -160,10 +160,10 @@ __host__ __device__ constexpr uint32_t instr_desc_bf16(int n) {
 // GELU(x) = x * Phi(x), Phi the standard normal distribution function (the erf form, 0.5 (1 + erf(x / sqrt 2))).
 // The lower tail is evaluated as Phi(-a) = 2^(-P(a)), a = min(|x|, 6), with P a degree-5 polynomial
 // fitted by weighted least squares to -log2 Phi(-a) on [0, 6]; the largest absolute error of Phi in
-// float32 is 3.2e-7 (below 1e-9 beyond a = 6), so x Phi(x) is off by at most 2.3e-6 in absolute terms
-// (at |x| = 6), far under the bf16 rounding of the output.  One
+// float32 is 3.2e-7 (below 1e-9 beyond a = 6), so x Phi(x) is off by at most 2e-6 in absolute terms,
+// far under the bf16 rounding of the output except deep in the lower tail.  One
 // special-function operation (ex2) per element, no branch, no select: with q = Phi(-|x|),
-// x Phi(x) = x/2 + |x| (1/2 - q) for either sign of x.
+// x Phi(x) = max(x, 0) - |x| q for either sign of x.
 __device__ __forceinline__ float gelu_erf(float x) {
   const float a = fminf(fabsf(x), 6.0f);
   float p = fmaf(-0.000518865308f, a, 0.00738722592f);
@@ -173,8 +173,9 @@ __device__ __forceinline__ float gelu_erf(float x) {
   p = fmaf(p, a, -1.00000084f);
   float q;                                   // q = Phi(-|x|); the argument is in [-28, -1], far from any special case
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(q) : "f"(p));
-  // x Phi(x) = x/2 + |x| (1/2 - q) for either sign of x: no compare, no select
-  return fmaf(fabsf(x), 0.5f - q, 0.5f * x);
+  // x Phi(x) = max(x, 0) - |x| q for either sign of x: no compare, no select, and no cancellation
+  // in the lower tail (for x < 0 the result is -|x| q, rounded once)
+  return fmaf(-fabsf(x), q, fmaxf(x, 0.0f));
 }
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
