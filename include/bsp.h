@@ -215,6 +215,11 @@ int bsp_apply_mask(void* W, int rows, int cols, int ldw, int block, int orient,
  * and only vals changes: tile of block b = rows of the block restricted to its kept columns.
  * W: bf16 [rows, cols] (ldw); blk_ptr / idx as written by bsp_prune_pack; vals is overwritten.
  */
+/* bsp_dense_mask — Algorithm 2's mask loop, element by element: mask[i, j] = 0 if W[i, j] == 0 else 1
+ * (either sign of zero counts as zero).  W bf16 [rows, cols] (ldw), mask uint8 [rows, cols] (ldm).
+ * The per-group keep flags of bsp_prune_pack are this mask reduced over each group; the calls of
+ * this library take the flags, the dense mask is for callers that want Algorithm 2's own object. */
+int bsp_dense_mask(const void* W, int rows, int cols, int ldw, uint8_t* mask, int ldm, void* stream);
 int bsp_masked_adam_step(float* W, const float* grad, float* m, float* v, int rows, int cols, int ldw, int ldg,
                          const uint8_t* keep, int block, int orient,
                          float lr, float beta1, float beta2, float eps, float weight_decay, int step,

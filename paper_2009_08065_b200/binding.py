@@ -82,6 +82,7 @@ _SIGNATURES = {
     "bsp_transpose": (_i, [_vp, _i, _i, _i, _vp, _i, _vp]),
     "bsp_linear_gathered": (_i, [_vp, _i, _i, _i, _vp, _i, _i, _vp, _i, _vp, _i, _vp]),
     "bsp_masked_adam_step": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _vp, _i, _i, _f, _f, _f, _f, _f, _i, _vp, _i, _vp]),
+    "bsp_dense_mask": (_i, [_vp, _i, _i, _i, _vp, _i, _vp]),
     "bsp_repack_values": (_i, [_vp, _i, _i, _i, _i, _vp, _vp, _vp, _vp]),
     "bsp_prepare_batched": (_i, [ctypes.POINTER(_LayerJob), _i, _i, _f, _i, _vp]),
     "bsp_linear_plan_bytes": (_i, [_i, _i, _i, _szp]),
@@ -325,6 +326,12 @@ def bsp_masked_adam_step(W: torch.Tensor, grad: torch.Tensor, m: torch.Tensor, v
     _check(lib.bsp_masked_adam_step(_ptr(W), _ptr(grad), _ptr(m), _ptr(v), rows, cols, _ld(W), _ld(grad), _ptr(keep),
                                     block, orient, lr, beta1, beta2, eps, weight_decay, step, _ptr(W_bf16),
                                     0 if W_bf16 is None else _ld(W_bf16), _stream(stream)), "bsp_masked_adam_step")
+
+
+def bsp_dense_mask(W: torch.Tensor, mask: torch.Tensor, stream=None) -> None:
+    """mask (uint8, same shape as W) = 1 where the bf16 weight is non-zero."""
+    _check(lib.bsp_dense_mask(_ptr(W), W.shape[0], W.shape[1], _ld(W), _ptr(mask), _ld(mask), _stream(stream)),
+           "bsp_dense_mask")
 
 
 def bsp_repack_values(W: torch.Tensor, packed: PackedMatrix, stream=None) -> None:

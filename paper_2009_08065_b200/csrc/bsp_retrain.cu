@@ -1,6 +1,6 @@
 // Algorithm 2's retraining loop on the device: "update W ... using Adam", then "W = W * Mask", in
 // one pass (bsp_masked_adam_step), and the refresh of the packed values of Section 3.1's storage
-// under the fixed kept sets (bsp_repack_values).
+// under the fixed kept sets (bsp_repack_values); and the mask loop itself (bsp_dense_mask).
 //
 // Adam is taken as published (Kingma & Ba 2015, with bias correction); the paper gives no
 // hyper-parameters beyond the learning rate, so they are the caller's.  The weights that the
@@ -90,8 +90,30 @@ repack_kernel(const uint16_t* __restrict__ W, int ldw, int block, const int32_t*
       tile[static_cast<size_t>(r) * kc + p] = wblk[static_cast<size_t>(r) * ldw + __ldg(idx + lo + p)];
 }
 
+// Algorithm 2's mask loop: Mask_ij = 0 if W_ij == 0 else 1 (either sign of zero is zero).
+__global__ void __launch_bounds__(256)
+dense_mask_kernel(const uint16_t* __restrict__ W, int rows, int cols, int ldw, uint8_t* __restrict__ mask, int ldm) {
+  const long long e = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (e >= static_cast<long long>(rows) * cols) return;
+  const int r = static_cast<int>(e / cols), c = static_cast<int>(e - static_cast<long long>(r) * cols);
+  mask[static_cast<size_t>(r) * ldm + c] = (W[static_cast<size_t>(r) * ldw + c] & 0x7fffu) != 0 ? 1 : 0;
+}
+
 }  // namespace
 }  // namespace bsp
+
+extern "C" int bsp_dense_mask(const void* W, int rows, int cols, int ldw, uint8_t* mask, int ldm, void* stream) {
+  using namespace bsp;
+  if (W == nullptr || mask == nullptr || rows <= 0 || cols <= 0) return BSP_ERR_ARG;
+  if (ldw < cols || ldm < cols) return BSP_ERR_SHAPE;
+  const long long elems = static_cast<long long>(rows) * cols;
+  const long long blocks = (elems + 255) / 256;
+  if (blocks > 0x7fffffffLL) return BSP_ERR_UNSUPPORTED;
+  dense_mask_kernel<<<static_cast<unsigned>(blocks), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<const uint16_t*>(W), rows, cols, ldw, mask, ldm);
+  BSP_LAUNCH_CHECK();
+  return BSP_OK;
+}
 
 extern "C" int bsp_masked_adam_step(float* W, const float* grad, float* m, float* v, int rows, int cols, int ldw,
                                     int ldg, const uint8_t* keep, int block, int orient, float lr, float beta1,

@@ -160,6 +160,8 @@ def test_retraining_entry_points_reject_bad_arguments_without_a_gpu():
     assert lib.bsp_masked_adam_step(*args(keep=p, block=3)) == -2                            # 3 does not divide 8
     assert lib.bsp_masked_adam_step(*args(cols=6, ldw=8)) == -6                              # cols not a multiple of 4
     assert lib.bsp_repack_values(p, 8, 8, 8, 4, None, p, p, None) == -1
+    assert lib.bsp_dense_mask(p, 8, 8, 8, None, 8, None) == -1
+    assert lib.bsp_dense_mask(p, 8, 8, 4, p, 8, None) == -2
     assert lib.bsp_repack_values(p, 8, 8, 8, 3, p, p, p, None) == -2
 
 

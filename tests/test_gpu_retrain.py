@@ -111,3 +111,24 @@ def test_repack_values_small_blocks_and_empty_blocks():
     ptr2, idx2, vals2, _, _ = packed_to_host(pk)
     assert np.array_equal(ptr2, ptr) and np.array_equal(idx2, idx)
     assert np.array_equal(vals2, O.repack_values(w2, ptr, idx, d))
+
+
+def test_dense_mask_is_algorithm_2s_mask():
+    """Mask_ij = (W_ij != 0), negative zero included, on a ragged shape with a padded leading dimension; and
+    its reduction over the groups is what bsp_prune_pack calls the keep flags at threshold 0."""
+    rows, cols, d = 96, 50, 12
+    spec = si.LinearSpec("dmask", rows, cols, False, 2.0, d)
+    wp, keep = si.make_pruned_weight(56, spec)
+    wp[5, 7] = 0x8000                                              # -0.0 is zero
+    wide = np.zeros((rows, 64), dtype=np.uint16)
+    wide[:, :cols] = wp
+    wd = to_dev(wide)[:, :cols]                                    # leading dimension 64
+    mask = torch.full((rows, cols), 9, dtype=torch.uint8, device=DEV)
+    bsp.bsp_dense_mask(wd, mask)
+    torch.cuda.synchronize()
+    ref = O.mask_of(wp)
+    assert np.array_equal(mask.cpu().numpy().astype(bool), ref) and mask.max().item() == 1
+    pk = bsp.PackedMatrix.allocate(rows, cols, d, bsp.ORIENT_C, DEV)
+    bsp.bsp_prune_pack(to_dev(wp), pk, 0.0)
+    torch.cuda.synchronize()
+    assert np.array_equal(pk.keep.cpu().numpy().astype(bool), O.group_any(ref, d, "C"))
