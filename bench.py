@@ -392,6 +392,17 @@ def run_cuda(args):
     layer.bsp.bsp_linear_status()
     total_ms = sum(step_ms)
 
+    # the same step back to back without the flush: W, X and the intermediate outputs (about 100 MB) are
+    # still in L2 from the previous step.  Context beside `value`, which is the flushed figure.
+    w_s, w_e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    graph.replay()
+    w_s.record()
+    for _ in range(20):
+        graph.replay()
+    w_e.record()
+    torch.cuda.synchronize()
+    warm_ms = w_s.elapsed_time(w_e) / 20
+
     # end to end: pinned host inputs -> device, the step, result back to the host, every step.
     # (a) one step at a time: copy in, compute, copy out, in order on one stream;
     # (b) double-buffered, as a caller that feeds batches continuously would run it: two sets of device
@@ -486,6 +497,8 @@ def run_cuda(args):
                 "nonzero_gflop_per_step_per_gpu": round(step_flops / 1e9, 3),
             },
             "percent_of_bf16_peak": round(100 * value / world / peak, 2),
+            "warm_l2": {"ms_per_step": round(warm_ms, 5), "value": round(step_flops / warm_ms / 1e9, 2), "unit": UNIT,
+                        "how": "rank 0, 20 steps back to back, no flush between them"},
             "e2e": {"value": round(job_throughput(world, step_flops, args.steps, e2e_total_ms), 3), "unit": UNIT,
                     "h2d_bytes_per_step": layer.h2d_bytes(),
                     "d2h_bytes_per_step": y_host.numel() * 2 + pen_host.numel() * 8,
