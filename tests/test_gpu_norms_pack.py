@@ -303,6 +303,41 @@ def test_prepare_batched_streaming_batch_larger_than_the_gpu():
             job.penalty.fill_(-5.0)
 
 
+@pytest.mark.parametrize("block", [3, 12, 96])
+def test_prepare_batched_paper_block_heights(block):
+    """The paper's block sizes (3, 12 and 96 rows): at 96 rows a row-block no longer fits the kernel's row
+    buffer and is split into six column ranges that wait for one another's counts."""
+    eps = 1e-3
+    jobs, refs = [], []
+    for n, (rows, cols) in enumerate([(768, 768), (96 * 4, 3072), (96, 72)]):
+        w = si.student_t_bf16(500 + n, f"paperblk{block}_{n}", (rows, cols), 3.0, 0.02)
+        t_b = float(np.quantile(O.group_norms(w, block, "C"), 0.5))
+        pk = bsp.PackedMatrix.allocate(rows, cols, block, bsp.ORIENT_C, DEV)
+        shape = (rows // block, cols)
+        jobs.append(bsp.LayerJob(W=to_dev(w), out=pk, threshold=t_b,
+                                 norms=torch.empty(shape, dtype=torch.float32, device=DEV),
+                                 gamma_out=torch.empty(shape, dtype=torch.float32, device=DEV),
+                                 penalty=torch.zeros(1, dtype=torch.float64, device=DEV),
+                                 plan=torch.empty(bsp.bsp_linear_plan_bytes(rows, cols, block), dtype=torch.uint8, device=DEV)))
+        refs.append((w, t_b))
+    bsp.bsp_prepare_batched(jobs, block, eps, bsp.PEN_L2)
+    bsp.bsp_linear_status()
+    torch.cuda.synchronize()
+    for job, (w, t_b) in zip(jobs, refs):
+        rows, cols = w.shape
+        n_ref = O.group_norms(w, block, "C")
+        assert np.allclose(job.norms.cpu().numpy(), n_ref, rtol=REL, atol=0)
+        assert np.allclose(job.gamma_out.cpu().numpy(), O.gamma_update(n_ref, eps), rtol=REL, atol=0)
+        assert float(job.penalty.item()) == pytest.approx(O.penalty_l2(n_ref, O.gamma_update(n_ref, eps)), rel=REL)
+        keep_ref = O.keep_flags(w, block, "C", t_b)
+        ref_ptr, ref_idx, ref_vals = O.pack(w, keep_ref, block, "C")
+        blk_ptr, idx, vals, keep, kept = packed_to_host(job.out)
+        assert np.array_equal(keep, keep_ref) and np.array_equal(blk_ptr, ref_ptr)
+        assert np.array_equal(idx, ref_idx) and np.array_equal(vals, ref_vals)
+        plan = bits_of(job.plan.view(torch.int16)[: rows * cols].reshape(rows, cols))
+        assert np.array_equal(plan, O.prune(w, block, "C", t_b))
+
+
 def test_prepare_batched_with_device_side_percentile_thresholds():
     """The heavy-tailed workload's recipe in batched form (32-row blocks, 1.79x): every matrix's threshold is
     found on the device (bsp_percentile_threshold) and read from there by the one batched call; kept counts
