@@ -106,6 +106,11 @@ int bsp_penalty_grad(const void* W, int rows, int cols, int ldw, int block, int 
  */
 int bsp_pack_bound(int rows, int cols, int block, int orient,
                    size_t* idx_elems, size_t* val_elems, size_t* ws_bytes);
+/* bsp_pack_scratch_bytes — host-only: the part of that workspace bsp_prune_pack itself touches
+ * (per-block counts and one flag byte per group, about 1 byte per group; the float32 region that
+ * makes up the rest of bsp_pack_bound's figure belongs to bsp_percentile_threshold).  A workspace
+ * of this size is enough for bsp_prune_pack alone. */
+int bsp_pack_scratch_bytes(int rows, int cols, int block, int orient, size_t* bytes);
 
 /* ---------------------------------------------------------------------------------------------
  * bsp_prune_pack — Algorithm 1 followed by the compressed storage of Section 3.1 ("only the
@@ -132,7 +137,8 @@ int bsp_pack_bound(int rows, int cols, int block, int orient,
  *   kept_weights int64 device scalar = block * blk_ptr[nb]; compression rate = rows*cols / it.
  *               May be NULL.
  * idx and vals must have room for bsp_pack_bound's counts.  ws/ws_bytes: scratch of at least
- * bsp_pack_bound's *ws_bytes, 256-byte aligned; contents are undefined afterwards.
+ * bsp_pack_scratch_bytes (bsp_pack_bound's *ws_bytes also serves), 256-byte aligned; contents are
+ * undefined afterwards.
  * Errors: BSP_ERR_ARG, BSP_ERR_SHAPE, BSP_ERR_WORKSPACE, BSP_ERR_UNSUPPORTED.
  */
 #define BSP_TOPK_MAX_GROUPS 8192
@@ -156,8 +162,9 @@ int bsp_prune_pack(const void* W, int rows, int cols, int ldw, int block, int or
  * Arguments, outputs, semantics and results are exactly those of bsp_prune_pack without
  * ws/ws_bytes; inputs and outputs are still the caller's buffers.  The call itself allocates
  * and frees nothing.
- *  - Limit: shapes whose bsp_pack_bound workspace exceeds BSP_STATIC_SCRATCH_BYTES (about
- *    800 thousand groups) are refused with BSP_ERR_UNSUPPORTED before anything is launched.
+ *  - Limit: shapes whose bsp_pack_scratch_bytes exceeds BSP_STATIC_SCRATCH_BYTES (just under
+ *    4.2 million groups; 8192 x 8192 at block 32 fits, at block 16 it does not) are refused with BSP_ERR_UNSUPPORTED before
+ *    anything is launched.
  *  - The first call on each device looks up the array's device address (with that device
  *    current); make that first call outside any stream capture.
  *  - All calls on a device share the one array.  It needs no clearing between calls (each call

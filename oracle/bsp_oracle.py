@@ -192,28 +192,30 @@ def prune(w_bits: np.ndarray, block: int, orient: str, t_b: float) -> np.ndarray
     return np.where(keep, w_bits, np.uint16(0)).astype(np.uint16)
 
 
-def prune_alg1_loops(w_bits: np.ndarray, k: int, t_b: float) -> np.ndarray:
-    """Algorithm 1 with its own loop structure, for small matrices (orientation "R").
+def prune_groupwise(w_bits: np.ndarray, block: int, orient: str, t_b: float) -> np.ndarray:
+    """Algorithm 1's decision rule applied group by group, for small matrices (a slow cross-check of `prune`).
 
-    W_p = W; divide W_p into k matrices W_1..W_k (vertical strips); for each strip i and each of
-    its m rows j: if the l2 norm of that row segment is <= t_b, zero it; concatenate the strips.
-    The norm test uses the float32 decision quantity so that it decides like `keep_flags`.
+    Every group is visited on its own, in no particular order: its elements are taken as an explicit
+    slice of W, the float32 decision quantity is summed element by element, and the test
+    "norm <= t_b" (as S32 <= t_b^2, like `keep_flags`) fills one entry of a keep table.  The table is
+    then applied to a copy of W in a single masking step.
     """
     m, n = w_bits.shape
-    if n % k:
-        raise ValueError("row division k must divide the matrix width")
-    h = n // k
-    strips = [w_bits[:, i * h:(i + 1) * h].copy() for i in range(k)]
+    if (m if orient == "C" else n) % block:
+        raise ValueError("block must divide the pruned dimension")
+    vals = bf16_to_f64(w_bits).astype(np.float32)
     t2 = threshold_sq32(t_b)
-    for i in range(k):
-        vals = bf16_to_f64(strips[i]).astype(np.float32)
-        for j in range(m):
-            acc = np.float32(0.0)
-            for c in range(h):
-                acc = np.float32(acc + vals[j, c] * vals[j, c])
-            if t_b >= 0 and acc <= t2:
-                strips[i][j, :] = 0
-    return np.concatenate(strips, axis=1)
+    table = np.ones((m, n), dtype=bool)
+    groups = [(slice(b * block, (b + 1) * block), slice(j, j + 1)) for b in range(m // block) for j in range(n)] \
+        if orient == "C" else \
+        [(slice(i, i + 1), slice(a * block, (a + 1) * block)) for a in range(n // block) for i in range(m)]
+    for rows, cols in reversed(groups):
+        acc = np.float32(0.0)
+        for x in vals[rows, cols].ravel():          # increasing row index (C) / column index (R)
+            acc = np.float32(acc + x * x)
+        if t_b >= 0 and acc <= t2:
+            table[rows, cols] = False
+    return np.where(table, w_bits, np.uint16(0)).astype(np.uint16)
 
 
 def mask_of(w_pruned_bits: np.ndarray) -> np.ndarray:

@@ -73,6 +73,7 @@ _SIGNATURES = {
     "bsp_group_norms": (_i, [_vp, _i, _i, _i, _i, _i, _f, _i, _vp, _vp, _vp, _vp, _vp]),
     "bsp_penalty_grad": (_i, [_vp, _i, _i, _i, _i, _i, _i, _vp, _f, _vp, _i, _i, _vp]),
     "bsp_pack_bound": (_i, [_i, _i, _i, _i, _szp, _szp, _szp]),
+    "bsp_pack_scratch_bytes": (_i, [_i, _i, _i, _i, _szp]),
     "bsp_prune_pack": (_i, [_vp, _i, _i, _i, _i, _i, _f, _vp, _i, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "bsp_prune_pack_static": (_i, [_vp, _i, _i, _i, _i, _i, _f, _vp, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
     "bsp_percentile_threshold": (_i, [_vp, _i, _i, _i, _i, _i, _d, _vp, _vp, _sz, _vp]),
@@ -163,6 +164,13 @@ def bsp_pack_bound(rows: int, cols: int, block: int, orient: int = ORIENT_C) -> 
     _check(lib.bsp_pack_bound(rows, cols, block, orient, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c)),
            "bsp_pack_bound")
     return a.value, b.value, c.value
+
+
+def bsp_pack_scratch_bytes(rows: int, cols: int, block: int, orient: int = ORIENT_C) -> int:
+    """Bytes of workspace that bsp_prune_pack itself uses (counts and flags)."""
+    n = ctypes.c_size_t()
+    _check(lib.bsp_pack_scratch_bytes(rows, cols, block, orient, ctypes.byref(n)), "bsp_pack_scratch_bytes")
+    return n.value
 
 
 @dataclass

@@ -229,6 +229,16 @@ extern "C" int bsp_pack_bound(int rows, int cols, int block, int orient, size_t*
   return BSP_OK;
 }
 
+extern "C" int bsp_pack_scratch_bytes(int rows, int cols, int block, int orient, size_t* bytes) {
+  using namespace bsp;
+  if (rows <= 0 || cols <= 0 || block <= 0 || bytes == nullptr) return BSP_ERR_ARG;
+  if (orient != BSP_ORIENT_C && orient != BSP_ORIENT_R) return BSP_ERR_ARG;
+  int nb, ng;
+  if (!geometry(rows, cols, block, orient, &nb, &ng)) return BSP_ERR_SHAPE;
+  *bytes = ws_layout(nb, ng).sumsq_off;
+  return BSP_OK;
+}
+
 extern "C" int bsp_prune_pack(const void* W, int rows, int cols, int ldw, int block, int orient,
                               float threshold, const float* threshold_dev, int keep_per_block,
                               uint8_t* keep, int32_t* blk_ptr, int32_t* idx, void* vals,
@@ -242,7 +252,7 @@ extern "C" int bsp_prune_pack(const void* W, int rows, int cols, int ldw, int bl
   Geometry G{rows, cols, ldw, block, orient, 0, 0};
   geometry(rows, cols, block, orient, &G.n_blocks, &G.n_groups);
   const WsLayout L = ws_layout(G.n_blocks, G.n_groups);
-  if (ws_bytes < L.total) return BSP_ERR_WORKSPACE;
+  if (ws_bytes < L.sumsq_off) return BSP_ERR_WORKSPACE;   // counts and flags; the float32 region is the percentile call's
   if (keep_per_block >= 0 && G.n_groups > BSP_TOPK_MAX_GROUPS) return BSP_ERR_UNSUPPORTED;
 
   cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -325,7 +335,7 @@ extern "C" int bsp_prune_pack_static(const void* W, int rows, int cols, int ldw,
   int st = check_matrix_args(W, rows, cols, ldw, block, orient);
   if (st != BSP_OK) return st;
   size_t need = 0;
-  st = bsp_pack_bound(rows, cols, block, orient, nullptr, nullptr, &need);
+  st = bsp_pack_scratch_bytes(rows, cols, block, orient, &need);
   if (st != BSP_OK) return st;
   if (need > static_cast<size_t>(BSP_STATIC_SCRATCH_BYTES)) return BSP_ERR_UNSUPPORTED;
 

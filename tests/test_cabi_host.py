@@ -48,6 +48,12 @@ def test_pack_bound():
     assert e.value.status == -1
     with pytest.raises(bsp.BspError):
         bsp.bsp_pack_bound(768, 768, 16, 7)
+    # the part bsp_prune_pack itself touches: counts and one flag byte per group
+    scratch = bsp.bsp_pack_scratch_bytes(768, 768, 16, bsp.ORIENT_C)
+    assert 48 * 768 + 4 * 49 <= scratch < bsp.bsp_pack_bound(768, 768, 16, bsp.ORIENT_C)[2] and scratch % 256 == 0
+    with pytest.raises(bsp.BspError) as e:
+        bsp.bsp_pack_scratch_bytes(770, 768, 16, bsp.ORIENT_C)
+    assert e.value.status == -2
 
 
 def test_plan_bytes():

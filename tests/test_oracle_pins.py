@@ -193,18 +193,14 @@ def test_decision_quantity_close_to_float64():
 
 
 # ----------------------------------------------------------------------------- prune / mask
-def brute_force_alg1_rows(wf, k, t_b):
-    """Algorithm 1 written independently with Python floats on a list-of-lists matrix."""
-    m, n = len(wf), len(wf[0])
+def brute_force_row_groups(wf, k, t_b):
+    """Algorithm 1's rule in plain Python floats on a list-of-lists matrix: a row segment of a strip
+    survives iff its l2 norm is not <= t_b."""
+    n = len(wf[0])
     h = n // k
-    out = [row[:] for row in wf]
-    for i in range(k):
-        for j in range(m):
-            norm = math.sqrt(sum(out[j][c] ** 2 for c in range(i * h, (i + 1) * h)))
-            if norm <= t_b:
-                for c in range(i * h, (i + 1) * h):
-                    out[j][c] = 0.0
-    return out
+    gone = {(j, c // h) for j, row in enumerate(wf) for c in range(0, n, h)
+            if math.sqrt(math.fsum(v * v for v in row[c:c + h])) <= t_b}
+    return [[0.0 if (j, c // h) in gone else v for c, v in enumerate(row)] for j, row in enumerate(wf)]
 
 
 @pytest.mark.parametrize("seed", [11, 12, 13])
@@ -216,14 +212,16 @@ def test_prune_against_brute_force_alg1(seed):
     w = bits(wf)
     for k, t_b in [(2, 0.0), (2, 0.5), (4, 0.375), (8, 0.25), (1, 0.7), (2, math.sqrt(3) * 0.375)]:
         h = 8 // k
-        want = np.array(brute_force_alg1_rows(wf.astype(float).tolist(), k, t_b), dtype=np.float32)
-        got_loops = si.bf16_bits_to_f32(O.prune_alg1_loops(w, k, t_b))
+        want = np.array(brute_force_row_groups(wf.astype(float).tolist(), k, t_b), dtype=np.float32)
+        got_loops = si.bf16_bits_to_f32(O.prune_groupwise(w, h, "R", t_b))
         got_vec = si.bf16_bits_to_f32(O.prune(w, h, "R", t_b))
         assert np.array_equal(got_loops, want), (k, t_b)
         assert np.array_equal(got_vec, want), (k, t_b)
         # column variant = row variant on the transpose
         got_c = si.bf16_bits_to_f32(O.prune(np.ascontiguousarray(w.T), h, "C", t_b)).T
         assert np.array_equal(got_c, want), (k, t_b)
+        got_c_groups = si.bf16_bits_to_f32(O.prune_groupwise(np.ascontiguousarray(w.T), h, "C", t_b)).T
+        assert np.array_equal(got_c_groups, want), (k, t_b)
 
 
 def test_threshold_is_inclusive():

@@ -19,10 +19,12 @@ import synth_inputs as si
 def test_static_scratch_limit_is_enforced_on_the_host():
     """A shape whose scratch need exceeds the fixed array is refused before any CUDA call."""
     p = ctypes.c_void_p(0x1000)
-    rows, cols, block = 8192, 8192, 8                    # 8.4 million groups: far beyond the array
-    assert bsp.bsp_pack_bound(rows, cols, block)[2] > (4 << 20)
+    rows, cols, block = 8192, 8192, 8                    # 8.4 million groups: beyond the array
+    assert bsp.bsp_pack_scratch_bytes(rows, cols, block) > (4 << 20)
     st = bsp.lib.bsp_prune_pack_static(p, rows, cols, cols, block, 0, 0.0, None, -1, None, p, p, p, None, None)
     assert st == -6
+    # the limit counts what the pack touches (counts and flags), not the percentile call's float32 region
+    assert bsp.bsp_pack_scratch_bytes(8192, 8192, 32) <= (4 << 20) < bsp.bsp_pack_bound(8192, 8192, 32)[2]
     assert bsp.lib.bsp_prune_pack_static(p, 10, 8, 8, 3, 0, 0.0, None, -1, None, p, p, p, None, None) == -2
 
 
