@@ -280,8 +280,8 @@ int bsp_prepare_batched(const bsp_layer_job* jobs, int n_jobs, int block, float 
  *
  * Alignment for the tensor-core path: X, Y and plan 16-byte aligned, k_in, ldx and ldy multiples
  * of 8 elements.  Other cases run on a slower CUDA-core kernel with identical semantics.
- * Device-side waits in the tensor-core kernel are bounded; if one expires the kernel stops
- * early and records it: bsp_linear_status (host; synchronises the stream) then returns
+ * Device-side waits in the tensor-core kernel are bounded (bsp_set_wait_limit_ms); if one expires
+ * the kernel stops early and records it: bsp_linear_status (host; synchronises the stream) then returns
  * BSP_ERR_TIMEOUT and Y is undefined.  It returns BSP_OK otherwise.
  * Errors: BSP_ERR_ARG, BSP_ERR_SHAPE (block does not divide n_out), BSP_ERR_WORKSPACE, BSP_ERR_CUDA.
  */
@@ -329,6 +329,21 @@ int bsp_linear(const int32_t* blk_ptr, const int32_t* idx, const void* vals,
                const void* X, int tokens, int ldx, const void* bias, int act,
                void* Y, int ldy, void* ws, size_t ws_bytes, void* stream);
 int bsp_linear_status(void* stream);
+/* bsp_set_wait_limit_ms — how long one device-side wait of the tensor-core and batched weight-side
+ * kernels may last before the kernel gives up (default 2000; 1 <= ms <= 600000), for kernels
+ * launched afterwards on the current device.  Host call; synchronises the device first, so kernels
+ * already in flight keep the limit they started with.  Errors: BSP_ERR_ARG, BSP_ERR_CUDA.
+ *
+ * bsp_wait_selftest — runs the bail-out path once, without any fault: a single CTA sets up an
+ * mbarrier and tensor memory as the tensor-core kernels do, then waits through the same bounded-wait
+ * helpers on a barrier and on a counter that nothing ever signals.  Both waits run out at the
+ * configured limit; the CTA records it, sits out a fixed millisecond for operations in flight, frees
+ * its tensor memory and returns by itself.  Afterwards bsp_linear_status returns BSP_ERR_TIMEOUT once
+ * and BSP_OK again from then on.  *expired (host, may be NULL) receives the number of waits that ran
+ * out (2), *waited_ns (host, may be NULL) how long the mbarrier wait lasted.  Synchronises the stream;
+ * takes about the wait limit, so lower the limit first. */
+int bsp_set_wait_limit_ms(int ms);
+int bsp_wait_selftest(int* expired, long long* waited_ns, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
  * bsp_linear_chain — several pruned linear layers, each reading the chain input or an earlier

@@ -14,5 +14,5 @@ from .binding import (  # noqa: F401
     LINEAR_AUTO, LINEAR_ONE_CTA, LINEAR_CTA_PAIR, bsp_linear, bsp_linear_status, bsp_linear_chain, bsp_linear_chain_ws_bytes,
     bsp_linear_gather_plan_bytes, bsp_linear_gather_plan, bsp_transpose, bsp_linear_gathered,
     bsp_masked_adam_step, bsp_repack_values, bsp_dense_mask,
-    bsp_linear_cuda_core, bsp_status_string,
+    bsp_linear_cuda_core, bsp_status_string, bsp_set_wait_limit_ms, bsp_wait_selftest,
 )

@@ -97,6 +97,8 @@ _SIGNATURES = {
     "bsp_linear_chain_ws_bytes": (_i, [_i, _i, _szp]),
     "bsp_linear_chain": (_i, [ctypes.POINTER(_ChainOp), _i, _vp, _i, _i, _vp, _sz, _vp]),
     "bsp_linear_status": (_i, [_vp]),
+    "bsp_set_wait_limit_ms": (_i, [_i]),
+    "bsp_wait_selftest": (_i, [ctypes.POINTER(_i), ctypes.POINTER(ctypes.c_longlong), _vp]),
     "bsp_linear_cuda_core": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _i, _i, _vp, _i, _vp, _i, _vp]),
 }
 for _name, (_res, _args) in _SIGNATURES.items():
@@ -420,3 +422,16 @@ def bsp_linear_cuda_core(packed: PackedMatrix, X: torch.Tensor, bias: Optional[t
 def bsp_linear_status(stream=None) -> None:
     """Synchronises the stream; raises BspError(BSP_ERR_TIMEOUT) if a tensor-core launch gave up on a wait."""
     _check(lib.bsp_linear_status(_stream(stream)), "bsp_linear_status")
+
+
+def bsp_set_wait_limit_ms(ms: int) -> None:
+    """Limit of one device-side wait for kernels launched afterwards on the current device (default 2000 ms)."""
+    _check(lib.bsp_set_wait_limit_ms(int(ms)), "bsp_set_wait_limit_ms")
+
+
+def bsp_wait_selftest(stream=None) -> Tuple[int, int]:
+    """Lets one CTA's bounded waits run out on purpose-made idle barriers; returns (waits that ran out, ns the
+    mbarrier wait lasted).  bsp_linear_status reports BSP_ERR_TIMEOUT once afterwards."""
+    n, ns = ctypes.c_int(0), ctypes.c_longlong(0)
+    _check(lib.bsp_wait_selftest(ctypes.byref(n), ctypes.byref(ns), _stream(stream)), "bsp_wait_selftest")
+    return n.value, ns.value

@@ -41,7 +41,6 @@ constexpr int kStreamMaxJobs = 96;       // per launch; the job table travels as
 constexpr int kStreamThreads = 128;
 constexpr int kStreamRowBytes = 24 * 1024;   // the row buffer
 constexpr int kReadyBit = 0x40000000;    // set in a published count
-constexpr unsigned long long kSpinLimitNs = 2000000000ull;   // 2 s per wait
 
 struct StreamJob {
   FusedJob j;
@@ -101,6 +100,7 @@ __device__ __forceinline__ int wait_count(const int32_t* slot, int* status) {
   int v;
   asm volatile("ld.relaxed.gpu.global.b32 %0, [%1];" : "=r"(v) : "l"(slot) : "memory");
   if (v & kReadyBit) return v & (kReadyBit - 1);
+  const unsigned long long limit = tc::wait_limit_ns(status);
   const unsigned long long start = tc::global_timer_ns();
   for (;;) {
 #pragma unroll 1
@@ -109,7 +109,7 @@ __device__ __forceinline__ int wait_count(const int32_t* slot, int* status) {
       if (v & kReadyBit) return v & (kReadyBit - 1);
       __nanosleep(32);
     }
-    if (tc::global_timer_ns() - start > kSpinLimitNs) { atomicExch(status, BSP_ERR_TIMEOUT); return 0; }
+    if (tc::global_timer_ns() - start > limit) { atomicExch(status, BSP_ERR_TIMEOUT); return 0; }
   }
 }
 
@@ -118,6 +118,7 @@ __device__ __forceinline__ double wait_partial(const unsigned long long* slot, i
   unsigned long long v;
   asm volatile("ld.relaxed.gpu.global.b64 %0, [%1];" : "=l"(v) : "l"(slot) : "memory");
   if (v & 1ull) return __longlong_as_double(static_cast<long long>(v));
+  const unsigned long long limit = tc::wait_limit_ns(status);
   const unsigned long long start = tc::global_timer_ns();
   for (;;) {
 #pragma unroll 1
@@ -126,7 +127,7 @@ __device__ __forceinline__ double wait_partial(const unsigned long long* slot, i
       if (v & 1ull) return __longlong_as_double(static_cast<long long>(v));
       __nanosleep(32);
     }
-    if (tc::global_timer_ns() - start > kSpinLimitNs) { atomicExch(status, BSP_ERR_TIMEOUT); return 0.0; }
+    if (tc::global_timer_ns() - start > limit) { atomicExch(status, BSP_ERR_TIMEOUT); return 0.0; }
   }
 }
 
@@ -166,8 +167,12 @@ fused_stream_kernel(const __grid_constant__ StreamBatch B) {
     const int chunks = pc >> 3;
     const uint16_t* s_w = reinterpret_cast<const uint16_t*>(s_raw);                     // [d][pc]
     uint8_t* s_flag = reinterpret_cast<uint8_t*>(s_idx + O.part_cols);                  // [pc]
-    if (!mbar_wait(bar, 0u)) {
-      atomicExch(B.status, BSP_ERR_TIMEOUT);
+    // one decision for the whole CTA; if the rows never arrived, hold the buffer a millisecond for
+    // copies that may still be on their way, then leave
+    if (!__syncthreads_and(mbar_wait(bar, 0u, B.status) ? 1 : 0)) {
+      if (threadIdx.x == 0) atomicExch(B.status, BSP_ERR_TIMEOUT);
+      const unsigned long long start = tc::global_timer_ns();
+      while (tc::global_timer_ns() - start < tc::kQuietNs) __nanosleep(2000);
       return;
     }
 

@@ -52,6 +52,7 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant
   uint16_t* s_zero = reinterpret_cast<uint16_t*>(smem + S * Cfg::kStage + kEpiBytes);       // zero "bias"
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S * Cfg::kStage + kEpiBytes + 2 * kTnBN * 2);
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 2 * S + 4);
+  volatile uint32_t* timed_out = tmem_holder + 1;     // set by a role whose wait expired
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t smem_base = smem_u32(smem);
@@ -62,6 +63,7 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant
   auto acc_empty_bar = [&](int a) { return bar_base + 8u * (2 * S + 2 + a); };
 
   if (threadIdx.x == 0) {
+    *timed_out = 0u;
     for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 2); mbar_init(empty_bar(s), 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(acc_full_bar(a), 1); mbar_init(acc_empty_bar(a), 8); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -94,7 +96,7 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
       const int m0 = (tile / n_tiles) * kBlockM;
       for (int kb = 0; kb < k_blocks; ++kb) {
-        if (!mbar_wait(empty_bar(stage), phase ^ 1u)) { ok = false; break; }
+        if (!mbar_wait(empty_bar(stage), phase ^ 1u, P.status)) { ok = false; break; }
         const uint32_t a_dst = smem_base + stage * Cfg::kStage;
         mbar_arrive_expect_tx(full_bar(stage), Cfg::kStageA);
 #pragma unroll
@@ -103,7 +105,7 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant
         if (++stage == S) { stage = 0; phase ^= 1u; }
       }
     }
-    if (!ok) atomicExch(P.status, BSP_ERR_TIMEOUT);
+    if (!ok) record_timeout(P.status, timed_out);
   } else if (warp == 10 && lane == 0) {
     // ---------------------------------------------------------------- TMA producer of the X tiles
     int stage = 0;
@@ -112,7 +114,7 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
       const int n0 = (tile % n_tiles) * kTnBN;
       for (int kb = 0; kb < k_blocks; ++kb) {
-        if (!mbar_wait(empty_bar(stage), phase ^ 1u)) { ok = false; break; }
+        if (!mbar_wait(empty_bar(stage), phase ^ 1u, P.status)) { ok = false; break; }
         const uint32_t b_dst = smem_base + stage * Cfg::kStage + Cfg::kStageA;
         mbar_arrive_expect_tx(full_bar(stage), Cfg::kStageB);
 #pragma unroll
@@ -121,7 +123,7 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant
         if (++stage == S) { stage = 0; phase ^= 1u; }
       }
     }
-    if (!ok) atomicExch(P.status, BSP_ERR_TIMEOUT);
+    if (!ok) record_timeout(P.status, timed_out);
   } else if (warp == 1 && lane == 0) {
     // ---------------------------------------------------------------- MMA issuer
     int stage = 0;
@@ -130,11 +132,11 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant
     int acc = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-      if (!mbar_wait(acc_empty_bar(acc), acc_phase[acc] ^ 1u)) { ok = false; break; }
+      if (!mbar_wait(acc_empty_bar(acc), acc_phase[acc] ^ 1u, P.status)) { ok = false; break; }
       tcgen05_fence_after();
       const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * kTnBN);
       for (int kb = 0; kb < k_blocks; ++kb) {
-        if (!mbar_wait(full_bar(stage), phase)) { ok = false; break; }
+        if (!mbar_wait(full_bar(stage), phase, P.status)) { ok = false; break; }
         tcgen05_fence_after();
         const uint32_t a_addr = smem_base + stage * Cfg::kStage;
         const uint32_t b_addr = a_addr + Cfg::kStageA;
@@ -150,7 +152,7 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant
       acc_phase[acc] ^= 1u;
       acc ^= 1;
     }
-    if (!ok) atomicExch(P.status, BSP_ERR_TIMEOUT);
+    if (!ok) record_timeout(P.status, timed_out);
   } else if (warp >= 2 && warp < 10) {
     // ---------------------------------------------------------------- epilogue (as in bsp_linear_tc.cu, no bias)
     const int group = (warp - 2) >> 2;
@@ -167,7 +169,8 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant
     bool ok = true;
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
       const int m0 = (tile / n_tiles) * kBlockM, n0 = (tile % n_tiles) * kTnBN;
-      if (!mbar_wait(acc_full_bar(acc), acc_phase[acc])) { ok = false; break; }
+      // all 256 threads take the same decision, so nobody is left alone at a named barrier below
+      if (!epilogue_all_ok(mbar_wait(acc_full_bar(acc), acc_phase[acc], P.status))) { ok = false; break; }
       tcgen05_fence_after();
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + static_cast<uint32_t>(acc * kTnBN);
       const int pieces = (min(kTnBN, P.k_in - n0) + kEpiCols - 1) / kEpiCols;
@@ -204,11 +207,12 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant
       acc ^= 1;
     }
     if (issuer) tma_store_wait_read<0>();
-    if (!ok && lane == 0) atomicExch(P.status, BSP_ERR_TIMEOUT);
+    if (!ok && lane == 0) record_timeout(P.status, timed_out);
   }
 
   tcgen05_fence_before();
   __syncthreads();
+  quiet_period(timed_out);
   if (warp == 1) {
     tcgen05_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),

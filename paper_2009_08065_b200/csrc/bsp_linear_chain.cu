@@ -57,20 +57,6 @@ __device__ __forceinline__ TileRef decode_tile(const ChainParams& P, int t) {
   return TileRef{g, m, local - m * P.op[g].n_tiles};
 }
 
-// Bounded wait until *counter >= need (acquire at GPU scope).
-__device__ __forceinline__ bool wait_counter(const int* counter, int need) {
-  const unsigned long long start = global_timer_ns();
-  for (;;) {
-#pragma unroll 1
-    for (int i = 0; i < 64; ++i) {
-      int v;
-      asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(counter) : "memory");
-      if (v >= need) return true;
-    }
-    if (global_timer_ns() - start > kWaitLimitNs) return false;
-  }
-}
-
 __global__ void __launch_bounds__(kThreads, 1)
 linear_chain_kernel(const __grid_constant__ ChainMaps M, const __grid_constant__ ChainParams P) {
   constexpr int S = Cfg::kStages;
@@ -79,6 +65,7 @@ linear_chain_kernel(const __grid_constant__ ChainMaps M, const __grid_constant__
   // [S operand stages][2 epilogue staging buffers][bias, bf16, for two tiles][mbarriers, TMEM base]
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S * Cfg::kStage + kEpiBytes + 2 * kBN * 2);
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 2 * S + 4);
+  volatile uint32_t* timed_out = tmem_holder + 1;     // set by a role whose wait expired
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t smem_base = smem_u32(smem);
@@ -89,6 +76,7 @@ linear_chain_kernel(const __grid_constant__ ChainMaps M, const __grid_constant__
   auto acc_empty_bar = [&](int a) { return bar_base + 8u * (2 * S + 2 + a); };
 
   if (threadIdx.x == 0) {
+    *timed_out = 0u;
     for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(acc_full_bar(a), 1); mbar_init(acc_empty_bar(a), 8); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -114,11 +102,11 @@ linear_chain_kernel(const __grid_constant__ ChainMaps M, const __grid_constant__
       const ChainOp& op = P.op[T.g];
       if (op.dep >= 0) {
         // the rows this tile reads were written by other CTAs' TMA stores
-        if (!wait_counter(P.done + op.dep * P.m_tiles + T.m, op.dep_need)) { ok = false; break; }
+        if (!wait_counter(P.done + op.dep * P.m_tiles + T.m, op.dep_need, P.status)) { ok = false; break; }
         asm volatile("fence.proxy.async;" ::: "memory");   // order the acquire before the async-proxy reads below
       }
       for (int kb = 0; kb < op.k_blocks; ++kb) {
-        if (!mbar_wait(empty_bar(stage), phase ^ 1u)) { ok = false; break; }
+        if (!mbar_wait(empty_bar(stage), phase ^ 1u, P.status)) { ok = false; break; }
         const uint32_t a_dst = smem_base + stage * Cfg::kStage;
         const uint32_t b_dst = a_dst + Cfg::kStageA;
         mbar_arrive_expect_tx(full_bar(stage), Cfg::kStage);
@@ -127,14 +115,7 @@ linear_chain_kernel(const __grid_constant__ ChainMaps M, const __grid_constant__
         if (++stage == S) { stage = 0; phase ^= 1u; }
       }
     }
-    if (!ok) {
-      atomicExch(P.status, BSP_ERR_TIMEOUT);
-      for (int s = 0; s < S; ++s) {   // bounded chance for copies already issued to land
-        const int back = (stage - 1 - s + 2 * S) % S;
-        const uint32_t ph = (back < stage) ? phase : (phase ^ 1u);
-        (void)mbar_wait(full_bar(back), ph);
-      }
-    }
+    if (!ok) record_timeout(P.status, timed_out);
   } else if (warp == 1 && lane == 0) {
     // ---------------------------------------------------------------- MMA issuer
     constexpr uint32_t idesc = instr_desc_bf16(kBN);
@@ -145,11 +126,11 @@ linear_chain_kernel(const __grid_constant__ ChainMaps M, const __grid_constant__
     bool ok = true;
     for (int tile = blockIdx.x; tile < P.total_tiles && ok; tile += gridDim.x) {
       const int k_blocks = P.op[decode_tile(P, tile).g].k_blocks;
-      if (!mbar_wait(acc_empty_bar(acc), acc_phase[acc] ^ 1u)) { ok = false; break; }
+      if (!mbar_wait(acc_empty_bar(acc), acc_phase[acc] ^ 1u, P.status)) { ok = false; break; }
       tcgen05_fence_after();
       const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * kBN);
       for (int kb = 0; kb < k_blocks; ++kb) {
-        if (!mbar_wait(full_bar(stage), phase)) { ok = false; break; }
+        if (!mbar_wait(full_bar(stage), phase, P.status)) { ok = false; break; }
         tcgen05_fence_after();
         const uint32_t a_addr = smem_base + stage * Cfg::kStage;
         const uint32_t b_addr = a_addr + Cfg::kStageA;
@@ -165,7 +146,7 @@ linear_chain_kernel(const __grid_constant__ ChainMaps M, const __grid_constant__
       acc_phase[acc] ^= 1u;
       acc ^= 1;
     }
-    if (!ok) atomicExch(P.status, BSP_ERR_TIMEOUT);
+    if (!ok) record_timeout(P.status, timed_out);
   } else if (warp >= 2) {
     // ---------------------------------------------------------------- epilogue (two groups of four warps)
     const int group = (warp - 2) >> 2;
@@ -188,7 +169,8 @@ linear_chain_kernel(const __grid_constant__ ChainMaps M, const __grid_constant__
       for (int c = epi_tid; c < kBN; c += 256)
         s_bias[acc * kBN + c] = (op.bias != nullptr && n0 + c < op.n_out) ? __ldg(op.bias + n0 + c) : static_cast<uint16_t>(0);
       epilogue_sync_all();
-      if (!mbar_wait(acc_full_bar(acc), acc_phase[acc])) { ok = false; break; }
+      // all 256 threads take the same decision, so nobody is left alone at a named barrier below
+      if (!epilogue_all_ok(mbar_wait(acc_full_bar(acc), acc_phase[acc], P.status))) { ok = false; break; }
       tcgen05_fence_after();
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + static_cast<uint32_t>(acc * kBN);
       const int pieces = (min(kBN, op.n_out - n0) + kEpiCols - 1) / kEpiCols;
@@ -232,11 +214,12 @@ linear_chain_kernel(const __grid_constant__ ChainMaps M, const __grid_constant__
       acc_phase[acc] ^= 1u;
       acc ^= 1;
     }
-    if (!ok && lane == 0) atomicExch(P.status, BSP_ERR_TIMEOUT);
+    if (!ok && lane == 0) record_timeout(P.status, timed_out);
   }
 
   tcgen05_fence_before();
   __syncthreads();
+  quiet_period(timed_out);
   if (warp == 1) {
     tcgen05_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),

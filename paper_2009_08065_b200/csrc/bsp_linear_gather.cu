@@ -229,6 +229,7 @@ linear_gather_kernel(const __grid_constant__ CUtensorMap map_xt, const __grid_co
   // bars[0..S) full, [S..2S) empty, [2S..2S+2) accumulator full, [2S+2..2S+4) accumulator empty
   uint8_t* s_meta = reinterpret_cast<uint8_t*>(bars + 2 * S + 4);
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(s_meta + 16);
+  volatile uint32_t* timed_out = tmem_holder + 1;     // set by a role whose wait expired
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t smem_base = smem_u32(smem);
@@ -239,6 +240,7 @@ linear_gather_kernel(const __grid_constant__ CUtensorMap map_xt, const __grid_co
   auto acc_empty_bar = [&](int a) { return bar_base + 8u * (2 * S + 2 + a); };
 
   if (threadIdx.x == 0) {
+    *timed_out = 0u;
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_xt)) : "memory");
     for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(acc_full_bar(a), 1); mbar_init(acc_empty_bar(a), 4); }
@@ -289,7 +291,7 @@ linear_gather_kernel(const __grid_constant__ CUtensorMap map_xt, const __grid_co
             const long long n = n0 + (g - g_begin);
             const int stage = static_cast<int>(n % S);
             const uint32_t phase = static_cast<uint32_t>((n / S) & 1);
-            if (!mbar_wait(empty_bar(stage), phase ^ 1u)) { ok = false; }
+            if (!mbar_wait(empty_bar(stage), phase ^ 1u, P.status)) { ok = false; }
             if (ok) {
               const uint2 cv = cq[q];
               const uint32_t mt = mq[q];
@@ -327,7 +329,7 @@ linear_gather_kernel(const __grid_constant__ CUtensorMap map_xt, const __grid_co
       }
       n0 += g_end - g_begin;
     }
-    if (!ok && lane == 0) atomicExch(P.status, BSP_ERR_TIMEOUT);
+    if (!ok && lane == 0) record_timeout(P.status, timed_out);
   } else if (warp == 4) {
     // ---------------------------------------------------------------- MMA issuer
     if (lane == 0) {
@@ -342,13 +344,13 @@ linear_gather_kernel(const __grid_constant__ CUtensorMap map_xt, const __grid_co
         const int rb0 = ch * P.rb_per_chunk, rb1 = min(P.n_blocks, rb0 + P.rb_per_chunk);
         const int g_begin = __ldg(P.soff + rb0), g_end = __ldg(P.soff + rb1);
         for (int g = g_begin; g < g_end; ++g) {
-          if (!mbar_wait(full_bar(stage), phase)) { ok = false; break; }
+          if (!mbar_wait(full_bar(stage), phase, P.status)) { ok = false; break; }
           tcgen05_fence_after();
           const uint32_t mt = s_meta[stage];
           const int groups = static_cast<int>(mt & 7u);
           const bool first = (mt & 0x10u) != 0, last = (mt & 0x20u) != 0;
           if (first) {
-            if (!mbar_wait(acc_empty_bar(acc), acc_phase[acc] ^ 1u)) { ok = false; break; }
+            if (!mbar_wait(acc_empty_bar(acc), acc_phase[acc] ^ 1u, P.status)) { ok = false; break; }
             tcgen05_fence_after();
           }
           const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * D);
@@ -369,7 +371,7 @@ linear_gather_kernel(const __grid_constant__ CUtensorMap map_xt, const __grid_co
           if (++stage == S) { stage = 0; phase ^= 1u; }
         }
       }
-      if (!ok) atomicExch(P.status, BSP_ERR_TIMEOUT);
+      if (!ok) record_timeout(P.status, timed_out);
     }
   } else {
     // ---------------------------------------------------------------- epilogue
@@ -392,7 +394,7 @@ linear_gather_kernel(const __grid_constant__ CUtensorMap map_xt, const __grid_co
 #pragma unroll
           for (int j = 0; j < D / 8; ++j) bv[j] = __ldg(bp + j);
         }
-        if (!mbar_wait(acc_full_bar(acc), acc_phase[acc])) { ok = false; break; }
+        if (!mbar_wait(acc_full_bar(acc), acc_phase[acc], P.status)) { ok = false; break; }
         tcgen05_fence_after();
         const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + static_cast<uint32_t>(acc * D);
         constexpr int kPiece = 16;
@@ -428,11 +430,12 @@ linear_gather_kernel(const __grid_constant__ CUtensorMap map_xt, const __grid_co
         acc ^= 1;
       }
     }
-    if (!ok && lane == 0) atomicExch(P.status, BSP_ERR_TIMEOUT);
+    if (!ok && lane == 0) record_timeout(P.status, timed_out);
   }
 
   tcgen05_fence_before();
   __syncthreads();
+  quiet_period(timed_out);
   if (warp == 4) {
     tcgen05_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),

@@ -22,10 +22,12 @@
 //                      128 x 32 piece to a TMA store (full-line writes, tails clipped by the
 //                      tensor map).  The epilogue runs concurrently with the next tile's main
 //                      loop on the other accumulator.
-// Every wait is bounded by a wall-clock deadline; on expiry the role records BSP_ERR_TIMEOUT in
-// the status word and leaves its loop, the other roles then time out on their own waits, and
-// the CTA frees its tensor memory and exits.
+// Every wait is bounded by a wall-clock deadline (bsp_set_wait_limit_ms); on expiry the role records
+// BSP_ERR_TIMEOUT in the status word and leaves its loop, the other roles then time out on their
+// own waits (the epilogue threads by a common vote), and the CTA waits a millisecond for whatever
+// it still has in flight, frees its tensor memory and exits.
 #include <mutex>
+#include <cstring>
 
 #include "bsp_tc.cuh"
 
@@ -40,7 +42,10 @@ using namespace tc;
 
 namespace {
 
-__device__ int g_linear_status;   // 0, or BSP_ERR_TIMEOUT once a bounded wait expired
+// [0]: 0, or BSP_ERR_TIMEOUT once a bounded wait expired; [1]: a counter nothing ever bumps (self-test);
+// [2..3]: the limit of one wait in nanoseconds; [4]: waits that ran out in the last self-test;
+// [6..7]: how long its mbarrier wait lasted, nanoseconds
+__device__ __align__(16) int g_linear_status[8];
 
 
 struct LinearParams {
@@ -64,6 +69,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S * Cfg::kStage + kEpiBytes + 2 * BN * 2);
   // bars[0..S) full, [S..2S) empty, [2S..2S+2) accumulator full, [2S+2..2S+4) accumulator empty
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 2 * S + 4);
+  volatile uint32_t* timed_out = tmem_holder + 1;     // set by a role whose wait expired
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t smem_base = smem_u32(smem);
@@ -74,6 +80,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
   auto acc_empty_bar = [&](int a) { return bar_base + 8u * (2 * S + 2 + a); };
 
   if (threadIdx.x == 0) {
+    *timed_out = 0u;
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_x)) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_w)) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_y)) : "memory");
@@ -114,22 +121,14 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
       const int m0 = (tile / n_tiles) * kBlockM;
       for (int kb = 0; kb < k_blocks; ++kb) {
-        if (!mbar_wait(empty_bar(stage), phase ^ 1u)) { ok = false; break; }
+        if (!mbar_wait(empty_bar(stage), phase ^ 1u, P.status)) { ok = false; break; }
         const uint32_t a_dst = smem_base + stage * Cfg::kStage;
         mbar_arrive_expect_tx(full_bar(stage), Cfg::kStageA);
         tma_load_2d(a_dst, &map_x, kb * kBlockK, m0, full_bar(stage));
         if (++stage == S) { stage = 0; phase ^= 1u; }
       }
     }
-    if (!ok) {
-      atomicExch(P.status, BSP_ERR_TIMEOUT);
-      // copies already issued land in this CTA's shared memory: give them a bounded chance to finish
-      for (int s = 0; s < S; ++s) {
-        const int back = (stage - 1 - s + 2 * S) % S;
-        const uint32_t ph = (back < stage) ? phase : (phase ^ 1u);
-        (void)mbar_wait(full_bar(back), ph);
-      }
-    }
+    if (!ok) record_timeout(P.status, timed_out);
   } else if (warp == 10 && lane == 0) {
     // ---------------------------------------------------------------- TMA producer of the weight tiles
     int stage = 0;
@@ -138,13 +137,13 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
       const int n0 = (tile % n_tiles) * BN;
       for (int kb = 0; kb < k_blocks; ++kb) {
-        if (!mbar_wait(empty_bar(stage), phase ^ 1u)) { ok = false; break; }
+        if (!mbar_wait(empty_bar(stage), phase ^ 1u, P.status)) { ok = false; break; }
         mbar_arrive_expect_tx(full_bar(stage), Cfg::kStageB);
         tma_load_2d(smem_base + stage * Cfg::kStage + Cfg::kStageA, &map_w, kb * kBlockK, n0, full_bar(stage));
         if (++stage == S) { stage = 0; phase ^= 1u; }
       }
     }
-    if (!ok) atomicExch(P.status, BSP_ERR_TIMEOUT);
+    if (!ok) record_timeout(P.status, timed_out);
   } else if (warp == 1 && lane == 0) {
     // ---------------------------------------------------------------- MMA issuer
     constexpr uint32_t idesc = instr_desc_bf16(BN);
@@ -154,11 +153,11 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     int acc = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-      if (!mbar_wait(acc_empty_bar(acc), acc_phase[acc] ^ 1u)) { ok = false; break; }
+      if (!mbar_wait(acc_empty_bar(acc), acc_phase[acc] ^ 1u, P.status)) { ok = false; break; }
       tcgen05_fence_after();
       const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN);
       for (int kb = 0; kb < k_blocks; ++kb) {
-        if (!mbar_wait(full_bar(stage), phase)) { ok = false; break; }
+        if (!mbar_wait(full_bar(stage), phase, P.status)) { ok = false; break; }
         tcgen05_fence_after();
         const uint32_t a_addr = smem_base + stage * Cfg::kStage;
         const uint32_t b_addr = a_addr + Cfg::kStageA;
@@ -176,7 +175,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
       acc_phase[acc] ^= 1u;
       acc ^= 1;
     }
-    if (!ok) atomicExch(P.status, BSP_ERR_TIMEOUT);
+    if (!ok) record_timeout(P.status, timed_out);
   } else if (warp >= 2 && warp < 10) {
     // ---------------------------------------------------------------- epilogue
     const int group = (warp - 2) >> 2;       // 0 or 1
@@ -200,7 +199,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
       for (int c = epi_tid; c < BN; c += 256)
         s_bias[acc * BN + c] = (P.bias != nullptr && n0 + c < P.n_out) ? __ldg(P.bias + n0 + c) : static_cast<uint16_t>(0);
       epilogue_sync_all();
-      if (!mbar_wait(acc_full_bar(acc), acc_phase[acc])) { ok = false; break; }
+      // all 256 threads take the same decision, so nobody is left alone at a named barrier below
+      if (!epilogue_all_ok(mbar_wait(acc_full_bar(acc), acc_phase[acc], P.status))) { ok = false; break; }
       tcgen05_fence_after();
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + static_cast<uint32_t>(acc * BN);
       const int pieces = (min(BN, P.n_out - n0) + kEpiCols - 1) / kEpiCols;
@@ -237,15 +237,62 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
       acc ^= 1;
     }
     if (issuer) tma_store_wait_read<0>();   // shared memory must outlive the reads; the writes complete with the grid
-    if (!ok && lane == 0) atomicExch(P.status, BSP_ERR_TIMEOUT);
+    if (!ok && lane == 0) record_timeout(P.status, timed_out);
   }
 
   tcgen05_fence_before();
   __syncthreads();
+  quiet_period(timed_out);
   if (warp == 1) {
     tcgen05_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
                  "r"(static_cast<uint32_t>(Cfg::kTmemCols)) : "memory");
+  }
+}
+
+// Self-test of the bail-out path: one CTA sets up what the tensor-core kernels set up (an mbarrier,
+// tensor memory), then two of its threads wait through the same helpers on a barrier and on a
+// counter that nothing ever signals.  Both waits run out at the configured limit, the roles record
+// it, the CTA sits out the quiet period, frees its tensor memory and returns by itself.
+__global__ void __launch_bounds__(128, 1) wait_selftest_kernel(int* status) {
+  __shared__ __align__(8) uint64_t s_bar;
+  __shared__ uint32_t s_tmem[2];
+  volatile uint32_t* timed_out = s_tmem + 1;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    *timed_out = 0u;
+    status[4] = 0;
+    mbar_init(smem_u32(&s_bar), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(s_tmem)), "r"(32u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tcgen05_fence_before();
+  __syncthreads();
+  tcgen05_fence_after();
+  const uint32_t tmem_base = s_tmem[0];
+  if (warp == 0 && lane == 0) {
+    const unsigned long long t0 = global_timer_ns();
+    if (!mbar_wait(smem_u32(&s_bar), 0u, status)) {
+      record_timeout(status, timed_out);
+      atomicAdd(status + 4, 1);
+    }
+    const unsigned long long dt = global_timer_ns() - t0;
+    *reinterpret_cast<volatile unsigned long long*>(status + 6) = dt;
+  } else if (warp == 2 && lane == 0) {
+    if (!wait_counter(status + 1, 1, status)) {
+      record_timeout(status, timed_out);
+      atomicAdd(status + 4, 1);
+    }
+  }
+  tcgen05_fence_before();
+  __syncthreads();
+  quiet_period(timed_out);
+  if (warp == 1) {
+    tcgen05_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(32u) : "memory");
   }
 }
 
@@ -384,7 +431,10 @@ TcDevice* tc_device() {
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return nullptr;
     void* p = nullptr;
     if (cudaGetSymbolAddress(&p, g_linear_status) != cudaSuccess) return nullptr;
-    if (cudaMemset(p, 0, sizeof(int)) != cudaSuccess) return nullptr;
+    const unsigned long long limit = kDefaultWaitLimitNs;
+    int init[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    memcpy(&init[2], &limit, sizeof(limit));
+    if (cudaMemcpy(p, init, sizeof(init), cudaMemcpyHostToDevice) != cudaSuccess) return nullptr;
     d.status = static_cast<int*>(p);
     d.sms = sms;
   }
@@ -496,6 +546,32 @@ extern "C" int bsp_linear(const int32_t* blk_ptr, const int32_t* idx, const void
   st = bsp_linear_plan(blk_ptr, idx, vals, n_out, k_in, block, ws, ws_bytes, stream);
   if (st != BSP_OK) return st;
   return bsp_linear_planned(ws, n_out, k_in, block, X, tokens, ldx, bias, act, Y, ldy, stream);
+}
+
+extern "C" int bsp_set_wait_limit_ms(int ms) {
+  using namespace bsp;
+  if (ms < 1 || ms > 600000) return BSP_ERR_ARG;
+  TcDevice* dev = tc_device();
+  if (dev == nullptr) return BSP_ERR_CUDA;
+  const unsigned long long ns = static_cast<unsigned long long>(ms) * 1000000ull;
+  BSP_CUDA_TRY(cudaDeviceSynchronize());         // kernels in flight keep the limit they started with
+  BSP_CUDA_TRY(cudaMemcpy(dev->status + 2, &ns, sizeof(ns), cudaMemcpyHostToDevice));
+  return BSP_OK;
+}
+
+extern "C" int bsp_wait_selftest(int* expired, long long* waited_ns, void* stream) {
+  using namespace bsp;
+  TcDevice* dev = tc_device();
+  if (dev == nullptr) return BSP_ERR_CUDA;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  wait_selftest_kernel<<<1, 128, 0, s>>>(dev->status);
+  BSP_LAUNCH_CHECK();
+  int report[4] = {0, 0, 0, 0};
+  BSP_CUDA_TRY(cudaMemcpyAsync(report, dev->status + 4, sizeof(report), cudaMemcpyDeviceToHost, s));
+  BSP_CUDA_TRY(cudaStreamSynchronize(s));
+  if (expired) *expired = report[0];
+  if (waited_ns) memcpy(waited_ns, &report[2], sizeof(long long));
+  return BSP_OK;
 }
 
 extern "C" int bsp_linear_status(void* stream) {

@@ -85,6 +85,7 @@ linear_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
   // [S operand stages][2 epilogue staging buffers][bias, bf16, for two tiles][mbarriers, TMEM base]
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S * kPairStage + kEpiBytes + 2 * kPairBN * 2);
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 2 * S + 4);
+  volatile uint32_t* timed_out = tmem_holder + 1;     // set by a role of this CTA whose wait expired
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();          // 0 = leader of the pair
@@ -97,6 +98,7 @@ linear_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
   auto acc_empty_bar = [&](int a) { return bar_base + 8u * (2 * S + 2 + a); };   // used in the leader only
 
   if (threadIdx.x == 0) {
+    *timed_out = 0u;
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_x)) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_w)) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_y)) : "memory");
@@ -133,7 +135,7 @@ linear_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
       const int m0 = (tile / n_tiles) * 256 + static_cast<int>(rank) * kBlockM;
       const int w0 = (tile % n_tiles) * kPairBN + static_cast<int>(rank) * (kPairBN / 2);
       for (int kb = 0; kb < k_blocks; ++kb) {
-        if (!mbar_wait(empty_bar(stage), phase ^ 1u)) { ok = false; break; }
+        if (!mbar_wait(empty_bar(stage), phase ^ 1u, P.status)) { ok = false; break; }
         const uint32_t a_dst = smem_base + stage * kPairStage;
         const uint32_t b_dst = a_dst + kPairStageA;
         const uint32_t leader_full = map_to_cta(full_bar(stage), 0);
@@ -143,7 +145,7 @@ linear_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
         if (++stage == S) { stage = 0; phase ^= 1u; }
       }
     }
-    if (!ok) atomicExch(P.status, BSP_ERR_TIMEOUT);
+    if (!ok) record_timeout(P.status, timed_out);
   } else if (warp == 1 && lane == 0 && rank == 0) {
     // ---------------------------------------------------------------- MMA issuer (leader CTA only)
     int stage = 0;
@@ -152,11 +154,11 @@ linear_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
     int acc = 0;
     bool ok = true;
     for (int tile = pair; tile < total_tiles && ok; tile += n_pairs) {
-      if (!mbar_wait(acc_empty_bar(acc), acc_phase[acc] ^ 1u)) { ok = false; break; }
+      if (!mbar_wait(acc_empty_bar(acc), acc_phase[acc] ^ 1u, P.status)) { ok = false; break; }
       tcgen05_fence_after();
       const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * kPairBN);
       for (int kb = 0; kb < k_blocks; ++kb) {
-        if (!mbar_wait(full_bar(stage), phase)) { ok = false; break; }
+        if (!mbar_wait(full_bar(stage), phase, P.status)) { ok = false; break; }
         tcgen05_fence_after();
         const uint32_t a_addr = smem_base + stage * kPairStage;
         const uint32_t b_addr = a_addr + kPairStageA;
@@ -175,7 +177,7 @@ linear_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
       acc_phase[acc] ^= 1u;
       acc ^= 1;
     }
-    if (!ok) atomicExch(P.status, BSP_ERR_TIMEOUT);
+    if (!ok) record_timeout(P.status, timed_out);
   } else if (warp >= 2) {
     // ---------------------------------------------------------------- epilogue of this CTA's 128 rows
     const int group = (warp - 2) >> 2;
@@ -196,7 +198,8 @@ linear_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
       for (int c = epi_tid; c < kPairBN; c += 256)
         s_bias[acc * kPairBN + c] = (P.bias != nullptr && n0 + c < P.n_out) ? __ldg(P.bias + n0 + c) : static_cast<uint16_t>(0);
       epilogue_sync_all();
-      if (!mbar_wait(acc_full_bar(acc), acc_phase[acc])) { ok = false; break; }
+      // all 256 threads take the same decision, so nobody is left alone at a named barrier below
+      if (!epilogue_all_ok(mbar_wait(acc_full_bar(acc), acc_phase[acc], P.status))) { ok = false; break; }
       tcgen05_fence_after();
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + static_cast<uint32_t>(acc * kPairBN);
       const uint32_t leader_acc_empty = map_to_cta(acc_empty_bar(acc), 0);
@@ -234,11 +237,12 @@ linear_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
       acc ^= 1;
     }
     if (issuer) tma_store_wait_read<0>();
-    if (!ok && lane == 0) atomicExch(P.status, BSP_ERR_TIMEOUT);
+    if (!ok && lane == 0) record_timeout(P.status, timed_out);
   }
 
   tcgen05_fence_before();
   __syncthreads();
+  quiet_period(timed_out);
   cluster_sync_all();          // neither CTA leaves while the other may still touch its memory or barriers
   if (warp == 1) {
     tcgen05_fence_after();

@@ -21,7 +21,8 @@ constexpr int kEpiCols = 32;                    // columns per epilogue piece = 
 constexpr int kEpiStage = kBlockM * kEpiCols * 2;     // one staging buffer: 128 rows x 64 bytes
 constexpr int kEpiBuffers = 4;                  // two per epilogue group, so a store can drain while the next piece is staged
 constexpr int kEpiBytes = kEpiBuffers * kEpiStage;
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s per wait
+constexpr unsigned long long kDefaultWaitLimitNs = 2000000000ull;  // 2 s per wait unless bsp_set_wait_limit_ms says otherwise
+constexpr unsigned long long kQuietNs = 1000000ull;         // 1 ms for operations in flight after a wait gave up
 
 
 // Shared-memory plan of a CTA for an output tile 128 x BN: operand stages, two epilogue staging
@@ -69,16 +70,55 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+// The status area of a device is four 32-bit words: [0] the status code that kernels set when a
+// bounded wait expires, [1] unused, [2..3] the limit of one wait in nanoseconds (64 bits).
+__device__ __forceinline__ unsigned long long wait_limit_ns(const int* status) {
+  return *reinterpret_cast<const volatile unsigned long long*>(status + 2);
+}
 // Bounded wait: false when the deadline passed (the caller records the failure and bails out).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+// The limit is read only once the first probe has failed.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const int* status) {
   if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long limit = wait_limit_ns(status);
   const unsigned long long start = global_timer_ns();
   for (;;) {
 #pragma unroll 1
     for (int i = 0; i < 256; ++i)
       if (mbar_try_wait(bar, parity)) return true;
-    if (global_timer_ns() - start > kWaitLimitNs) return false;
+    if (global_timer_ns() - start > limit) return false;
   }
+}
+// Bounded wait until *counter >= need (acquire at GPU scope): a counter in global memory that
+// other CTAs of the same launch bump.
+__device__ __forceinline__ bool wait_counter(const int* counter, int need, const int* status) {
+  const unsigned long long limit = wait_limit_ns(status);
+  const unsigned long long start = global_timer_ns();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 64; ++i) {
+      int v;
+      asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(counter) : "memory");
+      if (v >= need) return true;
+    }
+    if (global_timer_ns() - start > limit) return false;
+  }
+}
+// A role whose wait expired: the device-wide status word for the host, and this CTA's own flag so that
+// the CTA holds on to its shared and tensor memory for a while before it exits (see quiet_period).
+__device__ __forceinline__ void record_timeout(int* status, volatile uint32_t* cta_flag) {
+  atomicExch(status, BSP_ERR_TIMEOUT);
+  *cta_flag = 1u;
+}
+// After a wait gave up, copies and tensor-core operations that were already issued may still be
+// writing this CTA's shared or tensor memory; they complete within microseconds once their data
+// arrives.  The CTA waits a fixed millisecond before it gives that memory back.  Call after the
+// block-wide barrier that follows the role loops; every thread takes part.
+__device__ __forceinline__ void quiet_period(const volatile uint32_t* cta_flag) {
+  if (*cta_flag != 0u) {
+    const unsigned long long start = global_timer_ns();
+    while (global_timer_ns() - start < kQuietNs) __nanosleep(2000);
+  }
+  __syncthreads();
 }
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
   asm volatile(
@@ -127,6 +167,20 @@ __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.a
 // epilogue group g, 3 among all 256 epilogue threads.
 __device__ __forceinline__ void group_sync(int g) { asm volatile("bar.sync %0, 128;" ::"r"(1 + g) : "memory"); }
 __device__ __forceinline__ void epilogue_sync_all() { asm volatile("bar.sync 3, 256;" ::: "memory"); }
+// The 256 epilogue threads agree on whether all of their waits succeeded (named barrier 4 with an AND
+// reduction): either every one of them goes on to the named barriers of the tile, or none does.
+__device__ __forceinline__ bool epilogue_all_ok(bool ok) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.b32 p, %1, 0;\n\t"
+      "barrier.cta.red.and.pred q, 4, 256, p;\n\t"
+      "selp.u32 %0, 1, 0, q;\n\t}"
+      : "=r"(r)
+      : "r"(ok ? 1u : 0u)
+      : "memory");
+  return r != 0u;
+}
 // Shared-memory accesses of the epilogue as volatile asm WITHOUT a memory clobber: they keep their
 // order among themselves and with the fences and barriers around them (all volatile asm), but do
 // not stop the compiler from hoisting the bias loads of a whole piece ahead of its stores.

@@ -24,3 +24,20 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(autouse=True)
+def guard_words(request):
+    """GPU tests run with guard zones around every CUDA tensor they (or the binding) allocate; the zones are
+    checked when the test ends.  compute-sanitizer's stand-in: a kernel that writes past an output fails here."""
+    if "gpu" not in request.keywords:
+        yield
+        return
+    import torch
+    if not torch.cuda.is_available():
+        yield
+        return
+    from gpu_util import GuardedAllocations
+    with GuardedAllocations() as guards:
+        yield
+        guards.check()

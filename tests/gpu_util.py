@@ -6,6 +6,96 @@ import paper_2009_08065_b200 as bsp
 
 DEV = "cuda"
 
+GUARD_BYTES = 256
+GUARD_PATTERN = 0xA5
+
+
+class GuardedAllocations:
+    """Stand-in for a memory checker: while active, every CUDA tensor made through torch's factory functions
+    (torch.empty / zeros / ones / full / *_like, called by a test or by the binding's allocate helpers) is a view
+    into a larger byte buffer with GUARD_BYTES of a known pattern before and after it.  `check()` asserts that
+    no kernel wrote outside the tensors it was given.  The payload stays 256-byte aligned."""
+
+    FACTORIES = ("empty", "zeros", "ones", "full")
+
+    def __init__(self):
+        self.live = []          # (raw byte buffer, payload bytes, description)
+        self._saved = {}
+
+    def _is_cuda(self, device):
+        return device is not None and torch.device(device).type == "cuda"
+
+    def _guarded(self, shape, dtype, device, what):
+        dtype = dtype or torch.get_default_dtype()
+        if isinstance(shape, int):
+            shape = (shape,)
+        shape = tuple(int(v) for v in shape)
+        itemsize = torch.empty((), dtype=dtype).element_size()
+        n = itemsize
+        for v in shape:
+            n *= v
+        padded = (n + 255) // 256 * 256
+        raw = self._saved["empty"](GUARD_BYTES + padded + GUARD_BYTES, dtype=torch.uint8, device=device)
+        raw[:GUARD_BYTES] = GUARD_PATTERN
+        raw[GUARD_BYTES + n:] = GUARD_PATTERN
+        self.live.append((raw, n, f"{what}{shape} {dtype}"))
+        return raw[GUARD_BYTES:GUARD_BYTES + n].view(dtype).view(shape)
+
+    def __enter__(self):
+        alloc = self
+
+        def wrap(name, orig):
+            def factory(*size, **kw):
+                if not alloc._is_cuda(kw.get("device")) or kw.get("pin_memory") or kw.get("out") is not None:
+                    return orig(*size, **kw)
+                args = list(size)
+                fill = args.pop() if name == "full" else None
+                shape = args[0] if len(args) == 1 and not isinstance(args[0], int) else tuple(args)
+                t = alloc._guarded(shape, kw.get("dtype"), kw["device"], name)
+                if name == "zeros":
+                    t.zero_()
+                elif name == "ones":
+                    t.fill_(1)
+                elif name == "full":
+                    t.fill_(fill)
+                return t
+            return factory
+
+        def wrap_like(name, orig):
+            def like(t, **kw):
+                device = kw.get("device", t.device)
+                if not alloc._is_cuda(device) or kw.get("pin_memory"):
+                    return orig(t, **kw)
+                out = alloc._guarded(tuple(t.shape), kw.get("dtype", t.dtype), device, name)
+                if name == "zeros_like":
+                    out.zero_()
+                return out
+            return like
+
+        for name in self.FACTORIES:
+            self._saved[name] = getattr(torch, name)
+        for name in ("empty_like", "zeros_like"):
+            self._saved[name] = getattr(torch, name)
+        for name in self.FACTORIES:
+            setattr(torch, name, wrap(name, self._saved[name]))
+        for name in ("empty_like", "zeros_like"):
+            setattr(torch, name, wrap_like(name, self._saved[name]))
+        return self
+
+    def __exit__(self, *exc):
+        for name, fn in self._saved.items():
+            setattr(torch, name, fn)
+
+    def check(self):
+        if torch.cuda.is_available():
+            torch.cuda.synchronize()
+        for raw, n, what in self.live:
+            head = raw[:GUARD_BYTES]
+            tail = raw[GUARD_BYTES + n:]
+            assert bool((head == GUARD_PATTERN).all()), f"bytes before {what} were overwritten"
+            assert bool((tail == GUARD_PATTERN).all()), f"bytes after {what} were overwritten"
+        return len(self.live)
+
 
 def to_dev(bits: np.ndarray) -> torch.Tensor:
     """uint16 bf16 bit patterns -> int16 CUDA tensor holding the same bits."""
