@@ -148,7 +148,7 @@ class LayerOnDevice:
                 "gamma": torch.empty((n_blocks, spec.k_in), dtype=torch.float32, device=device),
                 "penalty": torch.zeros(1, dtype=torch.float64, device=device),
                 "pk": bsp.PackedMatrix.allocate(spec.n_out, spec.k_in, spec.block, bsp.ORIENT_C, device),
-                "plan": torch.empty(bsp.bsp_linear_plan_bytes(spec.n_out, spec.k_in, spec.block), dtype=torch.uint8, device=device),
+                "plan": view(*parts[1 + 2 * i]),      # in-place mode: W, masked where it is pruned, is its own execution layout
                 "Y": torch.empty((wl.tokens, spec.n_out), dtype=torch.int16, device=device),
             }
             self.lin.append(e)

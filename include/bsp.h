@@ -244,6 +244,13 @@ int bsp_repack_values(const void* W, int rows, int cols, int ldw, int block,
  * for bit; the penalty is summed in a fixed order here and is reproducible run to run.
  * The kernel's bounded waits report through bsp_linear_status (BSP_ERR_TIMEOUT).
  *
+ * In-place mode: a job whose `plan` pointer equals its `W` pointer gets no separate execution
+ * layout.  Instead the weights of the pruned groups are overwritten with +0 inside W (Algorithm
+ * 2's W = W * Mask) and nothing else of W is written; W, which must then be writable, is
+ * afterwards its own execution layout (pass it to bsp_linear_planned as `plan`; that call wants
+ * ldw == cols).  When W already holds zeros in every pruned group (threshold 0 on a pruned
+ * matrix) this writes nothing at all.
+ *
  * jobs: HOST array of n_jobs descriptors; the pointers inside are device pointers with the
  * meaning they have in the single-matrix calls.  norms, gamma_in, gamma_out, penalty, keep,
  * kept_weights, plan may be NULL (that output is skipped).  ws/ws_bytes as bsp_prune_pack.

@@ -225,7 +225,9 @@ fused_stage2_kernel(const __grid_constant__ Batch B) {
     for (int rr = warp; rr < n_rows; rr += n_warps) {
       const uint16_t* src = wblk + static_cast<size_t>(r_lo + rr) * J.ldw;
       uint16_t* dst = s_w + rr * J.cols;
-      uint16_t* pdst = J.plan ? J.plan + (static_cast<size_t>(b) * d + r_lo + rr) * J.cols : nullptr;
+      // (a plan that IS W: in-place mode, only pieces that change are written)
+      const bool in_place = J.plan == J.W;
+      uint16_t* pdst = J.plan ? J.plan + (static_cast<size_t>(b) * d + r_lo + rr) * (in_place ? J.ldw : J.cols) : nullptr;
       for (int q0 = lane; q0 < chunks; q0 += 128) {
         uint4 w[4];
 #pragma unroll
@@ -243,7 +245,8 @@ fused_stage2_kernel(const __grid_constant__ Batch B) {
             m.y = w[u].y & ((((f.x >> 16) & 0xffu) * 0xffffu) | (((f.x >> 24) & 0xffu) * 0xffff0000u));
             m.z = w[u].z & (((f.y & 0xffu) * 0xffffu) | (((f.y >> 8) & 0xffu) * 0xffff0000u));
             m.w = w[u].w & ((((f.y >> 16) & 0xffu) * 0xffffu) | (((f.y >> 24) & 0xffu) * 0xffff0000u));
-            *reinterpret_cast<uint4*>(pdst + (q << 3)) = m;
+            if (!in_place || ((m.x ^ w[u].x) | (m.y ^ w[u].y) | (m.z ^ w[u].z) | (m.w ^ w[u].w)) != 0u)
+              *reinterpret_cast<uint4*>(pdst + (q << 3)) = m;
           }
         }
       }
@@ -356,7 +359,7 @@ extern "C" int bsp_prepare_batched(const bsp_layer_job* jobs, int n_jobs, int bl
     if (!aligned_to(u.ws, 256) || !aligned_to(u.blk_ptr, 4) || !aligned_to(u.idx, 4) || !aligned_to(u.vals, 2)) return BSP_ERR_ARG;
     if (u.threshold != u.threshold) return BSP_ERR_ARG;
     if (u.ws_bytes < ws_layout(u.rows / block, u.cols).total) return BSP_ERR_WORKSPACE;
-    if (u.plan != nullptr) {
+    if (u.plan != nullptr && u.plan != u.W) {          // plan == W: in-place mode, W itself becomes the layout
       if (!aligned_to(u.plan, 256)) return BSP_ERR_ARG;
       if (u.plan_bytes < static_cast<size_t>(u.rows) * u.cols * 2) return BSP_ERR_WORKSPACE;
     }

@@ -273,10 +273,14 @@ fused_stream_kernel(const __grid_constant__ StreamBatch B) {
         if (bit) s_idx[p++] = static_cast<uint16_t>((k << 3) + i);
       }
     }
-    // execution layout: the rows with the pruned columns zeroed, one warp per row, 16-byte stores
+    // execution layout: the rows with the pruned columns zeroed, one warp per row, 16-byte stores.
+    // When the job's plan IS its W (in-place mode, Algorithm 2's W = W * Mask), only 8-column pieces
+    // that hold a weight of a pruned group are written: W read once, and written only where it changes.
     if (J.plan != nullptr) {
+      const bool in_place = J.plan == J.W;
+      const size_t pld = in_place ? static_cast<size_t>(J.ldw) : static_cast<size_t>(J.cols);
       for (int r = warp; r < d; r += n_warps) {
-        uint16_t* pdst = J.plan + (static_cast<size_t>(b) * d + r) * J.cols + c0;
+        uint16_t* pdst = J.plan + (static_cast<size_t>(b) * d + r) * pld + c0;
         for (int k = lane; k < chunks; k += 32) {
           const uint4 w = *reinterpret_cast<const uint4*>(s_w + r * pc + (k << 3));
           const uint2 f = *reinterpret_cast<const uint2*>(s_flag + (k << 3));
@@ -285,7 +289,8 @@ fused_stream_kernel(const __grid_constant__ StreamBatch B) {
           m.y = w.y & ((((f.x >> 16) & 0xffu) * 0xffffu) | (((f.x >> 24) & 0xffu) * 0xffff0000u));
           m.z = w.z & (((f.y & 0xffu) * 0xffffu) | (((f.y >> 8) & 0xffu) * 0xffff0000u));
           m.w = w.w & ((((f.y >> 16) & 0xffu) * 0xffffu) | (((f.y >> 24) & 0xffu) * 0xffff0000u));
-          *reinterpret_cast<uint4*>(pdst + (k << 3)) = m;
+          if (!in_place || ((m.x ^ w.x) | (m.y ^ w.y) | (m.z ^ w.z) | (m.w ^ w.w)) != 0u)
+            *reinterpret_cast<uint4*>(pdst + (k << 3)) = m;
         }
       }
     }

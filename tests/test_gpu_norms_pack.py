@@ -10,7 +10,7 @@ import torch
 import paper_2009_08065_b200 as bsp
 import synth_inputs as si
 from oracle import bsp_oracle as O
-from gpu_util import DEV, bits_of, packed_to_host, to_dev
+from gpu_util import DEV, assert_linear_close, bits_of, packed_to_host, to_dev
 
 pytestmark = pytest.mark.gpu
 REL = 1e-5
@@ -301,6 +301,44 @@ def test_prepare_batched_streaming_batch_larger_than_the_gpu():
             assert np.array_equal(plan, O.prune(w, block, "C", t_b))
             job.out.idx.fill_(-7)
             job.penalty.fill_(-5.0)
+
+
+def test_prepare_batched_in_place_masks_w_and_writes_nothing_else():
+    """A job whose plan is its W: the pruned groups are zeroed inside W (Algorithm 2's W = W * Mask), every other
+    output is what the separate-plan call gives, a second call on the now-masked W with threshold 0 leaves W
+    as it is, and the masked W runs through the linear layer as its own execution layout."""
+    eps = 1e-3
+    # the last case is beyond the one-pass kernel (32 column ranges per row-block) and takes the two-stage path
+    for rows, cols, block in [(768, 768, 16), (768, 3072, 16), (3072, 768, 16), (192, 4096, 96)]:
+        w = si.student_t_bf16(610 + rows + cols, f"inplace{rows}x{cols}", (rows, cols), 3.0, 0.02)
+        t_b = float(np.quantile(O.group_norms(w, block, "C"), 0.6))
+        W = to_dev(w)
+        pk = bsp.PackedMatrix.allocate(rows, cols, block, bsp.ORIENT_C, DEV)
+        pen = torch.zeros(1, dtype=torch.float64, device=DEV)
+        bsp.bsp_prepare_batched([bsp.LayerJob(W=W, out=pk, threshold=t_b, penalty=pen, plan=W)], block, eps, bsp.PEN_L2)
+        bsp.bsp_linear_status()
+        keep_ref = O.keep_flags(w, block, "C", t_b)
+        w_masked = O.prune(w, block, "C", t_b)
+        assert np.array_equal(bits_of(W), w_masked)
+        ref_ptr, ref_idx, ref_vals = O.pack(w, keep_ref, block, "C")
+        blk_ptr, idx, vals, keep, kept = packed_to_host(pk)
+        assert np.array_equal(keep, keep_ref) and np.array_equal(blk_ptr, ref_ptr)
+        assert np.array_equal(idx, ref_idx) and np.array_equal(vals, ref_vals)
+        n_ref = O.group_norms(w, block, "C")
+        assert float(pen.item()) == pytest.approx(O.penalty_l2(n_ref, O.gamma_update(n_ref, eps)), rel=REL)
+        # second pass, threshold 0 on the masked matrix: same kept sets, W untouched
+        pk2 = bsp.PackedMatrix.allocate(rows, cols, block, bsp.ORIENT_C, DEV)
+        bsp.bsp_prepare_batched([bsp.LayerJob(W=W, out=pk2, threshold=0.0, plan=W)], block, eps, bsp.PEN_L2)
+        bsp.bsp_linear_status()
+        assert np.array_equal(bits_of(W), w_masked)
+        assert torch.equal(pk2.blk_ptr, pk.blk_ptr) and torch.equal(pk2.keep, pk.keep)
+        # W is now its own execution layout
+        x = si.normal_bf16(3, "inplace_x", (200, cols), 1.0)
+        y = torch.full((200, rows), 0x7FC0, dtype=torch.int16, device=DEV)
+        bsp.bsp_linear_planned(W, rows, cols, block, to_dev(x), None, bsp.ACT_NONE, y)
+        bsp.bsp_linear_status()
+        mask = O.mask_of(w_masked)
+        assert_linear_close(bits_of(y), O.linear_masked_dense(x, w_masked, mask, None, 0), O.row_scales(x, w_masked, mask, None))
 
 
 @pytest.mark.parametrize("block", [3, 12, 96])
