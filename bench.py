@@ -152,7 +152,7 @@ class LayerOnDevice:
                 "Y": torch.empty((wl.tokens, spec.n_out), dtype=torch.int16, device=device),
             }
             self.lin.append(e)
-        self.kernels_per_step = 2 + len(self.lin)   # two weight-side launches for the batch, one GEMM per matrix
+        self.kernels_per_step = 1 + len(self.lin)   # one weight-side launch for the batch, one GEMM per matrix
 
     def source(self, spec, outs):
         if spec.src == "x":

@@ -25,6 +25,8 @@
 // lowest mantissa bit of the float64 partial), read with relaxed loads: a reader needs nothing but
 // the word itself, so no fence is involved.  The last item of a matrix adds the partials in a fixed
 // order.  Masks, indices, tiles, norms and gamma are bit-identical to the two-stage path.
+#include <cstddef>
+#include <cstring>
 #include <new>
 
 #include "bsp_tc.cuh"
@@ -49,19 +51,26 @@ struct StreamJob {
   int32_t* part_counts;      // [n_blocks * parts] published counts, then (job 0) the ticket
   unsigned long long* part_partial;   // [n_blocks * parts] published penalty partials (float64 bits, lowest bit set)
 };
-struct StreamBatch {
+template <int N>
+struct StreamBatchT {
   int n_jobs, block, squared;
   float eps;
   int total_items, buf_bytes;
   int* ticket;
   int* status;               // receives BSP_ERR_TIMEOUT when a bounded wait expires
-  StreamJob job[kStreamMaxJobs];
+  StreamJob job[N];
 };
+// The job table travels as a kernel parameter: 14 KB for a full batch, which every launch has to
+// move; a batch of up to eight matrices (an encoder layer's) gets a table of 1.2 KB.  Both have the
+// same fields in the same order, so the small one is a copy of the large one's beginning.
+constexpr int kStreamFewJobs = 8;
+using StreamBatch = StreamBatchT<kStreamMaxJobs>;
 
 struct Item {
   int jn, local, b, q, c0, pc;
 };
-__device__ __forceinline__ Item locate(const StreamBatch& B, int item) {
+template <class Batch>
+__device__ __forceinline__ Item locate(const Batch& B, int item) {
   int lo = 0, hi = B.n_jobs - 1;
   while (lo < hi) {
     const int mid = (lo + hi + 1) >> 1;
@@ -79,8 +88,8 @@ __device__ __forceinline__ Item locate(const StreamBatch& B, int item) {
 }
 
 // Rows of an item into a shared-memory buffer, one bulk copy per row (called by one warp).
-__device__ __forceinline__ void issue_rows(const StreamBatch& B, int item, uint32_t dst, uint32_t bar, int lane) {
-  const Item I = locate(B, item);
+template <class Batch>
+__device__ __forceinline__ void issue_rows(const Batch& B, const Item& I, uint32_t dst, uint32_t bar, int lane) {
   const FusedJob& J = B.job[I.jn].j;
   const int d = B.block;
   const uint32_t row_bytes = static_cast<uint32_t>(I.pc) * 2u;
@@ -131,8 +140,9 @@ __device__ __forceinline__ double wait_partial(const unsigned long long* slot, i
   }
 }
 
+template <int N>
 __global__ void __launch_bounds__(kStreamThreads, 8)
-fused_stream_kernel(const __grid_constant__ StreamBatch B) {
+fused_stream_kernel(const __grid_constant__ StreamBatchT<N> B) {
   extern __shared__ __align__(128) uint8_t s_raw[];
   __shared__ __align__(8) uint64_t s_bar;
   __shared__ int s_item;
@@ -146,6 +156,16 @@ fused_stream_kernel(const __grid_constant__ StreamBatch B) {
   uint16_t* s_idx = reinterpret_cast<uint16_t*>(s_raw + static_cast<size_t>(B.buf_bytes));    // [max part columns], local column numbers
   const uint32_t bar = smem_u32(&s_bar);
 
+  // A batch that fits the GPU in one wave needs no ticket: every CTA is resident, item = block index,
+  // and the item's job is looked up (which brings its part of the kernel parameters into the constant
+  // cache) while the clearing kernel is still running.
+  const bool direct = B.ticket == nullptr;
+  int item = static_cast<int>(blockIdx.x);
+  Item I = locate(B, direct ? item : 0);
+  if (direct) {
+    const FusedJob& J0 = B.job[I.jn].j;
+    asm volatile("" ::"l"(J0.W), "r"(J0.ldw), "l"(J0.flags), "l"(J0.vals), "l"(B.job[I.jn].part_counts));
+  }
   if (threadIdx.x == 0) {
     mbar_init(bar, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -153,14 +173,16 @@ fused_stream_kernel(const __grid_constant__ StreamBatch B) {
     // launched with programmatic stream serialization: everything above overlapped the clearing
     // kernel; the ticket and the slots it zeroes are touched only from here on
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    s_item = atomicAdd(B.ticket, 1);
+    if (!direct) s_item = atomicAdd(B.ticket, 1);
   }
   __syncthreads();
-  const int item = s_item;
-  if (item >= B.total_items) return;
-  if (warp == 0) issue_rows(B, item, smem_u32(s_raw), bar, lane);
+  if (!direct) {
+    item = s_item;
+    if (item >= B.total_items) return;
+    I = locate(B, item);
+  }
+  if (warp == 0) issue_rows(B, I, smem_u32(s_raw), bar, lane);
   {
-    const Item I = locate(B, item);
     const StreamJob& O = B.job[I.jn];
     const FusedJob& J = O.j;
     const int b = I.b, q = I.q, c0 = I.c0, pc = I.pc, local = I.local;
@@ -184,10 +206,13 @@ fused_stream_kernel(const __grid_constant__ StreamBatch B) {
     const float t2 = __fmul_rn(t, t);
     int count = 0;
     float pen = 0.0f;
+    const bool in_place = J.plan != nullptr && J.plan == J.W;
+    int changes = 0;                         // in-place mode: a pruned group that still holds a non-zero weight
     for (int k = threadIdx.x; k < chunks; k += blockDim.x) {
       float acc[8];
 #pragma unroll
       for (int i = 0; i < 8; ++i) acc[i] = 0.0f;
+#pragma unroll 4
       for (int r = 0; r < d; ++r) {
         const uint4 v = *reinterpret_cast<const uint4*>(s_w + r * pc + (k << 3));
         const uint32_t w32[4] = {v.x, v.y, v.z, v.w};
@@ -206,6 +231,7 @@ fused_stream_kernel(const __grid_constant__ StreamBatch B) {
         lo |= k0 << (8 * i);
         hi |= k1 << (8 * i);
         count += static_cast<int>(k0 + k1);
+        changes |= static_cast<int>((k0 == 0u && acc[i] != 0.0f) || (k1 == 0u && acc[4 + i] != 0.0f));
       }
       const size_t g0 = static_cast<size_t>(b) * J.cols + c0 + (k << 3);
       *reinterpret_cast<uint2*>(s_flag + (k << 3)) = make_uint2(lo, hi);
@@ -243,7 +269,7 @@ fused_stream_kernel(const __grid_constant__ StreamBatch B) {
     count = warp_sum(count);
     double pd = warp_sum(static_cast<double>(pen));
     if (lane == 0) { s_cnt[warp] = count; s_pen[warp] = pd; }
-    __syncthreads();
+    const bool rewrite = __syncthreads_or(changes) != 0;     // (the block-wide barrier of this point)
     const int n_parts = J.n_blocks * O.parts;
     if (threadIdx.x == 0) {
       int c = 0;
@@ -275,9 +301,9 @@ fused_stream_kernel(const __grid_constant__ StreamBatch B) {
     }
     // execution layout: the rows with the pruned columns zeroed, one warp per row, 16-byte stores.
     // When the job's plan IS its W (in-place mode, Algorithm 2's W = W * Mask), only 8-column pieces
-    // that hold a weight of a pruned group are written: W read once, and written only where it changes.
-    if (J.plan != nullptr) {
-      const bool in_place = J.plan == J.W;
+    // that hold a weight of a pruned group are written: W read once, and written only where it changes
+    // (an item whose pruned groups are all zero already skips the pass).
+    if (J.plan != nullptr && (!in_place || rewrite)) {
       const size_t pld = in_place ? static_cast<size_t>(J.ldw) : static_cast<size_t>(J.cols);
       for (int r = warp; r < d; r += n_warps) {
         uint16_t* pdst = J.plan + (static_cast<size_t>(b) * d + r) * pld + c0;
@@ -347,30 +373,63 @@ fused_stream_kernel(const __grid_constant__ StreamBatch B) {
       // vectors where the destination is aligned, ragged ends by element.
       const bool vec_ok = (reinterpret_cast<uintptr_t>(J.vals) & 15) == 0;
       const long long tile0 = static_cast<long long>(d) * block_base;
-      for (int r = warp; r < d; r += n_warps) {
-        const uint16_t* srow = s_w + r * pc;
-        const long long e0 = tile0 + static_cast<long long>(r) * kc_block + off_in_block;
-        uint16_t* out_row = J.vals + e0;
-        if (vec_ok) {
-          const int head = static_cast<int>((8 - (e0 & 7)) & 7);
-          const int n_vec = kc > head ? (kc - head) >> 3 : 0;
-          for (int v = lane; v < n_vec; v += 32) {
-            const int p = head + (v << 3);
+      if (vec_ok && (kc_block & 7) == 0 && (tile0 & 7) == 0) {
+        // every row of the tile starts at the same offset from a 16-byte boundary: a lane keeps the
+        // eight column numbers of its vector in registers and walks the rows of its warp with them
+        const int head = (8 - (off_in_block & 7)) & 7;
+        const int n_vec = kc > head ? (kc - head) >> 3 : 0;
+        for (int v = lane; v < n_vec; v += 32) {
+          const int p = head + (v << 3);
+          int col[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) col[i] = s_idx[p + i];
+          for (int r = warp; r < d; r += n_warps) {
+            const uint16_t* srow = s_w + r * pc;
             uint32_t o[4];
 #pragma unroll
             for (int i = 0; i < 4; ++i)
-              o[i] = static_cast<uint32_t>(srow[s_idx[p + 2 * i]]) | (static_cast<uint32_t>(srow[s_idx[p + 2 * i + 1]]) << 16);
-            *reinterpret_cast<uint4*>(out_row + p) = make_uint4(o[0], o[1], o[2], o[3]);
+              o[i] = static_cast<uint32_t>(srow[col[2 * i]]) | (static_cast<uint32_t>(srow[col[2 * i + 1]]) << 16);
+            *reinterpret_cast<uint4*>(J.vals + tile0 + static_cast<long long>(r) * kc_block + off_in_block + p) =
+                make_uint4(o[0], o[1], o[2], o[3]);
           }
-          const int tail0 = head + (n_vec << 3);
+        }
+        const int tail0 = head + (n_vec << 3);
+        for (int r = warp; r < d; r += n_warps) {      // ragged ends of each row by element
+          const uint16_t* srow = s_w + r * pc;
+          uint16_t* out_row = J.vals + tile0 + static_cast<long long>(r) * kc_block + off_in_block;
           if (lane < 8) {
             if (lane < head && lane < kc) out_row[lane] = srow[s_idx[lane]];
           } else if (lane < 16) {
             const int p = tail0 + (lane - 8);
             if (p >= head && p < kc) out_row[p] = srow[s_idx[p]];
           }
-        } else {
-          for (int p = lane; p < kc; p += 32) out_row[p] = srow[s_idx[p]];
+        }
+      } else {
+        for (int r = warp; r < d; r += n_warps) {
+          const uint16_t* srow = s_w + r * pc;
+          const long long e0 = tile0 + static_cast<long long>(r) * kc_block + off_in_block;
+          uint16_t* out_row = J.vals + e0;
+          if (vec_ok) {
+            const int head = static_cast<int>((8 - (e0 & 7)) & 7);
+            const int n_vec = kc > head ? (kc - head) >> 3 : 0;
+            for (int v = lane; v < n_vec; v += 32) {
+              const int p = head + (v << 3);
+              uint32_t o[4];
+#pragma unroll
+              for (int i = 0; i < 4; ++i)
+                o[i] = static_cast<uint32_t>(srow[s_idx[p + 2 * i]]) | (static_cast<uint32_t>(srow[s_idx[p + 2 * i + 1]]) << 16);
+              *reinterpret_cast<uint4*>(out_row + p) = make_uint4(o[0], o[1], o[2], o[3]);
+            }
+            const int tail0 = head + (n_vec << 3);
+            if (lane < 8) {
+              if (lane < head && lane < kc) out_row[lane] = srow[s_idx[lane]];
+            } else if (lane < 16) {
+              const int p = tail0 + (lane - 8);
+              if (p >= head && p < kc) out_row[p] = srow[s_idx[p]];
+            }
+          } else {
+            for (int p = lane; p < kc; p += 32) out_row[p] = srow[s_idx[p]];
+          }
         }
       }
     }
@@ -378,8 +437,9 @@ fused_stream_kernel(const __grid_constant__ StreamBatch B) {
 }
 
 // Zeroes the published counts and partials and the ticket slot of every matrix.
+template <int N>
 __global__ void __launch_bounds__(256)
-stream_clear_kernel(const __grid_constant__ StreamBatch B) {
+stream_clear_kernel(const __grid_constant__ StreamBatchT<N> B) {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the main kernel may take its seats now; it waits for this grid
   const StreamJob& O = B.job[blockIdx.x];
   const int n = O.j.n_blocks * O.parts;
@@ -444,11 +504,13 @@ int fused_stream(const FusedJob* jobs, int n_jobs, int block, float eps, int squ
   int st = BSP_OK;
   if (ok) {
     if (!td->attr_set[7]) {
-      cudaError_t e = cudaFuncSetAttribute(fused_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemCap);
+      cudaError_t e = cudaFuncSetAttribute(fused_stream_kernel<kStreamMaxJobs>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemCap);
+      if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(fused_stream_kernel<kStreamFewJobs>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemCap);
       if (e != cudaSuccess) { delete B; return cuda_fail(e); }
       td->attr_set[7] = true;
     }
-    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fused_stream_kernel, kStreamThreads, smem_max);
+    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fused_stream_kernel<kStreamMaxJobs>, kStreamThreads, smem_max);
     if (e != cudaSuccess) { delete B; return cuda_fail(e); }
     if (per_sm * td->sms < 32) ok = false;    // the no-deadlock argument needs 32 CTAs resident at once
   }
@@ -456,7 +518,16 @@ int fused_stream(const FusedJob* jobs, int n_jobs, int block, float eps, int squ
     const int n = n_jobs - j0 < kStreamMaxJobs ? n_jobs - j0 : kStreamMaxJobs;
     fill_batch(*B, jobs + j0, n, block, eps, squared, part_counts + j0, part_partial + j0, &smem);
     B->status = td->status;
-    stream_clear_kernel<<<n, 256, 0, s>>>(*B);
+    if (B->total_items <= per_sm * td->sms) B->ticket = nullptr;    // one wave: item = block index
+    const bool few = n <= kStreamFewJobs;
+    StreamBatchT<kStreamFewJobs> small;
+    static_assert(offsetof(StreamBatchT<kStreamFewJobs>, job) == offsetof(StreamBatch, job), "tables must share their beginning");
+    if (few) {
+      memcpy(&small, B, sizeof(small));
+      stream_clear_kernel<kStreamFewJobs><<<n, 256, 0, s>>>(small);
+    } else {
+      stream_clear_kernel<kStreamMaxJobs><<<n, 256, 0, s>>>(*B);
+    }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { st = cuda_fail(e); break; }
     cudaLaunchConfig_t cfg = {};
@@ -469,7 +540,8 @@ int fused_stream(const FusedJob* jobs, int n_jobs, int block, float eps, int squ
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    e = cudaLaunchKernelEx(&cfg, fused_stream_kernel, *B);
+    e = few ? cudaLaunchKernelEx(&cfg, fused_stream_kernel<kStreamFewJobs>, small)
+            : cudaLaunchKernelEx(&cfg, fused_stream_kernel<kStreamMaxJobs>, *B);
     if (e != cudaSuccess) { st = cuda_fail(e); break; }
     *used = true;
   }
