@@ -328,6 +328,11 @@ int bsp_linear_planned(const void* plan, int n_out, int k_in, int block,
  * BSP_LINEAR_CTA_PAIR (256 x 256 tiles shared by a cluster of two CTAs, one third less operand
  * traffic from L2).  Results are identical up to float32 summation order (the same in both). */
 typedef enum { BSP_LINEAR_AUTO = 0, BSP_LINEAR_ONE_CTA = 1, BSP_LINEAR_CTA_PAIR = 2 } bsp_linear_algo;
+/* May be OR-ed into `algo`: the caller vouches that the plan was complete before the work that
+ * immediately precedes this call in the stream was launched (the usual case in a chain of layers:
+ * the weights are old, only X is fresh).  The one-CTA kernel then starts fetching weight tiles
+ * while that work is still finishing.  Never set it when the preceding kernel writes the plan. */
+#define BSP_LINEAR_PLAN_STABLE 0x100
 int bsp_linear_planned_ex(const void* plan, int n_out, int k_in, int block,
                           const void* X, int tokens, int ldx, const void* bias, int act,
                           void* Y, int ldy, int algo, void* stream);

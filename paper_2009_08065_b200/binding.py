@@ -311,6 +311,7 @@ def bsp_linear_planned(plan: torch.Tensor, n_out: int, k_in: int, block: int, X:
 
 
 LINEAR_AUTO, LINEAR_ONE_CTA, LINEAR_CTA_PAIR = 0, 1, 2
+LINEAR_PLAN_STABLE = 0x100     # OR into `algo`: the plan is older than the previous kernel in the stream
 
 
 def bsp_linear_planned_ex(plan: torch.Tensor, n_out: int, k_in: int, block: int, X: torch.Tensor,

@@ -173,6 +173,7 @@ fused_stream_kernel(const __grid_constant__ StreamBatchT<N> B) {
     // launched with programmatic stream serialization: everything above overlapped the clearing
     // kernel; the ticket and the slots it zeroes are touched only from here on
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel may set up on SMs that become free
     if (!direct) s_item = atomicAdd(B.ticket, 1);
   }
   __syncthreads();

@@ -50,6 +50,7 @@ __device__ __align__(16) int g_linear_status[8];
 
 struct LinearParams {
   int tokens, n_out, k_in, act;
+  int plan_stable;      // the plan was complete before the kernel preceding this one in the stream began
   const uint16_t* bias;
   int* status;
 };
@@ -102,8 +103,10 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
   // Programmatic dependent launch: everything above touched only this CTA's shared and tensor
   // memory and overlaps the tail of the previous kernel in the stream.  From here on the kernel
   // reads memory that kernel may have written (X, the plan), so wait for it to finish; and let
-  // the next kernel in the stream start its own prologue as soon as SMs become free.
-  asm volatile("griddepcontrol.wait;" ::: "memory");
+  // the next kernel in the stream start its own prologue as soon as SMs become free.  When the
+  // caller vouches that the plan is older than the previous kernel, the weight producer does not
+  // wait: its first tiles are on their way while the previous kernel finishes writing X.
+  if (!(P.plan_stable && warp == 10)) asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   const int m_tiles = (P.tokens + kBlockM - 1) / kBlockM;
@@ -507,7 +510,9 @@ extern "C" int bsp_linear_planned_ex(const void* plan, int n_out, int k_in, int 
   using namespace bsp;
   int st = check_linear_args(plan, plan, plan, n_out, k_in, block, X, tokens, ldx, act, Y, ldy);
   if (st != BSP_OK) return st;
-  if (algo < BSP_LINEAR_AUTO || algo > BSP_LINEAR_CTA_PAIR) return BSP_ERR_ARG;
+  const int algo_flags = algo & ~0xff;
+  algo &= 0xff;
+  if (algo < BSP_LINEAR_AUTO || algo > BSP_LINEAR_CTA_PAIR || (algo_flags & ~BSP_LINEAR_PLAN_STABLE)) return BSP_ERR_ARG;
   if (!tc_path_ok(plan, n_out, k_in, X, ldx, Y, ldy)) return BSP_ERR_UNSUPPORTED;
   if (tokens == 0) return BSP_OK;
   TcDevice* dev = tc_device();
@@ -521,7 +526,8 @@ extern "C" int bsp_linear_planned_ex(const void* plan, int n_out, int k_in, int 
   const bool pair = algo == BSP_LINEAR_CTA_PAIR ||
                     (algo == BSP_LINEAR_AUTO && pair_tiles >= 4LL * dev->sms && act == BSP_ACT_NONE);
   if (pair) return launch_tc_pair(dev, plan, X, Y, tokens, n_out, k_in, act, bias, ldx, ldy, s);
-  LinearParams P{tokens, n_out, k_in, act, static_cast<const uint16_t*>(bias), dev->status};
+  LinearParams P{tokens, n_out, k_in, act, (algo_flags & BSP_LINEAR_PLAN_STABLE) ? 1 : 0,
+                 static_cast<const uint16_t*>(bias), dev->status};
   switch (choose_bn(tokens, n_out, dev->sms)) {
     case 256: return launch_tc<256>(dev, 0, plan, X, Y, P, ldx, ldy, s);
     case 192: return launch_tc<192>(dev, 1, plan, X, Y, P, ldx, ldy, s);
