@@ -152,7 +152,8 @@ class LayerOnDevice:
                 "Y": torch.empty((wl.tokens, spec.n_out), dtype=torch.int16, device=device),
             }
             self.lin.append(e)
-        self.kernels_per_step = 1 + len(self.lin)   # one weight-side launch for the batch, one GEMM per matrix
+        self.weight_side_launches = 2               # a small clearing kernel and the one-pass kernel
+        self.kernels_per_step = self.weight_side_launches + len(self.lin)
 
     def source(self, spec, outs):
         if spec.src == "x":
@@ -162,31 +163,32 @@ class LayerOnDevice:
             return outs["qkv"][:, 2 * h: 3 * h]
         return outs[spec.src]
 
-    def step(self, gemm_events=None):
+    def step(self, n_linears=None):
         """One pass of the path: one batched weight-side call for the four matrices (norms, gamma, penalty,
-        keep flags, pack, plan: two launches), then the four GEMMs in order."""
-        bsp, outs = self.bsp, {}
+        keep flags, pack; W, already zero where it is pruned, is its own execution layout: in-place mode), then the
+        four GEMMs in order.  `n_linears` < 4 runs only the first few GEMMs (the prefixes that give each launch's
+        share of the step)."""
+        bsp = self.bsp
+        outs = {e["spec"].name.split(".")[1]: e["Y"] for e in self.lin}   # (a prefix may start from earlier outputs)
         if not hasattr(self, "jobs"):
             self.jobs = bsp.make_job_array([
                 bsp.LayerJob(W=e["W"], out=e["pk"], threshold=0.0, norms=e["norms"], gamma_out=e["gamma"],
                              penalty=e["penalty"], plan=e["plan"]) for e in self.lin])
         bsp.bsp_prepare_batched(self.jobs, self.wl.linears[0].block, EPS, bsp.PEN_L2)
-        for i, e in enumerate(self.lin):
+        for i, e in enumerate(self.lin[:n_linears]):
             spec = e["spec"]
-            src = self.source(spec, outs)
-            if gemm_events is not None:
-                gemm_events[i][0].record()
-            bsp.bsp_linear_planned(e["plan"], spec.n_out, spec.k_in, spec.block, src, e["b"], int(spec.gelu), e["Y"])
-            if gemm_events is not None:
-                gemm_events[i][1].record()
-            outs[spec.name.split(".")[1]] = e["Y"]
+            # the weights of every linear but the first were finished before the kernel that precedes it began
+            algo = bsp.LINEAR_AUTO | (bsp.LINEAR_PLAN_STABLE if i > 0 else 0)
+            bsp.bsp_linear_planned_ex(e["plan"], spec.n_out, spec.k_in, spec.block, self.source(spec, outs), e["b"],
+                                      int(spec.gelu), e["Y"], algo)
         return outs
 
-    def upload_inputs(self):
-        self.dev_all.copy_(self.host_all, non_blocking=True)
+    def upload_inputs(self, activations_only=False):
+        n = self.x.numel() if activations_only else self.host_all.numel()       # x is the first view of the buffer
+        self.dev_all[:n].copy_(self.host_all[:n], non_blocking=True)
 
-    def h2d_bytes(self):
-        return self.host_all.numel() * 2
+    def h2d_bytes(self, activations_only=False):
+        return (self.x.numel() if activations_only else self.host_all.numel()) * 2
 
     def nonzero_flops(self):
         self.torch.cuda.synchronize()
@@ -258,7 +260,7 @@ def stack_jobs(device):
                                  norms=torch.empty(shape, dtype=torch.float32, device=device),
                                  gamma_out=torch.empty(shape, dtype=torch.float32, device=device),
                                  penalty=torch.zeros(1, dtype=torch.float64, device=device),
-                                 plan=torch.empty(rows * cols * 2, dtype=torch.uint8, device=device)))
+                                 plan=w))          # in-place mode: W, zero where pruned, is its own execution layout
         weights += rows * cols
         groups += shape[0] * shape[1]
         kept += int(keep.sum().item())
@@ -267,8 +269,9 @@ def stack_jobs(device):
 
 def weight_side_bandwidth(device, peaks, iters=10):
     """Achieved HBM GB/s of the weight-side kernels (bsp_prepare_batched: norms, gamma, penalty, keep flags,
-    pack, plan) on the 72 weight matrices of a BERT-base encoder stack in one call, L2 flushed before each
-    run.  A single 768x768 matrix is 1.2 MB, far too small to time against HBM on its own."""
+    pack; in-place mode, so no separate execution layout is written) on the 72 weight matrices of a BERT-base
+    encoder stack in one call, L2 flushed before each run.  A single 768x768 matrix is 1.2 MB, far too small to
+    time against HBM on its own."""
     import torch
     import paper_2009_08065_b200 as bsp
     arr, d, weights, groups, kept, _keepalive = stack_jobs(device)
@@ -283,15 +286,18 @@ def weight_side_bandwidth(device, peaks, iters=10):
         torch.cuda.synchronize()
         if i >= 3:
             ms.append(a.elapsed_time(b))
-    t = statistics.median(ms)
+    t = statistics.mean(ms)
     # algorithmic bytes: W read once (2 B/weight); norms + gamma (4 B each) and a flag (1 B) per group;
-    # kept values (2 B) and one index (4 B) per kept group; the execution layout (2 B/weight)
-    alg = 2 * weights + 9 * groups + 2 * d * kept + 4 * kept + 2 * weights
+    # kept values (2 B) and one index (4 B) per kept group.  No execution layout: W already holds zeros in the
+    # pruned groups, so in-place mode writes nothing into it.
+    alg = 2 * weights + 9 * groups + 2 * d * kept + 4 * kept
     return {"kernels": "fused_stream_kernel (bsp_prepare_batched; W read once) + its clearing kernel",
             "workload": f"72 BERT-base weight matrices in one call, {weights * 2 / 1e6:.1f} MB of bf16 weights, d=16, ~3x",
             "ms": round(t, 4), "algorithmic_mb": round(alg / 1e6, 1), "achieved_gbs": round(alg / t / 1e6, 1),
             "peak_gbs": float(peaks["hbm_gbs"]), "frac": round(alg / t / 1e6 / float(peaks["hbm_gbs"]), 4),
-            "l2": "flushed before each run"}
+            "algorithmic_bytes_formula": "2/weight (W once) + 9/group (norm, gamma, flag) + (2d + 4)/kept group (values, index)",
+            "plan_bytes": 0, "plan_note": "in-place mode: no separate execution layout is written",
+            "l2": "flushed before each run", "timing": f"mean of {iters} launches"}
 
 
 def retrain_step_bandwidth(device, peaks, iters=10):
@@ -324,6 +330,276 @@ def retrain_step_bandwidth(device, peaks, iters=10):
             "l2": "working set 2.5 GB per launch, larger than L2"}
 
 
+def _timed_graph(torch, fn, flush, iters, cold):
+    """Mean milliseconds of `fn` captured as a CUDA graph; cold = L2 flushed before every replay, else back to back."""
+    a, b = torch.cuda.Event(enable_timing=True, external=True), torch.cuda.Event(enable_timing=True, external=True)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        a.record()
+        fn()
+        b.record()
+    ms = []
+    for i in range(iters + 2):
+        if cold:
+            flush.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        if i >= 2:
+            ms.append(a.elapsed_time(b))
+    return statistics.mean(ms)
+
+
+def _stack_report(name, tokens, mats, t_full, t_gemm, peaks, note):
+    """Figures of a chained stack: mats = [(n_out, k_in, block, kept_weights)], t_* = {"cold": ms, "warm": ms}."""
+    peak, hbm = float(peaks["bf16_tflops"]), float(peaks["hbm_gbs"])
+    flops = [2 * tokens * kw for (_n, _k, _d, kw) in mats]
+    byts = [2 * tokens * k + 2 * kw + 4 * (kw // d) + 2 * tokens * n + 2 * n for (n, k, d, kw) in mats]
+    t_roof = sum(max(f / peak / 1e9, b / hbm / 1e6) for f, b in zip(flops, byts))     # ms, min(tensor, HBM) roofline
+    total = sum(n * k for (n, k, _d, _kw) in mats)
+    kept = sum(kw for (*_x, kw) in mats)
+    out = {"workload": name, "tokens": tokens, "matrices": len(mats), "nonzero_gflop": round(sum(flops) / 1e9, 2),
+           "compression": round(total / kept, 4), "algorithmic_mb": round(sum(byts) / 1e6, 1),
+           "roofline_ms": round(t_roof, 4), "note": note}
+    for label, t in (("gemms", t_gemm), ("with_weight_side", t_full)):
+        out[label] = {
+            k: {"ms": round(v, 4), "nonzero_tflops": round(sum(flops) / v / 1e9, 1),
+                "percent_of_bf16_peak": round(100 * sum(flops) / v / 1e9 / peak, 2),
+                "frac_of_min_tensor_hbm_roofline": round(t_roof / v, 4) if label == "gemms" else None}
+            for k, v in t.items()}
+    return out
+
+
+def stack_72_matrices(device, peaks, iters=5):
+    """The 72 weight matrices of a BERT-base encoder stack (12 layers of Q, K, V, O, FFN-up, FFN-down), 4096 tokens,
+    16-row blocks, per-matrix rates drawn from U(3, 7) and scaled to 5.0x overall, layer outputs chained (O reads V's
+    output, FFN-up reads O's through GELU, FFN-down reads FFN-up's, the next layer reads FFN-down's)."""
+    import torch
+    import paper_2009_08065_b200 as bsp
+    T, H, F, d = 4096, 768, 3072, 16
+    rates = si.bert_base_stack_rates(si.DEFAULT_SEED)
+    gen = torch.Generator(device=device)
+    gen.manual_seed(si.DEFAULT_SEED)
+    shapes = [("q", H, H, 0), ("k", H, H, 0), ("v", H, H, 0), ("o", H, H, 0), ("up", F, H, 1), ("down", H, F, 0)]
+    x0 = torch.randn(T, H, device=device, generator=gen).to(torch.bfloat16)
+    bufs = {nm: torch.empty(T, n, dtype=torch.bfloat16, device=device) for nm, n, _k, _a in shapes}
+    nxt = torch.empty(T, H, dtype=torch.bfloat16, device=device)
+    layers, jobs, mats = [], [], []
+    for l in range(12):
+        ops = []
+        for j, (nm, n, k, act) in enumerate(shapes):
+            kc = int(round(k / rates[l][j]))
+            w = (torch.randn(n, k, device=device, generator=gen) * 0.02).to(torch.bfloat16)
+            keep = torch.zeros(n // d, k, dtype=torch.bool, device=device)
+            keep.scatter_(1, torch.rand(n // d, k, device=device, generator=gen).topk(kc, dim=1).indices, True)
+            w = (w.view(n // d, d, k) * keep[:, None, :]).view(n, k).contiguous()
+            bias = (torch.randn(n, device=device, generator=gen) * 0.02).to(torch.bfloat16)
+            pk = bsp.PackedMatrix.allocate(n, k, d, bsp.ORIENT_C, device)
+            g = (n // d, k)
+            jobs.append(bsp.LayerJob(W=w, out=pk, threshold=0.0, norms=torch.empty(g, dtype=torch.float32, device=device),
+                                     gamma_out=torch.empty(g, dtype=torch.float32, device=device),
+                                     penalty=torch.zeros(1, dtype=torch.float64, device=device), plan=w))
+            ops.append((nm, w, bias, n, k, act))
+            mats.append((n, k, d, d * kc * (n // d)))
+        layers.append(ops)
+    arr = bsp.make_job_array(jobs)
+
+    def gemms():
+        src, first = x0, True
+        for l, ops in enumerate(layers):
+            out_down = nxt if l % 2 == 0 else bufs["down"]
+            for nm, w, bias, n, k, act in ops:
+                inp = {"q": src, "k": src, "v": src, "o": bufs["v"], "up": bufs["o"], "down": bufs["up"]}[nm]
+                dst = out_down if nm == "down" else bufs[nm]
+                bsp.bsp_linear_planned_ex(w, n, k, d, inp, bias, act, dst, 0 if first else bsp.LINEAR_PLAN_STABLE)
+                first = False
+            src = out_down
+
+    def full():
+        bsp.bsp_prepare_batched(arr, d, EPS, bsp.PEN_L2)
+        gemms()
+
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=device)
+    full()
+    bsp.bsp_linear_status()
+    t_gemm = {"cold": _timed_graph(torch, gemms, flush, iters, True), "warm": _timed_graph(torch, gemms, flush, iters, False)}
+    t_full = {"cold": _timed_graph(torch, full, flush, iters, True), "warm": _timed_graph(torch, full, flush, iters, False)}
+    bsp.bsp_linear_status()
+    return _stack_report("BERT-base stack, 72 matrices, 5.0x overall, d=16", T, mats, t_full, t_gemm, peaks,
+                         "cold = L2 flushed before each pass over the stack (activations then stay in L2 from one linear to the next); "
+                         "warm = passes back to back (170 MB of weights do not fit the 126 MB L2); one CUDA graph per pass")
+
+
+def stack_distil(device, peaks, iters=5):
+    """DistilBERT-shaped stack: 6 layers (fused QKV, O, FFN-up, FFN-down), 8192 tokens, 32-row blocks, heavy-tailed
+    weights (Student-t, 3 degrees of freedom, std 0.02), every matrix through the real pipeline in every pass:
+    bsp_percentile_threshold_batched (1.79x) -> bsp_prepare_batched with that device threshold (norms, gamma, penalty, flags,
+    pack, W masked in place) -> the linear layer; kept counts differ from block to block."""
+    import torch
+    import paper_2009_08065_b200 as bsp
+    wl = si.distil_stack()
+    T, d = wl.tokens, wl.linears[0].block
+    gen = torch.Generator(device=device)
+    gen.manual_seed(si.DEFAULT_SEED + 4)
+    x0 = torch.randn(T, 768, device=device, generator=gen).to(torch.bfloat16)
+    ops, jobs = [], []
+    for spec in wl.linears:
+        n, k = spec.n_out, spec.k_in
+        z = torch.randn(n, k, device=device, generator=gen)
+        chi = (torch.randn(3, n, k, device=device, generator=gen) ** 2).sum(0) / 3.0
+        w0 = (z / chi.sqrt() * (0.02 / 3 ** 0.5)).to(torch.bfloat16)
+        w = w0.clone()
+        thr = torch.zeros(1, dtype=torch.float32, device=device)
+        pk = bsp.PackedMatrix.allocate(n, k, d, bsp.ORIENT_C, device)
+        g = (n // d, k)
+        jobs.append(bsp.LayerJob(W=w, out=pk, threshold=0.0, threshold_dev=thr,
+                                 norms=torch.empty(g, dtype=torch.float32, device=device),
+                                 gamma_out=torch.empty(g, dtype=torch.float32, device=device),
+                                 penalty=torch.zeros(1, dtype=torch.float64, device=device), plan=w))
+        ops.append({"spec": spec, "w0": w0, "w": w, "thr": thr, "pk": pk,
+                    "bias": (torch.randn(n, device=device, generator=gen) * 0.02).to(torch.bfloat16),
+                    "y": torch.empty(T, n, dtype=torch.bfloat16, device=device)})
+    arr = bsp.make_job_array(jobs)
+
+    def restore():
+        for o in ops:
+            o["w"].copy_(o["w0"])
+
+    rates = [o["spec"].rate for o in ops]
+
+    def weight_side():
+        bsp.bsp_percentile_threshold_batched(arr, d, rates)
+        bsp.bsp_prepare_batched(arr, d, EPS, bsp.PEN_L2)
+
+    def gemms():
+        outs = {}
+        for i, o in enumerate(ops):
+            spec = o["spec"]
+            layer_tag, nm = spec.name.split(".")
+            if spec.src == "x":
+                src = x0
+            elif spec.src == "qkv_v":
+                src = outs[layer_tag + ".qkv"][:, 2 * spec.k_in: 3 * spec.k_in]
+            elif "." in spec.src:
+                src = outs[spec.src]
+            else:
+                src = outs[layer_tag + "." + spec.src]
+            bsp.bsp_linear_planned_ex(o["w"], spec.n_out, spec.k_in, d, src, o["bias"], int(spec.gelu), o["y"],
+                                      bsp.LINEAR_PLAN_STABLE if i > 0 else 0)
+            outs[spec.name] = o["y"]
+
+    def full():
+        restore()            # the pass prunes the unpruned weights every time (this copy is part of the timed pass)
+        weight_side()
+        gemms()
+
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=device)
+    full()
+    bsp.bsp_linear_status()
+    torch.cuda.synchronize()
+    mats = [(o["spec"].n_out, o["spec"].k_in, d, int(o["pk"].kept_weights.item())) for o in ops]
+    t_gemm = {"cold": _timed_graph(torch, gemms, flush, iters, True), "warm": _timed_graph(torch, gemms, flush, iters, False)}
+    t_full = {"cold": _timed_graph(torch, full, flush, iters, True), "warm": _timed_graph(torch, full, flush, iters, False)}
+    bsp.bsp_linear_status()
+    return _stack_report("DistilBERT-shaped stack, 24 matrices (fused QKV), 1.79x by per-matrix percentile, d=32, Student-t weights",
+                         T, mats, t_full, t_gemm, peaks,
+                         "with_weight_side = restore the unpruned weights (a device copy), percentile threshold, norms/gamma/penalty/"
+                         "flags/pack with W masked in place, then the linears; gemms = the linears alone on the masked weights")
+
+
+def bert_large_grid(device, peaks, tokens, iters, shapes_filter=None, emit=None):
+    """The BERT-large grid (hidden 1024, FFN 4096): compression 1.5/2/3/5/8 x block height 8/16/32/64 on the four linear
+    shapes; per point the zero-expanded route (bsp_linear_planned) and, where the block height allows, the gathering
+    kernel (bsp_linear_gathered on transposed activations), each launch after an L2 flush, mean of `iters`."""
+    import torch
+    import paper_2009_08065_b200 as bsp
+    peak = float(peaks["bf16_tflops"])
+    T = tokens
+    shapes = [("qkv", 3072, 1024, 0), ("attn_out", 1024, 1024, 0), ("ffn_up", 4096, 1024, 1), ("ffn_down", 1024, 4096, 0)]
+    if shapes_filter:
+        shapes = [sh for sh in shapes if sh[0] in shapes_filter]
+    gen = torch.Generator(device=device)
+    gen.manual_seed(si.DEFAULT_SEED)
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=device)
+
+    def timed(fn):
+        ms = []
+        for i in range(iters + 2):
+            flush.zero_()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            fn()
+            b.record()
+            torch.cuda.synchronize()
+            if i >= 2:
+                ms.append(a.elapsed_time(b))
+        return statistics.mean(ms)
+
+    points = []
+    for name, N, K, act in shapes:
+        X = torch.randn(T, K, device=device, generator=gen).to(torch.bfloat16)
+        XT = torch.empty(K, T, dtype=torch.bfloat16, device=device)
+        t_tr = timed(lambda: bsp.bsp_transpose(X, XT))
+        bias = (torch.randn(N, device=device, generator=gen) * 0.02).to(torch.bfloat16)
+        Y = torch.empty(T, N, dtype=torch.bfloat16, device=device)
+        Yg = torch.empty(T, N, dtype=torch.bfloat16, device=device)
+        Wd = (torch.randn(N, K, device=device, generator=gen) * 0.02).to(torch.bfloat16)
+        t_dense = timed(lambda: torch.matmul(X, Wd.t()))
+        for d in (8, 16, 32, 64):
+            for c in (1.5, 2.0, 3.0, 5.0, 8.0):
+                kc = int(round(K / c))
+                keep = torch.zeros(N // d, K, dtype=torch.bool, device=device)
+                keep.scatter_(1, torch.rand(N // d, K, device=device, generator=gen).topk(kc, dim=1).indices, True)
+                W = (Wd.view(N // d, d, K) * keep[:, None, :]).view(N, K).contiguous()      # masked W = its own execution layout
+                nz = 2.0 * T * d * kc * (N // d)
+                t_plan = timed(lambda: bsp.bsp_linear_planned(W, N, K, d, X, bias, act, Y))
+                point = {"shape": name, "tokens": T, "n_out": N, "k_in": K, "block": d, "compression": c,
+                         "nonzero_gflop": round(nz / 1e9, 2), "dense_route_ms": round(t_plan, 4),
+                         "dense_route_nonzero_tflops": round(nz / t_plan / 1e9, 1),
+                         "torch_dense_ms": round(t_dense, 4), "transpose_ms": round(t_tr, 4)}
+                best, route = nz / t_plan / 1e9, "zero-expanded"
+                if d in (16, 32, 64, 128):
+                    pk = bsp.PackedMatrix.allocate(N, K, d, bsp.ORIENT_C, device)
+                    bsp.bsp_prune_pack(W, pk, 0.0)
+                    gplan = torch.empty(bsp.bsp_linear_gather_plan_bytes(N, K, d), dtype=torch.uint8, device=device)
+                    bsp.bsp_linear_gather_plan(pk, gplan)
+                    t_g = timed(lambda: bsp.bsp_linear_gathered(gplan, N, K, d, XT, bias, act, Yg))
+                    point.update({"gather_ms": round(t_g, 4), "gather_nonzero_tflops": round(nz / t_g / 1e9, 1),
+                                  "max_abs_diff_between_routes": (Y.float() - Yg.float()).abs().max().item()})
+                    if nz / t_g / 1e9 > best:
+                        best, route = nz / t_g / 1e9, "gathered"
+                    del gplan, pk
+                f, b = nz, 2 * T * K + 2 * N * kc + 4 * (N // d) * kc + 2 * T * N + 2 * N
+                t_roof = max(f / peak / 1e9, b / float(peaks["hbm_gbs"]) / 1e6)
+                point.update({"best_route": route, "best_nonzero_tflops": round(best, 1),
+                              "best_percent_of_bf16_peak": round(100.0 * best / peak, 2),
+                              "frac_of_min_tensor_hbm_roofline": round(t_roof / (nz / best / 1e9), 4)})
+                bsp.bsp_linear_status()
+                points.append(point)
+                if emit:
+                    emit(point)
+                del W, keep
+    return points
+
+
+def other_workloads(device, peaks, args):
+    """Figures of the workloads that are not the bench line's own: outside its timed region, fewer repetitions."""
+    out = {"bert_base_stack_72": stack_72_matrices(device, peaks), "distil_stack": stack_distil(device, peaks)}
+    pts = bert_large_grid(device, peaks, 32768, 3)
+    out["bert_large_grid"] = {
+        "tokens": 32768, "how": "each launch after an L2 flush, mean of 3; cells = [best non-zero TFLOP/s, % of bf16 peak, route]; "
+                                "the gathering kernel's figures take the transposed activations as given (see transpose_ms)",
+        "cells": {f"{p['shape']}/d{p['block']}/c{p['compression']:g}": [p["best_nonzero_tflops"], p["best_percent_of_bf16_peak"],
+                                                                       "g" if p["best_route"] == "gathered" else "z"] for p in pts},
+        "transpose_ms": {p["shape"]: p["transpose_ms"] for p in pts}}
+    return out
+
+
+def section_8d_bytes(tokens, spec, kept_weights):
+    """Algorithmic bytes of one pruned linear: X once, the kept values and one index per kept group, Y once, the bias."""
+    return (2 * tokens * spec.k_in + 2 * kept_weights + 4 * (kept_weights // spec.block)
+            + 2 * tokens * spec.n_out + 2 * spec.n_out)
+
+
 def run_cuda(args):
     import torch
     import torch.distributed as dist
@@ -341,6 +617,7 @@ def run_cuda(args):
     wl = workload()
     layer = LayerOnDevice(wl, si.DEFAULT_SEED, rank, device)
     flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=device)
+    n_lin = len(layer.lin)
 
     # warm-up outside any graph (first calls set function attributes and the status word)
     for _ in range(max(args.warmup, 3)):
@@ -348,49 +625,45 @@ def run_cuda(args):
     layer.bsp.bsp_linear_status()
     flops = layer.nonzero_flops()
     step_flops = sum(flops)
+    kept = [f // (2 * wl.tokens) for f in flops]
 
-    # The step as a CUDA graph.  Two captures of the same call sequence: `graph` carries only the two
-    # events that bracket the step and gives `value`; `graph_k` also brackets every GEMM launch and gives
-    # the per-kernel durations of the roofline block (event nodes between kernels cost a few microseconds
-    # each, so they are kept out of the step that is timed as a whole).
+    # The step as a CUDA graph, bracketed by two event nodes: it gives `value`.  The same call sequence cut
+    # after the weight-side call and after each GEMM gives n_lin more graphs (prefixes); the difference between
+    # two neighbouring prefixes is what a launch adds to the step, so the shares add up to the step exactly and
+    # no event node sits between two kernels.  Every replay, of the step or of a prefix, follows its own L2 flush.
     ev = lambda: torch.cuda.Event(enable_timing=True, external=True)  # noqa: E731
-    ev_step = (ev(), ev())
-    ev_gemm = [(ev(), ev()) for _ in layer.lin]
-    graph, graph_k = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
-    with torch.cuda.graph(graph):
-        ev_step[0].record()
-        layer.step()
-        ev_step[1].record()
-    with torch.cuda.graph(graph_k):
-        layer.step(gemm_events=ev_gemm)
-    for _ in range(max(args.warmup, 3)):
-        flush.zero_()
-        graph.replay()
-        flush.zero_()
-        graph_k.replay()
-    torch.cuda.synchronize()
+    graphs = []
+    for k in range(n_lin + 1):
+        g, pair = torch.cuda.CUDAGraph(), (ev(), ev())
+        with torch.cuda.graph(g):
+            pair[0].record()
+            layer.step(n_linears=k)
+            pair[1].record()
+        graphs.append((g, pair))
+    graph, ev_step = graphs[n_lin]
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    step_ms, gemm_ms = [], [[] for _ in layer.lin]
-    barrier()
-    with ClockSampler(local_rank) as clocks:
+    prefix_ms = [[] for _ in graphs]
+    with ClockSampler(local_rank) as clocks:          # sampling starts with the warm-up replays: short runs still get samples
+        for _ in range(max(args.warmup, 3)):
+            for g, _pair in graphs:
+                flush.zero_()
+                g.replay()
+        barrier()
         for _ in range(args.steps):
-            flush.zero_()                  # untimed: evict the step's inputs from L2
-            graph.replay()
-            torch.cuda.synchronize()
-            step_ms.append(ev_step[0].elapsed_time(ev_step[1]))
-            flush.zero_()
-            graph_k.replay()               # same step again, instrumented per kernel (not part of `value`)
-            torch.cuda.synchronize()
-            for i, (a, b) in enumerate(ev_gemm):
-                gemm_ms[i].append(a.elapsed_time(b))
-    barrier()
+            for k in (n_lin, *range(n_lin)):          # the whole step first, then its prefixes
+                g, pair = graphs[k]
+                flush.zero_()                         # untimed: evict the inputs from L2
+                g.replay()
+                torch.cuda.synchronize()
+                prefix_ms[k].append(pair[0].elapsed_time(pair[1]))
+        barrier()
     layer.bsp.bsp_linear_status()
-    total_ms = sum(step_ms)
+    total_ms = sum(prefix_ms[n_lin])
 
     # the same step back to back without the flush: W, X and the intermediate outputs (about 100 MB) are
     # still in L2 from the previous step.  Context beside `value`, which is the flushed figure.
@@ -437,7 +710,7 @@ def run_cuda(args):
     pen_hosts = [pen_host, torch.empty_like(pen_host).pin_memory()]
     s_main, s_in, s_out = torch.cuda.current_stream(), torch.cuda.Stream(), torch.cuda.Stream()
 
-    def pipelined(n_steps):
+    def pipelined(n_steps, activations_only=False):
         ev_in = [torch.cuda.Event(), torch.cuda.Event()]
         ev_done = [torch.cuda.Event(), torch.cuda.Event()]
         ev_out = [torch.cuda.Event(), torch.cuda.Event()]
@@ -447,7 +720,7 @@ def run_cuda(args):
             with torch.cuda.stream(s_in):
                 if it >= 2:
                     s_in.wait_event(ev_done[k])        # the kernels of step it-2 have read this set's inputs
-                lay.upload_inputs()
+                lay.upload_inputs(activations_only)
                 ev_in[k].record(s_in)
             s_main.wait_event(ev_in[k])
             if it >= 2:
@@ -463,25 +736,37 @@ def run_cuda(args):
         for k in range(min(2, n_steps)):
             s_main.wait_event(ev_out[k])
 
-    pipelined(max(args.warmup, 3))
-    barrier()
-    e_s.record()
-    pipelined(args.steps)
-    e_e.record()
-    torch.cuda.synchronize()
-    e2e_total_ms = e_s.elapsed_time(e_e)
-    barrier()
+    e2e_totals = []
+    for act_only in (False, True):
+        pipelined(max(args.warmup, 3), act_only)
+        barrier()
+        e_s.record()
+        pipelined(args.steps, act_only)
+        e_e.record()
+        torch.cuda.synchronize()
+        e2e_totals.append(e_s.elapsed_time(e_e))
+        barrier()
+    e2e_total_ms, e2e_act_total_ms = e2e_totals
     layer_b.bsp.bsp_linear_status()
 
-    total_ms, e2e_total_ms, e2e_serial_total_ms = reduce_max([total_ms, e2e_total_ms, e2e_serial_total_ms], device, world)
+    reduced = reduce_max([total_ms, e2e_total_ms, e2e_serial_total_ms, e2e_act_total_ms], device, world)
+    total_ms, e2e_total_ms, e2e_serial_total_ms, e2e_act_total_ms = reduced
 
     if rank == 0:
         peaks, peak_src = measured_peaks()
-        gemm_mean_ms = [statistics.mean(v) for v in gemm_ms]
-        gemm_total = sum(gemm_mean_ms)
-        achieved = step_flops / gemm_total / 1e9          # TFLOP/s over the four GEMM launches of a step
-        peak = float(peaks["bf16_tflops"])
+        peak, hbm_peak = float(peaks["bf16_tflops"]), float(peaks["hbm_gbs"])
         value = job_throughput(world, step_flops, args.steps, total_ms)
+        step_mean = statistics.mean(prefix_ms[n_lin])
+        pre = [statistics.mean(v) for v in prefix_ms]                 # pre[k]: weight side + the first k GEMMs
+        weight_ms = pre[0]
+        share = [(pre[k + 1] if k + 1 < n_lin else step_mean) - pre[k] for k in range(n_lin)]
+        gemm_total = sum(share)                                       # = step - weight side, by construction
+        alg_bytes = [section_8d_bytes(wl.tokens, e["spec"], kept[i]) for i, e in enumerate(layer.lin)]
+        t_tensor = step_flops / peak / 1e9                            # ms at the tensor peak
+        t_hbm = sum(alg_bytes) / hbm_peak / 1e6                       # ms at the HBM peak, on the method's bytes
+        hbm_binds = t_hbm >= t_tensor
+        ach_tf, ach_gbs = step_flops / gemm_total / 1e9, sum(alg_bytes) / gemm_total / 1e6
+        names = [e["spec"].name.split(".")[1] for e in layer.lin]
         line = {
             "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": round(total_ms / args.steps, 5), "higher_is_better": True,
@@ -489,9 +774,10 @@ def run_cuda(args):
             "config": {
                 "workload": wl.name + " (one BERT-base encoder layer: QKV, attn-out, FFN-up+GELU, FFN-down; "
                             "tokens per GPU 4096; 16-row blocks; 3.0x compression)",
-                "step": "bsp_prepare_batched (norms+gamma+penalty, keep flags, pack, plan of the 4 matrices: a clearing kernel and one kernel that reads W once) "
-                        "then the 4 GEMMs in sequence (bsp_linear_planned; the single chained launch bsp_linear_chain measured "
-                        "8 % slower on this workload); one CUDA graph",
+                "step": "bsp_prepare_batched (norms+gamma+penalty, keep flags, pack of the 4 matrices, in-place mode: a clearing "
+                        "kernel and one kernel that reads W once) then the 4 GEMMs in sequence (bsp_linear_planned_ex on the "
+                        "zero-expanded weights; the single chained launch bsp_linear_chain measured 8 % slower on this "
+                        "workload); one CUDA graph",
                 "l2": f"flushed between steps by writing {L2_FLUSH_BYTES >> 20} MiB",
                 "parallelism": "token split, replicated weights, no collective" if world > 1 else "single GPU",
                 "nonzero_gflop_per_step_per_gpu": round(step_flops / 1e9, 3),
@@ -503,29 +789,49 @@ def run_cuda(args):
                     "h2d_bytes_per_step": layer.h2d_bytes(),
                     "d2h_bytes_per_step": y_host.numel() * 2 + pen_host.numel() * 8,
                     "how": "double-buffered: two sets of device buffers, copies on their own streams overlap the "
-                           "kernels of the neighbouring steps; every step copies all its inputs in and its result out",
-                    "one_step_at_a_time": round(job_throughput(world, step_flops, len(e2e_ms), e2e_serial_total_ms), 3)},
-            "gpu_launches": 2 * layer.kernels_per_step * args.steps,
+                           "kernels of the neighbouring steps; every step copies all its inputs (activations, weights, "
+                           "biases) in and its result out",
+                    "one_step_at_a_time": round(job_throughput(world, step_flops, len(e2e_ms), e2e_serial_total_ms), 3),
+                    "activations_only": {
+                        "value": round(job_throughput(world, step_flops, args.steps, e2e_act_total_ms), 3),
+                        "h2d_bytes_per_step": layer.h2d_bytes(True),
+                        "how": "the same, with the weights and biases left on the device (they are 14.2 of the 20.5 MB)"}},
+            "gpu_launches": args.steps * sum(layer.weight_side_launches + k for k in range(n_lin + 1)),
             "clocks": clocks.summary(),
             "roofline": {
-                "kernel": "linear_tc_kernel (bsp_linear_planned), the four launches of a step",
-                "bound": "tensor", "achieved": round(achieved, 2), "peak": peak, "unit": "TFLOP/s",
-                "frac": round(achieved / peak, 4),
-                # dram__bytes_read.sum + dram__bytes_write.sum of the four launches, one ncu capture each
-                # (profiles/linear_tc_kernel_bert_base_T4096.md); Y is still in L2 when each kernel ends
-                "traffic": 58.31e6, "algorithmic_bytes": sum(
-                    2 * wl.tokens * sp.k_in + 2 * sp.n_out * sp.k_in + 2 * wl.tokens * sp.n_out + 2 * sp.n_out
-                    for sp in wl.linears),
-                "peak_source": f"bf16_tflops burst, {peak_src}",
-                "per_launch": {e["spec"].name.split(".")[1]: {
-                    "ms": round(gemm_mean_ms[i], 5), "nonzero_tflops": round(flops[i] / gemm_mean_ms[i] / 1e9, 1)}
-                    for i, e in enumerate(layer.lin)},
+                "kernel": "linear_tc_kernel (bsp_linear_planned_ex), the four launches of a step",
+                "bound": "hbm" if hbm_binds else "tensor",
+                "achieved": round(ach_gbs if hbm_binds else ach_tf, 2),
+                "peak": hbm_peak if hbm_binds else peak, "unit": "GB/s" if hbm_binds else "TFLOP/s",
+                "frac": round((ach_gbs / hbm_peak) if hbm_binds else (ach_tf / peak), 4),
+                "binding": f"at this size the algorithmic bytes need {1e3 * t_hbm:.1f} us at the HBM peak and the non-zero FLOPs "
+                           f"{1e3 * t_tensor:.1f} us at the bf16 peak: the {'HBM' if hbm_binds else 'tensor'} roofline is the one that binds",
+                "tensor": {"achieved": round(ach_tf, 2), "peak": peak, "unit": "TFLOP/s", "frac": round(ach_tf / peak, 4),
+                           "executed_tflops": round(sum(2 * wl.tokens * e["spec"].n_out * e["spec"].k_in for e in layer.lin) / gemm_total / 1e9, 1),
+                           "note": "non-zero FLOPs; the kernel multiplies the zero-expanded weights, so it executes 3.0x as many"},
+                "hbm": {"achieved": round(ach_gbs, 1), "peak": hbm_peak, "unit": "GB/s", "frac": round(ach_gbs / hbm_peak, 4)},
+                "ms": round(gemm_total, 5),
+                "how": "step minus the weight-side prefix; each launch's share = difference of two neighbouring prefixes of the "
+                       "step, every prefix its own CUDA graph replayed after an L2 flush in the timed loop",
+                "algorithmic_bytes": sum(alg_bytes),
+                "algorithmic_bytes_formula": "per linear 2TK + 2 kept + 4 kept/d + 2TN + 2N (X once, kept values, one index per kept group, Y once, bias)",
+                "traffic": None,
+                "traffic_note": "dram bytes of the four launches are in profiles/linear_tc_kernel_bert_base_T4096.md (one ncu capture per launch); "
+                                "not re-measured by this run",
+                "peak_source": f"{'hbm_gbs' if hbm_binds else 'bf16_tflops burst'}, {peak_src}",
+                "weight_side_ms": round(weight_ms, 5),
+                "per_launch": {names[i]: {"ms": round(share[i], 5), "nonzero_tflops": round(flops[i] / share[i] / 1e9, 1),
+                                          "algorithmic_gbs": round(alg_bytes[i] / share[i] / 1e6, 1)}
+                               for i in range(n_lin)},
+                "sum_check": {"weight_side_plus_launches_ms": round(weight_ms + gemm_total, 5), "step_ms": round(step_mean, 5)},
             },
         }
         if world == 1:
             line["weight_side_hbm"] = weight_side_bandwidth(device, peaks)
             line["retrain_step_hbm"] = retrain_step_bandwidth(device, peaks)
             line["dense_gemm_context"] = dense_context(wl, device)
+            if not args.no_extras:
+                line["other_workloads"] = other_workloads(device, peaks, args)
             line["cpu_baseline"] = oracle_baseline(wl, reps=3)
         print(json.dumps(line), flush=True)
     if world > 1:
@@ -668,80 +974,13 @@ def run_case(args):
 
 
 def run_sweep(args):
-    """The BERT-large sweep (hidden 1024, FFN 4096, tokens 32768 by default): compression 1.5/2/3/5/8 x block height
-    8/16/32/64 (and 128) on the four linear shapes.  For every point: the zero-expanded dense route (bsp_linear_planned), the
-    gathering kernel (bsp_linear_gathered, block heights it takes; X transposed beforehand, that copy timed
-    separately once per input width), and torch.matmul on the dense shape as context.  L2 is flushed (256 MiB
-    written) before every timed launch; medians of `--steps` launches.  One JSON line per point."""
+    """The BERT-large grid, one JSON line per point (see bert_large_grid)."""
     import torch
-    import paper_2009_08065_b200 as bsp
     torch.cuda.set_device(0)
-    device = torch.device("cuda", 0)
     peaks, _ = measured_peaks()
-    peak = float(peaks["bf16_tflops"])
-    T = args.sweep_tokens
-    iters = max(3, min(args.steps, 20))
-    shapes = [("qkv", 3072, 1024, 0), ("attn_out", 1024, 1024, 0), ("ffn_up", 4096, 1024, 1), ("ffn_down", 1024, 4096, 0)]
-    if args.sweep_shapes:
-        shapes = [sh for sh in shapes if sh[0] in args.sweep_shapes.split(",")]
-    gen = torch.Generator(device=device)
-    gen.manual_seed(si.DEFAULT_SEED)
-    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=device)
-
-    def timed(fn):
-        ms = []
-        for i in range(iters + 2):
-            flush.zero_()
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record()
-            fn()
-            b.record()
-            torch.cuda.synchronize()
-            if i >= 2:
-                ms.append(a.elapsed_time(b))
-        return statistics.median(ms)
-
-    for name, N, K, act in shapes:
-        X = torch.randn(T, K, device=device, generator=gen).to(torch.bfloat16)
-        XT = torch.empty(K, T, dtype=torch.bfloat16, device=device)
-        t_tr = timed(lambda: bsp.bsp_transpose(X, XT))
-        bias = (torch.randn(N, device=device, generator=gen) * 0.02).to(torch.bfloat16)
-        Y = torch.empty(T, N, dtype=torch.bfloat16, device=device)
-        Yg = torch.empty(T, N, dtype=torch.bfloat16, device=device)
-        Wd = (torch.randn(N, K, device=device, generator=gen) * 0.02).to(torch.bfloat16)
-        t_dense = timed(lambda: torch.matmul(X, Wd.t()))
-        for d in (8, 16, 32, 64, 128):        # 128 is beyond the named grid: it shows where the gathering kernel is heading
-            for c in (1.5, 2.0, 3.0, 5.0, 8.0):
-                kc = int(round(K / c))
-                scores = torch.rand(N // d, K, device=device, generator=gen)
-                keep = torch.zeros(N // d, K, dtype=torch.bool, device=device)
-                keep.scatter_(1, scores.topk(kc, dim=1).indices, True)
-                W = (Wd.view(N // d, d, K) * keep[:, None, :]).view(N, K).contiguous()
-                pk = bsp.PackedMatrix.allocate(N, K, d, bsp.ORIENT_C, device)
-                bsp.bsp_prune_pack(W, pk, 0.0)
-                plan = torch.empty(bsp.bsp_linear_plan_bytes(N, K, d), dtype=torch.uint8, device=device)
-                bsp.bsp_linear_plan(pk, plan)
-                nz = 2.0 * T * d * kc * (N // d)
-                t_plan = timed(lambda: bsp.bsp_linear_planned(plan, N, K, d, X, bias, act, Y))
-                point = {"sweep": "bert_large", "shape": name, "tokens": T, "n_out": N, "k_in": K, "block": d,
-                         "compression": c, "kept_per_block": kc, "nonzero_gflop": round(nz / 1e9, 2),
-                         "dense_route_ms": round(t_plan, 4), "dense_route_nonzero_tflops": round(nz / t_plan / 1e9, 1),
-                         "torch_dense_ms": round(t_dense, 4), "torch_dense_tflops": round(2.0 * T * N * K / t_dense / 1e9, 1),
-                         "transpose_ms": round(t_tr, 4)}
-                best = nz / t_plan / 1e9
-                if d in (16, 32, 64, 128):
-                    gplan = torch.empty(bsp.bsp_linear_gather_plan_bytes(N, K, d), dtype=torch.uint8, device=device)
-                    bsp.bsp_linear_gather_plan(pk, gplan)
-                    t_g = timed(lambda: bsp.bsp_linear_gathered(gplan, N, K, d, XT, bias, act, Yg))
-                    diff = (Y.float() - Yg.float()).abs().max().item()
-                    point.update({"gather_ms": round(t_g, 4), "gather_nonzero_tflops": round(nz / t_g / 1e9, 1),
-                                  "gather_vs_dense_route": round(t_plan / t_g, 3), "max_abs_diff_between_routes": diff})
-                    best = max(best, nz / t_g / 1e9)
-                    del gplan
-                point["best_percent_of_bf16_peak"] = round(100.0 * best / peak, 2)
-                bsp.bsp_linear_status()
-                print(json.dumps(point), flush=True)
-                del plan, pk, W, keep, scores
+    shapes = args.sweep_shapes.split(",") if args.sweep_shapes else None
+    bert_large_grid(torch.device("cuda", 0), peaks, args.sweep_tokens, max(3, min(args.steps, 20)), shapes,
+                    emit=lambda p: print(json.dumps({"sweep": "bert_large", **p}), flush=True))
 
 
 def main():
@@ -756,6 +995,8 @@ def main():
                     help="time the BERT-large compression x block-height grid and print one JSON line per point")
     ap.add_argument("--sweep-tokens", type=int, default=32768)
     ap.add_argument("--sweep-shapes", default=None, help="comma-separated subset of qkv,attn_out,ffn_up,ffn_down")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="skip the figures of the other workloads (72-matrix stack, DistilBERT-shaped stack, BERT-large grid)")
     args = ap.parse_args()
     if args.sweep:
         run_sweep(args)
@@ -763,8 +1004,27 @@ def main():
         run_case(args)
     elif args.impl == "reference":
         run_reference(args)
+    elif args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        spawn_ranks(args)
     else:
         run_cuda(args)
+
+
+def _rank_main(local_rank, args, port):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), WORLD_SIZE=str(args.gpus),
+                      RANK=str(local_rank), LOCAL_RANK=str(local_rank))
+    run_cuda(args)
+
+
+def spawn_ranks(args):
+    """`python bench.py --gpus N` without a launcher: start the N ranks here, one per GPU (NCCL is only used for
+    the barrier and the max-over-ranks of the times)."""
+    import socket
+    import torch.multiprocessing as mp
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    mp.spawn(_rank_main, args=(args, port), nprocs=args.gpus, join=True)
 
 
 if __name__ == "__main__":

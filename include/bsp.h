@@ -268,6 +268,15 @@ typedef struct bsp_layer_job {
   void* ws; size_t ws_bytes;
 } bsp_layer_job;
 int bsp_prepare_batched(const bsp_layer_job* jobs, int n_jobs, int block, float eps, int pen, void* stream);
+/* bsp_percentile_threshold_batched — bsp_percentile_threshold (Section 3.1's percentile) for the
+ * matrices of a job array in two launches (orientation C): job i's threshold for the target rate
+ * rates[i] (HOST array of n_jobs doubles, each >= 1) is written to the device float that the job
+ * names as threshold_dev, where a following bsp_prepare_batched on the same array reads it.
+ * Uses each job's ws (as bsp_percentile_threshold does); only W, rows, cols, ldw, threshold_dev,
+ * ws and ws_bytes of a job are read.  Results are those of the single-matrix call, bit for bit.
+ * Errors: BSP_ERR_ARG (NULL threshold_dev or ws, rate < 1), BSP_ERR_SHAPE, BSP_ERR_WORKSPACE. */
+int bsp_percentile_threshold_batched(const bsp_layer_job* jobs, int n_jobs, int block, const double* rates,
+                                     void* stream);
 
 /* ---------------------------------------------------------------------------------------------
  * bsp_linear — the pruned linear layer (orientation C packed form):

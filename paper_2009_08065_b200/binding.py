@@ -86,6 +86,7 @@ _SIGNATURES = {
     "bsp_dense_mask": (_i, [_vp, _i, _i, _i, _vp, _i, _vp]),
     "bsp_repack_values": (_i, [_vp, _i, _i, _i, _i, _vp, _vp, _vp, _vp]),
     "bsp_prepare_batched": (_i, [ctypes.POINTER(_LayerJob), _i, _i, _f, _i, _vp]),
+    "bsp_percentile_threshold_batched": (_i, [ctypes.POINTER(_LayerJob), _i, _i, ctypes.POINTER(_d), _vp]),
     "bsp_linear_plan_bytes": (_i, [_i, _i, _i, _szp]),
     "bsp_linear_plan": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _sz, _vp]),
     "bsp_linear_plan_r": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _sz, _vp]),
@@ -270,6 +271,13 @@ def bsp_prepare_batched(jobs, block: int, eps: float = 1e-3, pen: int = PEN_L2, 
     """jobs: a list of LayerJob, or an array made by make_job_array."""
     arr = jobs if isinstance(jobs, ctypes.Array) else make_job_array(jobs)
     _check(lib.bsp_prepare_batched(arr, len(arr), block, eps, pen, _stream(stream)), "bsp_prepare_batched")
+
+
+def bsp_percentile_threshold_batched(jobs, block: int, rates, stream=None) -> None:
+    """Per-matrix percentile thresholds for a job array (each job's threshold_dev tensor receives its threshold)."""
+    arr = jobs if isinstance(jobs, ctypes.Array) else make_job_array(jobs)
+    r = (_d * len(arr))(*[float(v) for v in rates])
+    _check(lib.bsp_percentile_threshold_batched(arr, len(arr), block, r, _stream(stream)), "bsp_percentile_threshold_batched")
 
 
 def bsp_linear_plan_bytes(n_out: int, k_in: int, block: int) -> int:

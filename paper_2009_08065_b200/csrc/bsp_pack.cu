@@ -10,6 +10,7 @@
 // orientation R, with a single-CTA scan between (1) and (2)), the keep-count and percentile
 // kernels, and the entry points.
 #include <mutex>
+#include <new>
 
 #include "bsp_common.cuh"
 
@@ -156,47 +157,103 @@ sumsq_kernel(const uint16_t* __restrict__ W, Geometry G, float* __restrict__ S) 
 }
 
 // r-th smallest (1-based) of n non-negative floats by a 4-pass radix select on their bit
-// patterns (monotone for non-negative floats), one CTA; then the threshold whose float32
-// square is >= that value.
-__global__ void __launch_bounds__(1024)
-select_threshold_kernel(const float* __restrict__ S, long long n, long long r, float* __restrict__ out) {
-  __shared__ unsigned int hist[256];
-  __shared__ unsigned int s_prefix;
-  __shared__ long long s_remaining;
+// patterns (monotone for non-negative floats), one CTA of 1024 threads; then the threshold whose
+// float32 square is >= that value.  Sums of squares of one matrix share their leading byte, so a
+// single shared histogram would serialise on two or three counters: every warp counts into its own
+// 256-bin histogram and the lanes of a warp that hit the same bin add once (match_any).
+__device__ void select_threshold(const float* __restrict__ S, long long n, long long r, float* __restrict__ out,
+                                 unsigned int (*hist)[256], unsigned int* s_prefix, long long* s_remaining) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, n_warps = blockDim.x >> 5;
   if (r <= 0) {
     if (threadIdx.x == 0) *out = -1.0f;
     return;
   }
-  if (threadIdx.x == 0) { s_prefix = 0u; s_remaining = r; }
+  if (threadIdx.x == 0) { *s_prefix = 0u; *s_remaining = r; }
   for (int pass = 3; pass >= 0; --pass) {
-    for (int i = threadIdx.x; i < 256; i += blockDim.x) hist[i] = 0u;
+    for (int i = lane; i < 256; i += 32) hist[warp][i] = 0u;
     __syncthreads();
-    const unsigned int prefix = s_prefix;
+    const unsigned int prefix = *s_prefix;
     const int shift = pass * 8;
     const unsigned int high_mask = pass == 3 ? 0u : (0xffffffffu << (shift + 8));
-    for (long long i = threadIdx.x; i < n; i += blockDim.x) {
-      const unsigned int u = __float_as_uint(S[i]);
-      if ((u & high_mask) == prefix) atomicAdd(&hist[(u >> shift) & 0xffu], 1u);
+    for (long long i0 = 0; i0 < n; i0 += blockDim.x) {
+      const long long i = i0 + threadIdx.x;
+      unsigned int bin = 0xffffffffu;                    // lanes without an element, or outside the prefix, sit out
+      if (i < n) {
+        const unsigned int u = __float_as_uint(S[i]);
+        if ((u & high_mask) == prefix) bin = (u >> shift) & 0xffu;
+      }
+      const unsigned int peers = __match_any_sync(0xffffffffu, bin);
+      if (bin != 0xffffffffu && lane == __ffs(peers) - 1) hist[warp][bin] += static_cast<unsigned int>(__popc(peers));
+    }
+    __syncthreads();
+    if (threadIdx.x < 256) {                             // fold the warps' histograms into the first one
+      unsigned int c = 0;
+      for (int w = 0; w < n_warps; ++w) c += hist[w][threadIdx.x];
+      hist[0][threadIdx.x] = c;
     }
     __syncthreads();
     if (threadIdx.x == 0) {
-      long long rem = s_remaining;
+      long long rem = *s_remaining;
       unsigned int d = 0;
       for (; d < 256; ++d) {
-        if (rem <= static_cast<long long>(hist[d])) break;
-        rem -= hist[d];
+        if (rem <= static_cast<long long>(hist[0][d])) break;
+        rem -= hist[0][d];
       }
-      s_prefix = prefix | (d << shift);
-      s_remaining = rem;
+      *s_prefix = prefix | (d << shift);
+      *s_remaining = rem;
     }
     __syncthreads();
   }
   if (threadIdx.x == 0) {
-    const float s_r = __uint_as_float(s_prefix);
+    const float s_r = __uint_as_float(*s_prefix);
     float t = __fsqrt_rn(s_r);
     while (__fmul_rn(t, t) < s_r) t = __uint_as_float(__float_as_uint(t) + 1u);  // next float up (t >= 0)
     *out = t;
   }
+}
+
+__global__ void __launch_bounds__(1024)
+select_threshold_kernel(const float* __restrict__ S, long long n, long long r, float* __restrict__ out) {
+  __shared__ unsigned int hist[32][256];
+  __shared__ unsigned int s_prefix;
+  __shared__ long long s_remaining;
+  select_threshold(S, n, r, out, hist, &s_prefix, &s_remaining);
+}
+
+// The same for a batch of matrices: sums of squares of every row-block of every matrix in one launch
+// (orientation C, one CTA per row-block), then one selecting CTA per matrix.
+constexpr int kSelectBatch = 96;
+struct SelectJob {
+  const uint16_t* W;
+  int cols, ldw, n_blocks, first_block;
+  float* S;
+  float* out;
+  long long n, r;
+};
+struct SelectBatch {
+  int n_jobs, block;
+  SelectJob job[kSelectBatch];
+};
+__global__ void __launch_bounds__(kPackThreads)
+sumsq_batched_kernel(const __grid_constant__ SelectBatch B) {
+  int lo = 0, hi = B.n_jobs - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (B.job[mid].first_block <= static_cast<int>(blockIdx.x)) lo = mid; else hi = mid - 1;
+  }
+  const SelectJob& J = B.job[lo];
+  const int b = static_cast<int>(blockIdx.x) - J.first_block;
+  const uint16_t* wblk = J.W + static_cast<size_t>(b) * B.block * J.ldw;
+  for (int g = threadIdx.x; g < J.cols; g += blockDim.x)
+    J.S[static_cast<size_t>(b) * J.cols + g] = group_sumsq_strided(wblk + g, B.block, J.ldw);
+}
+__global__ void __launch_bounds__(1024)
+select_threshold_batched_kernel(const __grid_constant__ SelectBatch B) {
+  __shared__ unsigned int hist[32][256];
+  __shared__ unsigned int s_prefix;
+  __shared__ long long s_remaining;
+  const SelectJob& J = B.job[blockIdx.x];
+  select_threshold(J.S, J.n, J.r, J.out, hist, &s_prefix, &s_remaining);
 }
 
 __global__ void __launch_bounds__(256)
@@ -310,6 +367,56 @@ extern "C" int bsp_percentile_threshold(const void* W, int rows, int cols, int l
   select_threshold_kernel<<<1, 1024, 0, s>>>(S, groups, r, threshold_out);
   BSP_LAUNCH_CHECK();
   return BSP_OK;
+}
+
+extern "C" int bsp_percentile_threshold_batched(const bsp_layer_job* jobs, int n_jobs, int block, const double* rates,
+                                                void* stream) {
+  using namespace bsp;
+  if (jobs == nullptr || rates == nullptr || n_jobs <= 0 || block <= 0) return BSP_ERR_ARG;
+  if (n_jobs > 4096) return BSP_ERR_UNSUPPORTED;
+  for (int i = 0; i < n_jobs; ++i) {                       // everything is checked before the first launch
+    const bsp_layer_job& u = jobs[i];
+    int st = check_matrix_args(u.W, u.rows, u.cols, u.ldw, block, BSP_ORIENT_C);
+    if (st != BSP_OK) return st;
+    if (u.threshold_dev == nullptr || u.ws == nullptr || !aligned_to(u.ws, 256)) return BSP_ERR_ARG;
+    if (!(rates[i] >= 1.0)) return BSP_ERR_ARG;
+    if (u.ws_bytes < ws_layout(u.rows / block, u.cols).total) return BSP_ERR_WORKSPACE;
+  }
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  SelectBatch* B = new (std::nothrow) SelectBatch;
+  if (B == nullptr) return BSP_ERR_ARG;
+  int st = BSP_OK;
+  for (int j0 = 0; j0 < n_jobs && st == BSP_OK; j0 += kSelectBatch) {
+    const int n = n_jobs - j0 < kSelectBatch ? n_jobs - j0 : kSelectBatch;
+    B->n_jobs = n;
+    B->block = block;
+    int blocks = 0;
+    for (int i = 0; i < n; ++i) {
+      const bsp_layer_job& u = jobs[j0 + i];
+      const int nb = u.rows / block;
+      const long long groups = static_cast<long long>(nb) * u.cols;
+      SelectJob& J = B->job[i];
+      J.W = static_cast<const uint16_t*>(u.W);
+      J.cols = u.cols;
+      J.ldw = u.ldw;
+      J.n_blocks = nb;
+      J.first_block = blocks;
+      J.S = reinterpret_cast<float*>(static_cast<char*>(u.ws) + ws_layout(nb, u.cols).sumsq_off);
+      J.out = const_cast<float*>(u.threshold_dev);
+      J.n = groups;
+      J.r = static_cast<long long>(static_cast<double>(groups) * (1.0 - 1.0 / rates[j0 + i]));   // as the single-matrix call
+      blocks += nb;
+    }
+    sumsq_batched_kernel<<<blocks, kPackThreads, 0, s>>>(*B);
+    cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess) {
+      select_threshold_batched_kernel<<<n, 1024, 0, s>>>(*B);
+      e = cudaGetLastError();
+    }
+    if (e != cudaSuccess) st = cuda_fail(e);
+  }
+  delete B;
+  return st;
 }
 
 extern "C" int bsp_apply_mask(void* W, int rows, int cols, int ldw, int block, int orient,

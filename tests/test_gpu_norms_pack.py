@@ -417,6 +417,42 @@ def test_prepare_batched_with_device_side_percentile_thresholds():
         assert np.array_equal(plan, O.prune(w, block, "C", t_ref))
 
 
+def test_percentile_thresholds_for_a_batch_of_matrices():
+    """bsp_percentile_threshold_batched: one call finds every matrix's threshold (different rates, a rate of 1 that
+    prunes nothing, heavy ties); the device floats equal the oracle's thresholds and the single-matrix call's, bit
+    for bit, and feed bsp_prepare_batched."""
+    block = 16
+    cases = [((768, 768), 1.79, "t"), ((3072, 768), 3.0, "t"), ((768, 3072), 5.0, "t"), ((256, 512), 1.0, "t"),
+             ((512, 256), 2.0, "ties"), ((64, 72), 8.0, "t")]
+    jobs, refs, rates = [], [], []
+    for n, ((rows, cols), rate, kind) in enumerate(cases):
+        if kind == "ties":            # few distinct values: many groups share the selected sum of squares
+            g = si.stream(700 + n, 1)
+            w = si.f32_to_bf16_bits(g.integers(-2, 3, size=(rows, cols)).astype(np.float32) / 8)
+        else:
+            w = si.student_t_bf16(700 + n, f"pbatch{n}", (rows, cols), 3.0, 0.02)
+        pk = bsp.PackedMatrix.allocate(rows, cols, block, bsp.ORIENT_C, DEV)
+        jobs.append(bsp.LayerJob(W=to_dev(w), out=pk, threshold=0.0,
+                                 threshold_dev=torch.full((1,), 77.0, dtype=torch.float32, device=DEV)))
+        refs.append(w)
+        rates.append(rate)
+    bsp.bsp_percentile_threshold_batched(jobs, block, rates)
+    single = torch.zeros(1, dtype=torch.float32, device=DEV)
+    for job, w, rate in zip(jobs, refs, rates):
+        t_ref = O.percentile_threshold(w, block, "C", rate)
+        assert np.float32(job.threshold_dev.item()) == np.float32(t_ref), (w.shape, rate)
+        bsp.bsp_percentile_threshold(job.W, block, bsp.ORIENT_C, rate, single, job.out.ws)
+        assert torch.equal(single, job.threshold_dev)
+    bsp.bsp_prepare_batched(jobs, block, 1e-3, bsp.PEN_L2)
+    bsp.bsp_linear_status()
+    for job, w, rate in zip(jobs, refs, rates):
+        keep_ref = O.keep_flags(w, block, "C", O.percentile_threshold(w, block, "C", rate))
+        ref_ptr, ref_idx, ref_vals = O.pack(w, keep_ref, block, "C")
+        blk_ptr, idx, vals, keep, kept = packed_to_host(job.out)
+        assert np.array_equal(keep, keep_ref) and np.array_equal(blk_ptr, ref_ptr)
+        assert np.array_equal(idx, ref_idx) and np.array_equal(vals, ref_vals)
+
+
 # ---------------------------------------------------------------------------------------- penalty gradient
 @pytest.mark.parametrize("orient,block,shape", [(0, 16, (768, 768)), (0, 3, (96, 50)), (1, 12, (96, 768)), (1, 5, (33, 50))])
 def test_penalty_gradient(orient, block, shape):
