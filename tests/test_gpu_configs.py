@@ -145,3 +145,42 @@ def test_bert_large_shapes_32768_tokens(name, n, k, act, rate, d):
     # the last, partly filled wave of tiles and the first rows are covered too
     edge = np.concatenate([np.arange(0, 64), np.arange(T - 192, T)])
     check_sampled(spec.name + " edges", x, y, wp, b, act, edge)
+
+
+GRID_SHAPES = [("qkv", 3072, 1024, 0), ("attn_out", 1024, 1024, 0), ("ffn_up", 4096, 1024, 1), ("ffn_down", 1024, 4096, 0)]
+GRID = [(c, d) for d in (8, 16, 32, 64) for c in (1.5, 2.0, 3.0, 5.0, 8.0)]
+
+
+@pytest.mark.parametrize("point", range(len(GRID)))
+def test_bert_large_grid_every_compression_and_block_height(point):
+    """All 20 (compression, block height) pairs of the BERT-large grid at 32768 tokens, the four linear shapes taken in
+    turn, against the oracle on sampled token rows: the zero-expanded route always, the gathering kernel too where
+    the block height allows it.  The activations are drawn on the device; the oracle is fed the bits read back."""
+    c, d = GRID[point]
+    name, n, k, act = GRID_SHAPES[(point + point // 5) % 4]
+    seed, T = si.DEFAULT_SEED + point, 32768
+    spec = si.LinearSpec(f"grid.{name}.c{c:g}.d{d}", n, k, bool(act), c, d)
+    wp, keep = si.make_pruned_weight(seed, spec)
+    b = si.make_bias(seed, spec)
+    gen = torch.Generator(device=DEV)
+    gen.manual_seed(seed)
+    x = torch.randn(T, k, device=DEV, generator=gen).to(torch.bfloat16).view(torch.int16)
+    pk = bsp.PackedMatrix.allocate(n, k, d, bsp.ORIENT_C, DEV)
+    bsp.bsp_prune_pack(to_dev(wp), pk, 0.0)
+    assert int(pk.kept_weights.item()) == d * (n // d) * si.kept_per_block(k, c)
+    rows = np.concatenate([np.arange(0, 8), np.arange(T - 136, T - 128), np.arange(T - 8, T),
+                           np.sort(si.stream(seed, 0x67726964).choice(T, size=72, replace=False))])
+    y = torch.full((T, n), 0x7FC0, dtype=torch.int16, device=DEV)
+    ws = torch.empty(bsp.bsp_linear_plan_bytes(n, k, d), dtype=torch.uint8, device=DEV)
+    bsp.bsp_linear(pk, x, to_dev(b), act, y, ws)
+    bsp.bsp_linear_status()
+    check_sampled(spec.name + " zero-expanded", x, y, wp, b, act, rows)
+    if d in (16, 32, 64):
+        gplan = torch.empty(bsp.bsp_linear_gather_plan_bytes(n, k, d), dtype=torch.uint8, device=DEV)
+        bsp.bsp_linear_gather_plan(pk, gplan)
+        xt = torch.empty((k, T), dtype=torch.int16, device=DEV)
+        bsp.bsp_transpose(x, xt)
+        yg = torch.full((T, n), 0x7FC0, dtype=torch.int16, device=DEV)
+        bsp.bsp_linear_gathered(gplan, n, k, d, xt, to_dev(b), act, yg)
+        bsp.bsp_linear_status()
+        check_sampled(spec.name + " gathered", x, yg, wp, b, act, rows)
