@@ -342,6 +342,12 @@ typedef enum { BSP_LINEAR_AUTO = 0, BSP_LINEAR_ONE_CTA = 1, BSP_LINEAR_CTA_PAIR 
  * the weights are old, only X is fresh).  The one-CTA kernel then starts fetching weight tiles
  * while that work is still finishing.  Never set it when the preceding kernel writes the plan. */
 #define BSP_LINEAR_PLAN_STABLE 0x100
+/* May be OR-ed into `algo`: write the output TRANSPOSED, Y := YT [n_out, tokens] row-major with
+ * leading dimension ldy >= tokens (a multiple of 8), bit for bit the transpose of what the call
+ * writes otherwise.  It is the form bsp_linear_gathered reads its activations in, so a chain of
+ * layers can hand them on without a separate transposing pass.  One-CTA kernel only
+ * (BSP_LINEAR_CTA_PAIR with this flag is BSP_ERR_UNSUPPORTED). */
+#define BSP_LINEAR_OUT_TRANSPOSED 0x200
 int bsp_linear_planned_ex(const void* plan, int n_out, int k_in, int block,
                           const void* X, int tokens, int ldx, const void* bias, int act,
                           void* Y, int ldy, int algo, void* stream);
@@ -425,6 +431,12 @@ int bsp_transpose(const void* X, int rows, int cols, int ldx, void* XT, int ldxt
 int bsp_linear_gathered(const void* gplan, int n_out, int k_in, int block,
                         const void* XT, int tokens, int ldxt, const void* bias, int act,
                         void* Y, int ldy, void* stream);
+/* bsp_linear_gathered_ex — the same; with out_transposed != 0 the output is written as
+ * YT [n_out, tokens] row-major (ldy >= tokens, a multiple of 8), bit for bit the transpose of the
+ * other form: the next gathered layer of a chain reads it as its XT. */
+int bsp_linear_gathered_ex(const void* gplan, int n_out, int k_in, int block,
+                           const void* XT, int tokens, int ldxt, const void* bias, int act,
+                           void* Y, int ldy, int out_transposed, void* stream);
 
 /* bsp_linear_cuda_core — the same layer computed straight from the packed form by a plain
  * CUDA-core kernel (one thread per output, float32 accumulation in index order).  It is what

@@ -82,6 +82,7 @@ _SIGNATURES = {
     "bsp_linear_gather_plan": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _sz, _vp]),
     "bsp_transpose": (_i, [_vp, _i, _i, _i, _vp, _i, _vp]),
     "bsp_linear_gathered": (_i, [_vp, _i, _i, _i, _vp, _i, _i, _vp, _i, _vp, _i, _vp]),
+    "bsp_linear_gathered_ex": (_i, [_vp, _i, _i, _i, _vp, _i, _i, _vp, _i, _vp, _i, _i, _vp]),
     "bsp_masked_adam_step": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _vp, _i, _i, _f, _f, _f, _f, _f, _i, _vp, _i, _vp]),
     "bsp_dense_mask": (_i, [_vp, _i, _i, _i, _vp, _i, _vp]),
     "bsp_repack_values": (_i, [_vp, _i, _i, _i, _i, _vp, _vp, _vp, _vp]),
@@ -320,6 +321,7 @@ def bsp_linear_planned(plan: torch.Tensor, n_out: int, k_in: int, block: int, X:
 
 LINEAR_AUTO, LINEAR_ONE_CTA, LINEAR_CTA_PAIR = 0, 1, 2
 LINEAR_PLAN_STABLE = 0x100     # OR into `algo`: the plan is older than the previous kernel in the stream
+LINEAR_OUT_TRANSPOSED = 0x200  # OR into `algo`: Y is written as [n_out, tokens]
 
 
 def bsp_linear_planned_ex(plan: torch.Tensor, n_out: int, k_in: int, block: int, X: torch.Tensor,
@@ -381,6 +383,14 @@ def bsp_linear_gathered(gplan: torch.Tensor, n_out: int, k_in: int, block: int, 
     """XT is [k_in, tokens] (the transposed activations); Y is [tokens, n_out]."""
     _check(lib.bsp_linear_gathered(_ptr(gplan), n_out, k_in, block, _ptr(XT), XT.shape[1], _ld(XT), _ptr(bias), act,
                                    _ptr(Y), _ld(Y), _stream(stream)), "bsp_linear_gathered")
+
+
+def bsp_linear_gathered_ex(gplan: torch.Tensor, n_out: int, k_in: int, block: int, XT: torch.Tensor,
+                           bias: Optional[torch.Tensor], act: int, Y: torch.Tensor, out_transposed: bool = False,
+                           stream=None) -> None:
+    """As bsp_linear_gathered; with out_transposed the output tensor is [n_out, tokens]."""
+    _check(lib.bsp_linear_gathered_ex(_ptr(gplan), n_out, k_in, block, _ptr(XT), XT.shape[1], _ld(XT), _ptr(bias), act,
+                                      _ptr(Y), _ld(Y), int(out_transposed), _stream(stream)), "bsp_linear_gathered_ex")
 
 
 @dataclass

@@ -183,6 +183,7 @@ struct GatherParams {
   const uint16_t* bias;
   uint16_t* Y;
   int ldy;
+  int transposed;            // Y is [n_out, tokens] (leading dimension ldy spans the tokens)
   const int32_t* soff;
   const uint8_t* meta;
   const int16_t* cols;
@@ -420,7 +421,19 @@ linear_gather_kernel(const __grid_constant__ CUtensorMap map_xt, const __grid_co
 #pragma unroll
             for (int i = 0; i < 16; ++i) f[i] = gelu_erf(f[i]);
           }
-          if (t < P.tokens) {
+          if (P.transposed) {
+            // output row n = rb * D + c0 + i holds this thread's token in column t: the 32 lanes of a warp
+            // write 64 contiguous bytes per output row
+            if (t < P.tokens) {
+              uint16_t* col = P.Y + (static_cast<size_t>(rb) * D + c0) * P.ldy + t;
+#pragma unroll
+              for (int i = 0; i < 8; ++i) {
+                const uint32_t w = pack_bf16x2(f[2 * i], f[2 * i + 1]);
+                col[static_cast<size_t>(2 * i) * P.ldy] = static_cast<uint16_t>(w & 0xffffu);
+                col[static_cast<size_t>(2 * i + 1) * P.ldy] = static_cast<uint16_t>(w >> 16);
+              }
+            }
+          } else if (t < P.tokens) {
             uint4* out = reinterpret_cast<uint4*>(yrow + static_cast<size_t>(rb) * D + c0);
             out[0] = make_uint4(pack_bf16x2(f[0], f[1]), pack_bf16x2(f[2], f[3]), pack_bf16x2(f[4], f[5]), pack_bf16x2(f[6], f[7]));
             out[1] = make_uint4(pack_bf16x2(f[8], f[9]), pack_bf16x2(f[10], f[11]), pack_bf16x2(f[12], f[13]), pack_bf16x2(f[14], f[15]));
@@ -520,12 +533,18 @@ extern "C" int bsp_transpose(const void* X, int rows, int cols, int ldx, void* X
 
 extern "C" int bsp_linear_gathered(const void* gplan, int n_out, int k_in, int block, const void* XT, int tokens,
                                    int ldxt, const void* bias, int act, void* Y, int ldy, void* stream) {
+  return bsp_linear_gathered_ex(gplan, n_out, k_in, block, XT, tokens, ldxt, bias, act, Y, ldy, 0, stream);
+}
+
+extern "C" int bsp_linear_gathered_ex(const void* gplan, int n_out, int k_in, int block, const void* XT, int tokens,
+                                      int ldxt, const void* bias, int act, void* Y, int ldy, int out_transposed,
+                                      void* stream) {
   using namespace bsp;
   if (gplan == nullptr || XT == nullptr || Y == nullptr) return BSP_ERR_ARG;
   if (n_out <= 0 || k_in <= 0 || block <= 0 || tokens < 0) return BSP_ERR_ARG;
   if (act != BSP_ACT_NONE && act != BSP_ACT_GELU) return BSP_ERR_ARG;
   if (n_out % block) return BSP_ERR_SHAPE;
-  if (ldxt < tokens || ldy < n_out) return BSP_ERR_SHAPE;
+  if (ldxt < tokens || ldy < (out_transposed ? tokens : n_out)) return BSP_ERR_SHAPE;
   if (!gather_block_ok(block) || k_in > 32767) return BSP_ERR_UNSUPPORTED;
   if (!aligned_to(gplan, 256) || !aligned_to(XT, 16) || !aligned_to(Y, 16) || (bias != nullptr && !aligned_to(bias, 16)) ||
       tokens % 8 || ldxt % 8 || ldy % 8)
@@ -545,6 +564,7 @@ extern "C" int bsp_linear_gathered(const void* gplan, int n_out, int k_in, int b
   P.bias = static_cast<const uint16_t*>(bias);
   P.Y = static_cast<uint16_t*>(Y);
   P.ldy = ldy;
+  P.transposed = out_transposed ? 1 : 0;
   P.soff = reinterpret_cast<const int32_t*>(base + L.soff_off);
   P.meta = reinterpret_cast<const uint8_t*>(base + L.meta_off);
   P.cols = reinterpret_cast<const int16_t*>(base + L.cols_off);

@@ -51,6 +51,7 @@ __device__ __align__(16) int g_linear_status[8];
 struct LinearParams {
   int tokens, n_out, k_in, act;
   int plan_stable;      // the plan was complete before the kernel preceding this one in the stream began
+  int transposed;       // the output is written as [n_out, tokens] (map_y describes that matrix)
   const uint16_t* bias;
   int* status;
 };
@@ -223,11 +224,14 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
           if (lane == 0) mbar_arrive(acc_empty_bar(acc));
           released = true;
         }
-        piece_store(piece, P.act, buf + row_off, row_xor);
+        if (P.transposed) piece_store_transposed(piece, P.act, buf, row);
+        else piece_store(piece, P.act, buf + row_off, row_xor);
         fence_async_smem();                  // make the staged piece visible to the TMA engine
         group_sync(group);
         if (issuer) {
-          tma_store_2d(&map_y, n0 + c0, m0, buf);   // rows beyond `tokens` / columns beyond `n_out` are clipped
+          // rows beyond `tokens` / columns beyond `n_out` are clipped by the tensor map
+          if (P.transposed) tma_store_2d(&map_y, m0, n0 + c0, buf);
+          else tma_store_2d(&map_y, n0 + c0, m0, buf);
           tma_store_commit();
         }
       }
@@ -392,7 +396,11 @@ int launch_tc(TcDevice* dev, int slot, const void* plan, const void* X, void* Y,
   CUtensorMap map_x, map_w, map_y;
   if (!make_map(&map_x, X, P.k_in, P.tokens, ldx, kBlockM)) return BSP_ERR_CUDA;
   if (!make_map(&map_w, plan, P.k_in, P.n_out, P.k_in, BN)) return BSP_ERR_CUDA;
-  if (!make_map(&map_y, Y, P.n_out, P.tokens, ldy, kBlockM, kEpiCols)) return BSP_ERR_CUDA;
+  if (P.transposed) {     // Y is [n_out, tokens]: pieces of 32 output rows x 128 tokens
+    if (!make_map(&map_y, Y, P.tokens, P.n_out, ldy, kEpiCols, kBlockM)) return BSP_ERR_CUDA;
+  } else if (!make_map(&map_y, Y, P.n_out, P.tokens, ldy, kBlockM, kEpiCols)) {
+    return BSP_ERR_CUDA;
+  }
   if (!dev->attr_set[slot]) {
     BSP_CUDA_TRY(cudaFuncSetAttribute(linear_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes));
     dev->attr_set[slot] = true;
@@ -508,11 +516,16 @@ extern "C" int bsp_linear_plan_t(const int32_t* blk_ptr, const int32_t* idx, con
 extern "C" int bsp_linear_planned_ex(const void* plan, int n_out, int k_in, int block, const void* X, int tokens,
                                      int ldx, const void* bias, int act, void* Y, int ldy, int algo, void* stream) {
   using namespace bsp;
-  int st = check_linear_args(plan, plan, plan, n_out, k_in, block, X, tokens, ldx, act, Y, ldy);
-  if (st != BSP_OK) return st;
   const int algo_flags = algo & ~0xff;
   algo &= 0xff;
-  if (algo < BSP_LINEAR_AUTO || algo > BSP_LINEAR_CTA_PAIR || (algo_flags & ~BSP_LINEAR_PLAN_STABLE)) return BSP_ERR_ARG;
+  if (algo < BSP_LINEAR_AUTO || algo > BSP_LINEAR_CTA_PAIR || (algo_flags & ~(BSP_LINEAR_PLAN_STABLE | BSP_LINEAR_OUT_TRANSPOSED)))
+    return BSP_ERR_ARG;
+  const bool transposed = (algo_flags & BSP_LINEAR_OUT_TRANSPOSED) != 0;
+  if (transposed && algo == BSP_LINEAR_CTA_PAIR) return BSP_ERR_UNSUPPORTED;     // only the one-CTA kernel writes transposed
+  // (a transposed output is [n_out, tokens]: its leading dimension spans the tokens)
+  int st = check_linear_args(plan, plan, plan, n_out, k_in, block, X, tokens, ldx, act, Y, transposed ? n_out : ldy);
+  if (st != BSP_OK) return st;
+  if (transposed && ldy < tokens) return BSP_ERR_SHAPE;
   if (!tc_path_ok(plan, n_out, k_in, X, ldx, Y, ldy)) return BSP_ERR_UNSUPPORTED;
   if (tokens == 0) return BSP_OK;
   TcDevice* dev = tc_device();
@@ -524,9 +537,9 @@ extern "C" int bsp_linear_planned_ex(const void* plan, int n_out, int k_in, int 
   // With GELU the epilogue is the longer side of a tile and the one-CTA kernel's slower main loop hides
   // more of it: 202 us against 209 us at 32768 x 4096 x 1024.
   const bool pair = algo == BSP_LINEAR_CTA_PAIR ||
-                    (algo == BSP_LINEAR_AUTO && pair_tiles >= 4LL * dev->sms && act == BSP_ACT_NONE);
+                    (algo == BSP_LINEAR_AUTO && pair_tiles >= 4LL * dev->sms && act == BSP_ACT_NONE && !transposed);
   if (pair) return launch_tc_pair(dev, plan, X, Y, tokens, n_out, k_in, act, bias, ldx, ldy, s);
-  LinearParams P{tokens, n_out, k_in, act, (algo_flags & BSP_LINEAR_PLAN_STABLE) ? 1 : 0,
+  LinearParams P{tokens, n_out, k_in, act, (algo_flags & BSP_LINEAR_PLAN_STABLE) ? 1 : 0, transposed ? 1 : 0,
                  static_cast<const uint16_t*>(bias), dev->status};
   switch (choose_bn(tokens, n_out, dev->sms)) {
     case 256: return launch_tc<256>(dev, 0, plan, X, Y, P, ldx, ldy, s);

@@ -274,6 +274,33 @@ __device__ __forceinline__ void piece_store(const EpiloguePiece& p, int act, uin
                  pack_bf16x2(f[4], f[5]), pack_bf16x2(f[6], f[7]));
   }
 }
+// The same piece for a TRANSPOSED output [n_out, tokens]: the staging buffer is 32 output rows of 128
+// tokens (256 bytes each, no swizzle); this thread's token is column `row`, so the 32 lanes of a warp
+// write 64 contiguous bytes per output row.
+__device__ __forceinline__ void piece_store_transposed(const EpiloguePiece& p, int act, uint32_t buf, int row) {
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const uint32_t* v = &p.v[j * 8];
+    const uint32_t bw[4] = {p.bias[j].x, p.bias[j].y, p.bias[j].z, p.bias[j].w};
+    float f[8];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      f[2 * i] = __uint_as_float(v[2 * i]) + __uint_as_float(bw[i] << 16);
+      f[2 * i + 1] = __uint_as_float(v[2 * i + 1]) + __uint_as_float(bw[i] & 0xffff0000u);
+    }
+    if (act == BSP_ACT_GELU) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) f[i] = gelu_erf(f[i]);
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const uint32_t w = pack_bf16x2(f[2 * i], f[2 * i + 1]);
+      const uint32_t a = buf + static_cast<uint32_t>((j * 8 + 2 * i) * 256 + row * 2);
+      asm volatile("st.shared.b16 [%0], %1;" ::"r"(a), "h"(static_cast<uint16_t>(w & 0xffffu)));
+      asm volatile("st.shared.b16 [%0], %1;" ::"r"(a + 256u), "h"(static_cast<uint16_t>(w >> 16)));
+    }
+  }
+}
 #endif  // __CUDACC__
 
 // ------------------------------------------------------------------------------------------
@@ -300,6 +327,7 @@ inline EncodeTiledFn encode_tiled_fn() {
 // 2-D bf16 tensor [outer, inner] row-major with leading dimension ld; box [box_outer, box_inner]:
 // 64 columns with the 128-byte swizzle (operand tiles) or 32 columns with the 64-byte swizzle
 // (epilogue pieces); out-of-range elements read as zero and are not written.
+// A box of 128 columns is stored without a swizzle (the staging buffer of a transposed output piece).
 inline bool make_map(CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer, uint64_t ld, uint32_t box_outer,
                      uint32_t box_inner = 64, CUtensorMapL2promotion promote = CU_TENSOR_MAP_L2_PROMOTION_L2_256B) {
   EncodeTiledFn fn = encode_tiled_fn();
@@ -309,7 +337,8 @@ inline bool make_map(CUtensorMap* map, const void* base, uint64_t inner, uint64_
   const cuuint32_t box[2] = {box_inner, box_outer};
   const cuuint32_t elem[2] = {1, 1};
   return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, elem,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, box_inner == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B, promote,
+            CU_TENSOR_MAP_INTERLEAVE_NONE,
+            box_inner == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : box_inner == 32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE, promote,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 

@@ -172,3 +172,67 @@ def test_gelu_epilogue_is_tight_on_both_routes():
         assert (np.abs(got - ref_r) <= ulp_of_ref + 2.6e-6).all(), name
         big = np.abs(ref_r) > 1e-3                                  # where the absolute term is far below an ulp
         assert (got_bits[big] == ref_bits[big]).mean() > 0.99, (name, float((got_bits[big] == ref_bits[big]).mean()))
+
+
+@pytest.mark.parametrize("act", [0, 1])
+@pytest.mark.parametrize("T,N,K,d", [(328, 512, 712, 32), (1000, 200, 256, 8), (4096, 768, 768, 16)])
+def test_transposed_output_is_the_transpose_bit_for_bit(T, N, K, d, act):
+    """BSP_LINEAR_OUT_TRANSPOSED on the zero-expanded route and out_transposed on the gathering kernel: YT [n_out, tokens]
+    holds exactly the bits of Y^T (ragged token tiles and output tiles included), nothing outside it is written."""
+    spec = si.LinearSpec(f"tr_out{T}_{N}_{d}", N, K, bool(act), 3.0, d)
+    wp, _ = si.make_pruned_weight(43, spec)
+    x = to_dev(si.make_activations(43, spec.name, T, K))
+    b = to_dev(si.make_bias(43, spec))
+    W = to_dev(wp)                                        # zero where pruned: its own execution layout
+    y = torch.full((T, N), 0x7FC0, dtype=torch.int16, device=DEV)
+    ld = (T + 7) // 8 * 8 + 8                             # a leading dimension wider than the tokens
+    yt = torch.full((N, ld), 0x7FC0, dtype=torch.int16, device=DEV)
+    bsp.bsp_linear_planned_ex(W, N, K, d, x, b, act, y, bsp.LINEAR_ONE_CTA)
+    bsp.bsp_linear_planned_ex(W, N, K, d, x, b, act, yt[:, :T], bsp.LINEAR_ONE_CTA | bsp.LINEAR_OUT_TRANSPOSED)
+    bsp.bsp_linear_status()
+    assert torch.equal(yt[:, :T], y.t())
+    assert bool((yt[:, T:] == 0x7FC0).all())              # the padding columns keep their pattern
+    with pytest.raises(bsp.BspError) as e:
+        bsp.bsp_linear_planned_ex(W, N, K, d, x, b, act, yt[:, :T], bsp.LINEAR_CTA_PAIR | bsp.LINEAR_OUT_TRANSPOSED)
+    assert e.value.status == -6
+    if d in (16, 32) and T % 8 == 0:
+        pk = bsp.PackedMatrix.allocate(N, K, d, bsp.ORIENT_C, DEV)
+        bsp.bsp_prune_pack(W, pk, 0.0)
+        gplan = torch.empty(bsp.bsp_linear_gather_plan_bytes(N, K, d), dtype=torch.uint8, device=DEV)
+        bsp.bsp_linear_gather_plan(pk, gplan)
+        xt = torch.empty((K, T), dtype=torch.int16, device=DEV)
+        bsp.bsp_transpose(x, xt)
+        yg = torch.full((T, N), 0x7FC0, dtype=torch.int16, device=DEV)
+        ygt = torch.full((N, ld), 0x7FC0, dtype=torch.int16, device=DEV)
+        bsp.bsp_linear_gathered(gplan, N, K, d, xt, b, act, yg)
+        bsp.bsp_linear_gathered_ex(gplan, N, K, d, xt, b, act, ygt[:, :T], True)
+        bsp.bsp_linear_status()
+        assert torch.equal(ygt[:, :T], yg.t())
+        assert bool((ygt[:, T:] == 0x7FC0).all())
+
+
+def test_chain_hands_transposed_activations_on_without_a_transposing_pass():
+    """Two layers with 64-row blocks at 8x: the first (zero-expanded route) writes its output transposed, the second
+    (gathering kernel) reads that as its XT and writes transposed again; each layer is checked against the oracle on
+    the bf16 input it consumed."""
+    T, H, F, d, rate = 1024, 512, 1024, 64, 8.0
+    s1 = si.LinearSpec("chain_t.up", F, H, True, rate, d)
+    s2 = si.LinearSpec("chain_t.down", H, F, False, rate, d)
+    w1, _ = si.make_pruned_weight(47, s1)
+    w2, _ = si.make_pruned_weight(47, s2)
+    b1, b2 = si.make_bias(47, s1), si.make_bias(47, s2)
+    x = si.make_activations(47, "chain_t", T, H)
+    h_t = torch.full((F, T), 0x7FC0, dtype=torch.int16, device=DEV)
+    bsp.bsp_linear_planned_ex(to_dev(w1), F, H, d, to_dev(x), to_dev(b1), 1, h_t, bsp.LINEAR_OUT_TRANSPOSED)
+    pk = bsp.PackedMatrix.allocate(H, F, d, bsp.ORIENT_C, DEV)
+    bsp.bsp_prune_pack(to_dev(w2), pk, 0.0)
+    gplan = torch.empty(bsp.bsp_linear_gather_plan_bytes(H, F, d), dtype=torch.uint8, device=DEV)
+    bsp.bsp_linear_gather_plan(pk, gplan)
+    y_t = torch.full((H, T), 0x7FC0, dtype=torch.int16, device=DEV)
+    bsp.bsp_linear_gathered_ex(gplan, H, F, d, h_t, to_dev(b2), 0, y_t, True)
+    bsp.bsp_linear_status()
+    h = np.ascontiguousarray(bits_of(h_t).T)
+    ref1, sc1 = oracle_linear(x, w1, b1, 1)
+    assert_linear_close(h, ref1, sc1, "first layer, transposed output")
+    ref2, sc2 = oracle_linear(h, w2, b2, 0)
+    assert_linear_close(np.ascontiguousarray(bits_of(y_t).T), ref2, sc2, "second layer, gathered from the transposed output")
