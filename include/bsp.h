@@ -438,6 +438,46 @@ int bsp_linear_gathered_ex(const void* gplan, int n_out, int k_in, int block,
                            const void* XT, int tokens, int ldxt, const void* bias, int act,
                            void* Y, int ldy, int out_transposed, void* stream);
 
+/* ---------------------------------------------------------------------------------------------
+ * bsp_linear_route / bsp_linear_run / bsp_linear_tune — one call for the pruned linear layer
+ * (Sections 3.1 / 4.4) over both routes: the zero-expanded one (bsp_linear_planned_ex) and the
+ * gathering one (bsp_linear_gathered_ex).  The caller states what it has in a bsp_linear_call:
+ *   plan / gplan      the weights' execution layouts (either may be NULL);
+ *   kept_weights      host copy of the packed matrix's kept-weight count, or -1 (unknown: the
+ *                     estimate then assumes nothing was pruned);
+ *   X, ldx / XT, ldxt the activations, row-major [tokens, k_in] and/or transposed [k_in, tokens];
+ *   Y, ldy / YT, ldyt where the output goes: exactly one of the two (YT = [n_out, tokens]);
+ *   plan_stable       as BSP_LINEAR_PLAN_STABLE.
+ * A route is possible when its weight layout and its activation layout are both given (zero-expanded:
+ * plan and X; gathering: gplan and XT, block in {16, 32, 64, 128}).
+ *   bsp_linear_route  host-only: the route BSP_ROUTE_AUTO would take.  With both possible it compares
+ *                     estimates fitted to measurements on B200 (dense product at the zero-expanded
+ *                     kernel's rate, against 0.62 us per 64 kept columns and 0.45 us per row-block per
+ *                     128-token tile on every SM), which are good to about 10 %.
+ *   bsp_linear_run    runs `route` (or the automatic choice) and reports it in *route_taken (may be NULL).
+ *   bsp_linear_tune   times every possible route on the caller's own buffers (one untimed launch, then
+ *                     `reps` timed ones per route; the outputs are written) and returns the faster one and
+ *                     both times in milliseconds (-1 for a route that is not possible).  Synchronises the
+ *                     stream; not for use during stream capture.
+ * Errors: BSP_ERR_ARG (no possible route, both or neither output, bad route), BSP_ERR_SHAPE, and
+ * whatever the chosen route's own call returns. */
+typedef enum { BSP_ROUTE_AUTO = 0, BSP_ROUTE_ZERO_EXPANDED = 1, BSP_ROUTE_GATHERED = 2 } bsp_route;
+typedef struct bsp_linear_call {
+  const void* plan; const void* gplan; long long kept_weights;
+  int n_out, k_in, block;
+  const void* X; int ldx;
+  const void* XT; int ldxt;
+  int tokens;
+  const void* bias; int act;
+  void* Y; int ldy;
+  void* YT; int ldyt;
+  int plan_stable;
+} bsp_linear_call;
+int bsp_linear_route(const bsp_linear_call* call, int* route);
+int bsp_linear_run(const bsp_linear_call* call, int route, int* route_taken, void* stream);
+int bsp_linear_tune(const bsp_linear_call* call, int reps, int* best_route, float* ms_zero_expanded,
+                    float* ms_gathered, void* stream);
+
 /* bsp_linear_cuda_core — the same layer computed straight from the packed form by a plain
  * CUDA-core kernel (one thread per output, float32 accumulation in index order).  It is what
  * bsp_linear falls back to when the alignment rules above do not hold, and is exported so the

@@ -15,4 +15,5 @@ from .binding import (  # noqa: F401
     bsp_linear_gather_plan_bytes, bsp_linear_gather_plan, bsp_transpose, bsp_linear_gathered,
     bsp_masked_adam_step, bsp_repack_values, bsp_dense_mask,
     bsp_linear_cuda_core, bsp_status_string, bsp_set_wait_limit_ms, bsp_wait_selftest,
+    ROUTE_AUTO, ROUTE_ZERO_EXPANDED, ROUTE_GATHERED, make_linear_call, bsp_linear_route, bsp_linear_run, bsp_linear_tune,
 )

@@ -67,6 +67,18 @@ class _ChainOp(ctypes.Structure):
     ]
 
 
+class _LinearCall(ctypes.Structure):
+    """Mirror of `bsp_linear_call` in bsp.h."""
+    _fields_ = [
+        ("plan", _vp), ("gplan", _vp), ("kept_weights", ctypes.c_longlong),
+        ("n_out", _i), ("k_in", _i), ("block", _i),
+        ("X", _vp), ("ldx", _i), ("XT", _vp), ("ldxt", _i), ("tokens", _i),
+        ("bias", _vp), ("act", _i),
+        ("Y", _vp), ("ldy", _i), ("YT", _vp), ("ldyt", _i),
+        ("plan_stable", _i),
+    ]
+
+
 _SIGNATURES = {
     "bsp_status_string": (ctypes.c_char_p, [_i]),
     "bsp_last_cuda_error": (_i, []),
@@ -98,6 +110,9 @@ _SIGNATURES = {
     "bsp_linear": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _i, _i, _vp, _i, _vp, _i, _vp, _sz, _vp]),
     "bsp_linear_chain_ws_bytes": (_i, [_i, _i, _szp]),
     "bsp_linear_chain": (_i, [ctypes.POINTER(_ChainOp), _i, _vp, _i, _i, _vp, _sz, _vp]),
+    "bsp_linear_route": (_i, [ctypes.POINTER(_LinearCall), ctypes.POINTER(_i)]),
+    "bsp_linear_run": (_i, [ctypes.POINTER(_LinearCall), _i, ctypes.POINTER(_i), _vp]),
+    "bsp_linear_tune": (_i, [ctypes.POINTER(_LinearCall), _i, ctypes.POINTER(_i), ctypes.POINTER(_f), ctypes.POINTER(_f), _vp]),
     "bsp_linear_status": (_i, [_vp]),
     "bsp_set_wait_limit_ms": (_i, [_i]),
     "bsp_wait_selftest": (_i, [ctypes.POINTER(_i), ctypes.POINTER(ctypes.c_longlong), _vp]),
@@ -454,3 +469,44 @@ def bsp_wait_selftest(stream=None) -> Tuple[int, int]:
     n, ns = ctypes.c_int(0), ctypes.c_longlong(0)
     _check(lib.bsp_wait_selftest(ctypes.byref(n), ctypes.byref(ns), _stream(stream)), "bsp_wait_selftest")
     return n.value, ns.value
+
+
+ROUTE_AUTO, ROUTE_ZERO_EXPANDED, ROUTE_GATHERED = 0, 1, 2
+
+
+def make_linear_call(n_out: int, k_in: int, block: int, tokens: int, plan: Optional[torch.Tensor] = None,
+                     gplan: Optional[torch.Tensor] = None, kept_weights: int = -1, X: Optional[torch.Tensor] = None,
+                     XT: Optional[torch.Tensor] = None, bias: Optional[torch.Tensor] = None, act: int = ACT_NONE,
+                     Y: Optional[torch.Tensor] = None, YT: Optional[torch.Tensor] = None, plan_stable: bool = False):
+    """The descriptor of bsp_linear_route / bsp_linear_run / bsp_linear_tune (tensors as in the per-route calls)."""
+    c = _LinearCall()
+    c.plan, c.gplan, c.kept_weights = _ptr(plan), _ptr(gplan), int(kept_weights)
+    c.n_out, c.k_in, c.block, c.tokens = n_out, k_in, block, tokens
+    c.X, c.ldx = _ptr(X), 0 if X is None else _ld(X)
+    c.XT, c.ldxt = _ptr(XT), 0 if XT is None else _ld(XT)
+    c.bias, c.act = _ptr(bias), act
+    c.Y, c.ldy = _ptr(Y), 0 if Y is None else _ld(Y)
+    c.YT, c.ldyt = _ptr(YT), 0 if YT is None else _ld(YT)
+    c.plan_stable = int(plan_stable)
+    return c
+
+
+def bsp_linear_route(call) -> int:
+    r = _i(0)
+    _check(lib.bsp_linear_route(ctypes.byref(call), ctypes.byref(r)), "bsp_linear_route")
+    return r.value
+
+
+def bsp_linear_run(call, route: int = ROUTE_AUTO, stream=None) -> int:
+    """Runs the layer; returns the route taken (ROUTE_ZERO_EXPANDED or ROUTE_GATHERED)."""
+    r = _i(0)
+    _check(lib.bsp_linear_run(ctypes.byref(call), route, ctypes.byref(r), _stream(stream)), "bsp_linear_run")
+    return r.value
+
+
+def bsp_linear_tune(call, reps: int = 3, stream=None) -> Tuple[int, float, float]:
+    """(faster route, ms of the zero-expanded route, ms of the gathering route); -1 for a route that is not possible."""
+    r, a, b = _i(0), _f(0.0), _f(0.0)
+    _check(lib.bsp_linear_tune(ctypes.byref(call), reps, ctypes.byref(r), ctypes.byref(a), ctypes.byref(b), _stream(stream)),
+           "bsp_linear_tune")
+    return r.value, a.value, b.value

@@ -179,3 +179,40 @@ def test_product_code_does_not_touch_the_oracle():
                 src = open(os.path.join(dirpath, f)).read()
                 assert "oracle" not in src, f"{f} mentions the oracle"
     assert "paper_2009_08065_b200" not in open(os.path.join(ROOT, "oracle", "bsp_oracle.py")).read()
+
+
+def _fake_call(n, k, d, c, tokens=32768, act=0, z=True, g=True):
+    p = ctypes.c_void_p(0x1000).value
+    call = binding._LinearCall()
+    call.plan, call.gplan = (p if z else None), (p if g else None)
+    call.kept_weights = int(round(k / c)) * n
+    call.n_out, call.k_in, call.block, call.tokens = n, k, d, tokens
+    call.X, call.ldx, call.XT, call.ldxt = (p if z else None), k, (p if g else None), tokens
+    call.act = act
+    call.Y, call.ldy = p, n
+    return call
+
+
+def test_route_choice_follows_the_measured_crossovers():
+    """bsp_linear_route is host-only: with both routes possible it takes the gathering kernel where it was measured
+    to win on B200 (64-row blocks at 8x on the FFN shapes) and the zero-expanded route elsewhere."""
+    lib = bsp.lib
+    assert bsp.bsp_linear_route(_fake_call(1024, 4096, 64, 8.0)) == bsp.ROUTE_GATHERED             # FFN-down
+    assert bsp.bsp_linear_route(_fake_call(4096, 1024, 64, 8.0, act=1)) == bsp.ROUTE_GATHERED      # FFN-up + GELU
+    assert bsp.bsp_linear_route(_fake_call(3072, 1024, 64, 8.0)) == bsp.ROUTE_ZERO_EXPANDED        # QKV
+    assert bsp.bsp_linear_route(_fake_call(1024, 4096, 64, 5.0)) == bsp.ROUTE_ZERO_EXPANDED
+    assert bsp.bsp_linear_route(_fake_call(1024, 4096, 32, 8.0)) == bsp.ROUTE_ZERO_EXPANDED
+    assert bsp.bsp_linear_route(_fake_call(2304, 768, 16, 3.0, tokens=4096)) == bsp.ROUTE_ZERO_EXPANDED
+    # only one route possible: that one, whatever the estimate says
+    assert bsp.bsp_linear_route(_fake_call(2304, 768, 16, 3.0, z=False)) == bsp.ROUTE_GATHERED
+    assert bsp.bsp_linear_route(_fake_call(1024, 4096, 64, 8.0, g=False)) == bsp.ROUTE_ZERO_EXPANDED
+    assert bsp.bsp_linear_route(_fake_call(1024, 4096, 8, 8.0)) == bsp.ROUTE_ZERO_EXPANDED         # block 8: no gathering kernel
+    bad = _fake_call(1024, 4096, 64, 8.0)
+    bad.YT, bad.ldyt = bad.Y, 32768                                                                # both outputs
+    assert lib.bsp_linear_route(ctypes.byref(bad), ctypes.byref(ctypes.c_int())) == -1
+    none = _fake_call(1024, 4096, 64, 8.0)
+    none.X = None                                                                                  # plan without X, gplan with XT
+    assert bsp.bsp_linear_route(none) == bsp.ROUTE_GATHERED
+    none.XT = None
+    assert lib.bsp_linear_route(ctypes.byref(none), ctypes.byref(ctypes.c_int())) == -1
+    assert lib.bsp_linear_run(ctypes.byref(_fake_call(1024, 4096, 64, 8.0)), 7, None, None) == -1

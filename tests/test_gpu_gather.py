@@ -236,3 +236,47 @@ def test_chain_hands_transposed_activations_on_without_a_transposing_pass():
     assert_linear_close(h, ref1, sc1, "first layer, transposed output")
     ref2, sc2 = oracle_linear(h, w2, b2, 0)
     assert_linear_close(np.ascontiguousarray(bits_of(y_t).T), ref2, sc2, "second layer, gathered from the transposed output")
+
+
+def test_one_call_over_both_routes_run_and_tune():
+    """bsp_linear_run takes the route it is told, or chooses one, and reports it; both routes and both output layouts
+    give the bits of the per-route calls; bsp_linear_tune times the possible routes and names the faster."""
+    T, N, K, d, rate = 2048, 512, 2048, 64, 8.0
+    spec = si.LinearSpec("front_door", N, K, False, rate, d)
+    wp, _ = si.make_pruned_weight(53, spec)
+    x = to_dev(si.make_activations(53, spec.name, T, K))
+    b = to_dev(si.make_bias(53, spec))
+    W = to_dev(wp)
+    pk = bsp.PackedMatrix.allocate(N, K, d, bsp.ORIENT_C, DEV)
+    bsp.bsp_prune_pack(W, pk, 0.0)
+    gplan = torch.empty(bsp.bsp_linear_gather_plan_bytes(N, K, d), dtype=torch.uint8, device=DEV)
+    bsp.bsp_linear_gather_plan(pk, gplan)
+    xt = torch.empty((K, T), dtype=torch.int16, device=DEV)
+    bsp.bsp_transpose(x, xt)
+    kept = int(pk.kept_weights.item())
+    ref_z = torch.empty((T, N), dtype=torch.int16, device=DEV)
+    ref_g = torch.empty((T, N), dtype=torch.int16, device=DEV)
+    bsp.bsp_linear_planned(W, N, K, d, x, b, 0, ref_z)
+    bsp.bsp_linear_gathered(gplan, N, K, d, xt, b, 0, ref_g)
+    for transposed in (False, True):
+        for route, ref in ((bsp.ROUTE_ZERO_EXPANDED, ref_z), (bsp.ROUTE_GATHERED, ref_g)):
+            out = torch.full((N, T) if transposed else (T, N), 0x7FC0, dtype=torch.int16, device=DEV)
+            call = bsp.make_linear_call(N, K, d, T, plan=W, gplan=gplan, kept_weights=kept, X=x, XT=xt, bias=b,
+                                        **({"YT": out} if transposed else {"Y": out}))
+            assert bsp.bsp_linear_run(call, route) == route
+            bsp.bsp_linear_status()
+            assert torch.equal(out.t() if transposed else out, ref)
+    y = torch.full((T, N), 0x7FC0, dtype=torch.int16, device=DEV)
+    call = bsp.make_linear_call(N, K, d, T, plan=W, gplan=gplan, kept_weights=kept, X=x, XT=xt, bias=b, Y=y)
+    taken = bsp.bsp_linear_run(call)                                   # automatic choice
+    assert taken == bsp.bsp_linear_route(call) and taken in (bsp.ROUTE_ZERO_EXPANDED, bsp.ROUTE_GATHERED)
+    bsp.bsp_linear_status()
+    assert torch.equal(y, ref_z if taken == bsp.ROUTE_ZERO_EXPANDED else ref_g)
+    best, ms_z, ms_g = bsp.bsp_linear_tune(call, 3)
+    assert ms_z > 0 and ms_g > 0 and best == (bsp.ROUTE_GATHERED if ms_g < ms_z else bsp.ROUTE_ZERO_EXPANDED)
+    only_z = bsp.make_linear_call(N, K, d, T, plan=W, kept_weights=kept, X=x, bias=b, Y=y)
+    best, ms_z, ms_g = bsp.bsp_linear_tune(only_z, 2)
+    assert best == bsp.ROUTE_ZERO_EXPANDED and ms_z > 0 and ms_g == -1.0
+    with pytest.raises(bsp.BspError):
+        bsp.bsp_linear_run(only_z, bsp.ROUTE_GATHERED)                 # that route's operands were not given
+    bsp.bsp_linear_status()
