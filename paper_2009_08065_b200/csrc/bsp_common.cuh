@@ -193,6 +193,21 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* s_warp, int* tot
   return before + incl - v;
 }
 
+// Norm and reciprocal of the reported (not the deciding) quantities: the hardware's approximate square
+// root and reciprocal, each within about one unit in the last place of float32, far inside the 1e-5
+// these outputs are held to, at a sixth of the instructions of the correctly rounded forms.  Every
+// kernel that writes norms or gamma goes through these two, so all of them give the same bits.
+__device__ __forceinline__ float norm_from_sumsq(float S) {
+  float n;
+  asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(n) : "f"(S));
+  return n;
+}
+__device__ __forceinline__ float reciprocal(float x) {
+  float r;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+  return r;
+}
+
 struct NormOut {
   float* norms;
   const float* gamma_in;
@@ -204,9 +219,9 @@ struct NormOut {
 
 // Finishes one group from its float32 sum of squares; returns the group's penalty term.
 __device__ __forceinline__ double finish_group(const NormOut& o, size_t g, float S) {
-  const float n = __fsqrt_rn(S);
+  const float n = norm_from_sumsq(S);
   const float base = o.squared ? S : n;
-  const float fresh = __fdiv_rn(1.0f, base + o.eps);
+  const float fresh = reciprocal(base + o.eps);
   if (o.norms) o.norms[g] = n;
   if (o.gamma_out) o.gamma_out[g] = fresh;
   const float weight = o.gamma_in ? o.gamma_in[g] : fresh;

@@ -241,9 +241,9 @@ fused_stream_kernel(const __grid_constant__ StreamBatchT<N> B) {
         float n[8], base[8], fresh[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-          n[i] = __fsqrt_rn(acc[i]);
+          n[i] = norm_from_sumsq(acc[i]);
           base[i] = B.squared ? acc[i] : n[i];
-          fresh[i] = __fdiv_rn(1.0f, base[i] + B.eps);
+          fresh[i] = reciprocal(base[i] + B.eps);
         }
         if (J.norms) {
           *reinterpret_cast<float4*>(J.norms + g0) = make_float4(n[0], n[1], n[2], n[3]);
