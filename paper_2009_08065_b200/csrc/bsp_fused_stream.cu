@@ -47,7 +47,7 @@ constexpr int kReadyBit = 0x40000000;    // set in a published count
 struct StreamJob {
   FusedJob j;
   int parts, part_cols;      // column ranges per row-block, columns per range (multiple of 8)
-  int first_item;
+  int seg_round;             // first round of this matrix's segment (see locate) = row-blocks of the previous matrix
   int32_t* part_counts;      // [n_blocks * parts] published counts, then (job 0) the ticket
   unsigned long long* part_partial;   // [n_blocks * parts] published penalty partials (float64 bits, lowest bit set)
 };
@@ -56,32 +56,52 @@ struct StreamBatchT {
   int n_jobs, block, squared;
   float eps;
   int total_items, buf_bytes;
+  int parts_total;           // column ranges of one round over every matrix of the batch
   int* ticket;
   int* status;               // receives BSP_ERR_TIMEOUT when a bounded wait expires
+  // Item order (see locate): the table is sorted by row-block count; a matrix's "segment" is the run of
+  // rounds in which it is the smallest matrix still active.  The two arrays that locate searches are kept
+  // apart from the wide job records, so that a search stays within a few lines of the constant cache.
+  int seg_item[N];           // number of the first item of the matrix's segment
+  int parts_before[N];       // column ranges per round of the matrices before this one in the table
   StreamJob job[N];
 };
 // The job table travels as a kernel parameter: 14 KB for a full batch, which every launch has to
-// move; a batch of up to eight matrices (an encoder layer's) gets a table of 1.2 KB.  Both have the
-// same fields in the same order, so the small one is a copy of the large one's beginning.
+// move; a batch of up to eight matrices (an encoder layer's) gets a table of 1.2 KB with the same fields.
 constexpr int kStreamFewJobs = 8;
 using StreamBatch = StreamBatchT<kStreamMaxJobs>;
 
 struct Item {
   int jn, local, b, q, c0, pc;
 };
+// Items are numbered round by round: round r holds row-block r of every matrix that has one, matrix
+// after matrix, the column ranges of a block side by side.  The row-blocks of one matrix are therefore
+// a whole round apart, so the items whose counts an item needs were taken long before it (all but the
+// last few have finished), while a matrix-after-matrix order would make every item wait for the
+// slowest of some hundred items that started together with it.
 template <class Batch>
 __device__ __forceinline__ Item locate(const Batch& B, int item) {
   int lo = 0, hi = B.n_jobs - 1;
-  while (lo < hi) {
+  while (lo < hi) {                    // the segment: the last matrix whose segment starts at or before the item
     const int mid = (lo + hi + 1) >> 1;
-    if (B.job[mid].first_item <= item) lo = mid; else hi = mid - 1;
+    if (B.seg_item[mid] <= item) lo = mid; else hi = mid - 1;
+  }
+  const int seg_round = B.job[lo].seg_round;
+  const int per_round = B.parts_total - B.parts_before[lo];
+  const int u = item - B.seg_item[lo];
+  const int round = u / per_round;
+  const int o = u - round * per_round + B.parts_before[lo];
+  hi = B.n_jobs - 1;
+  while (lo < hi) {                    // the matrix: the last one whose ranges start at or before o
+    const int mid = (lo + hi + 1) >> 1;
+    if (B.parts_before[mid] <= o) lo = mid; else hi = mid - 1;
   }
   const StreamJob& O = B.job[lo];
   Item I;
   I.jn = lo;
-  I.local = item - O.first_item;
-  I.b = I.local / O.parts;
-  I.q = I.local - I.b * O.parts;
+  I.b = seg_round + round;
+  I.q = o - B.parts_before[lo];
+  I.local = I.b * O.parts + I.q;
   I.c0 = I.q * O.part_cols;
   I.pc = min(O.part_cols, O.j.cols - I.c0);
   return I;
@@ -104,22 +124,61 @@ __device__ __forceinline__ void issue_rows(const Batch& B, const Item& I, uint32
   }
 }
 
-// Published count of an item: waits (bounded) for its ready bit.
-__device__ __forceinline__ int wait_count(const int32_t* slot, int* status) {
+// Published word of an item as it is now (ready bit set or not).
+__device__ __forceinline__ int probe_count(const int32_t* slot) {
   int v;
   asm volatile("ld.relaxed.gpu.global.b32 %0, [%1];" : "=r"(v) : "l"(slot) : "memory");
-  if (v & kReadyBit) return v & (kReadyBit - 1);
-  const unsigned long long limit = tc::wait_limit_ns(status);
-  const unsigned long long start = tc::global_timer_ns();
+  return v;
+}
+// Published count of an item: waits (bounded) for its ready bit.  The limit is fetched only after
+// the first round of probes, so the usual short wait costs no extra trip to memory.
+__device__ __forceinline__ int wait_count(const int32_t* slot, int* status) {
+  unsigned long long limit = 0, start = 0;
   for (;;) {
 #pragma unroll 1
     for (int i = 0; i < 64; ++i) {
-      asm volatile("ld.relaxed.gpu.global.b32 %0, [%1];" : "=r"(v) : "l"(slot) : "memory");
+      const int v = probe_count(slot);
       if (v & kReadyBit) return v & (kReadyBit - 1);
       __nanosleep(32);
     }
-    if (tc::global_timer_ns() - start > limit) { atomicExch(status, BSP_ERR_TIMEOUT); return 0; }
+    if (limit == 0) {
+      limit = tc::wait_limit_ns(status);
+      start = tc::global_timer_ns();
+    } else if (tc::global_timer_ns() - start > limit) {
+      atomicExch(status, BSP_ERR_TIMEOUT);
+      return 0;
+    }
   }
+}
+
+// Up to four published counts, words slot[0], slot[stride], ...: v[u] holds what an earlier probe saw
+// (any word with the ready bit is final).  Words that are not ready are asked for again, all of them
+// at once, until every one is; returns the sum of the counts.  n = how many of the four exist.
+__device__ __forceinline__ int wait_counts4(const int32_t* slot, int stride, int n, int (&v)[4], int* status) {
+  unsigned long long limit = 0, start = 0;
+  for (int round = 0;; ++round) {
+    bool all = true;
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      if (u < n && !(v[u] & kReadyBit)) v[u] = probe_count(slot + u * stride);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) all = all && (u >= n || (v[u] & kReadyBit) != 0);
+    if (all) break;
+    __nanosleep(32);
+    if ((round & 63) == 63) {
+      if (limit == 0) {
+        limit = tc::wait_limit_ns(status);
+        start = tc::global_timer_ns();
+      } else if (tc::global_timer_ns() - start > limit) {
+        atomicExch(status, BSP_ERR_TIMEOUT);
+        return 0;
+      }
+    }
+  }
+  int sum = 0;
+#pragma unroll
+  for (int u = 0; u < 4; ++u) sum += u < n ? (v[u] & (kReadyBit - 1)) : 0;
+  return sum;
 }
 
 // Published penalty partial of an item: waits (bounded) for its ready bit.
@@ -140,7 +199,11 @@ __device__ __forceinline__ double wait_partial(const unsigned long long* slot, i
   }
 }
 
-template <int N>
+// kOneWave: the batch fits the GPU in one wave (every CTA resident, item = block index, no ticket).
+// All items then start together and every one of them waits for the slowest of the items before it,
+// so the packed tile is built in shared memory while that wait lasts; with tickets the counts an item
+// needs are ready long before it asks, and the tile goes from the row buffer straight to memory.
+template <int N, bool kOneWave>
 __global__ void __launch_bounds__(kStreamThreads, 8)
 fused_stream_kernel(const __grid_constant__ StreamBatchT<N> B) {
   extern __shared__ __align__(128) uint8_t s_raw[];
@@ -159,7 +222,7 @@ fused_stream_kernel(const __grid_constant__ StreamBatchT<N> B) {
   // A batch that fits the GPU in one wave needs no ticket: every CTA is resident, item = block index,
   // and the item's job is looked up (which brings its part of the kernel parameters into the constant
   // cache) while the clearing kernel is still running.
-  const bool direct = B.ticket == nullptr;
+  constexpr bool direct = kOneWave;
   int item = static_cast<int>(blockIdx.x);
   Item I = locate(B, direct ? item : 0);
   if (direct) {
@@ -182,8 +245,13 @@ fused_stream_kernel(const __grid_constant__ StreamBatchT<N> B) {
     if (item >= B.total_items) return;
     I = locate(B, item);
   }
-  if (warp == 0) issue_rows(B, I, smem_u32(s_raw), bar, lane);
-  {
+  // A CTA works through items until the tickets run out.  It takes its next ticket only when every
+  // wait of the current item is behind it (what is left then, writing indices and the tile, waits for
+  // nobody), so an item is never held by a CTA that is itself waiting, and the trip to the ticket
+  // counter overlaps those writes.
+  uint32_t parity = 0u;
+  for (;;) {
+    if (warp == 0) issue_rows(B, I, smem_u32(s_raw), bar, lane);
     const StreamJob& O = B.job[I.jn];
     const FusedJob& J = O.j;
     const int b = I.b, q = I.q, c0 = I.c0, pc = I.pc, local = I.local;
@@ -192,7 +260,7 @@ fused_stream_kernel(const __grid_constant__ StreamBatchT<N> B) {
     uint8_t* s_flag = reinterpret_cast<uint8_t*>(s_idx + O.part_cols);                  // [pc]
     // one decision for the whole CTA; if the rows never arrived, hold the buffer a millisecond for
     // copies that may still be on their way, then leave
-    if (!__syncthreads_and(mbar_wait(bar, 0u, B.status) ? 1 : 0)) {
+    if (!__syncthreads_and(tc::mbar_wait_suspended(bar, parity, B.status) ? 1 : 0)) {
       if (threadIdx.x == 0) atomicExch(B.status, BSP_ERR_TIMEOUT);
       const unsigned long long start = tc::global_timer_ns();
       while (tc::global_timer_ns() - start < tc::kQuietNs) __nanosleep(2000);
@@ -322,15 +390,70 @@ fused_stream_kernel(const __grid_constant__ StreamBatchT<N> B) {
       }
     }
 
-    // ---- phase B: offsets from the published counts
-    int before = 0, in_block_before = 0, in_block = 0;
-    for (int i = threadIdx.x; i < local; i += blockDim.x) before += wait_count(O.part_counts + i, B.status);
-    if (O.parts > 1) {
-      for (int i = threadIdx.x; i < O.parts; i += blockDim.x) {
-        const int c = wait_count(O.part_counts + b * O.parts + i, B.status);
-        in_block += c;
-        if (i < q) in_block_before += c;
+    if constexpr (kOneWave) {
+    // ---- local work, continued: the packed tile of this part, built in place.  Row r's kept values
+    // move to the front of row r in the row buffer (position p comes from column idx[p] >= p, so moving
+    // left in ascending order never overwrites a value that is still needed).  Nothing here depends on
+    // other items: the trip of the published counts through memory (phase B) overlaps it, and what is
+    // left once the offsets are known is a copy of contiguous rows.
+    // A lane takes two neighbouring kept positions: their column numbers are one 32-bit word of the
+    // list and the two values lie about six columns apart (three banks from lane to lane at the usual
+    // densities, where eight positions per lane would put four lanes on each bank).  A warp owns its
+    // rows from here to the end of the item; it handles 32 pairs of four rows at a time: reads, then
+    // writes, with the reads of later pairs lying beyond everything written so far.
+    __syncthreads();                          // the list is complete and the execution-layout pass has read the rows
+    {
+      const int kc_part = s_kc;
+      const int n_pairs = kc_part >> 1;
+      uint16_t* s_wm = reinterpret_cast<uint16_t*>(s_raw);
+      uint32_t* s_w32 = reinterpret_cast<uint32_t*>(s_raw);
+      const int row_words = pc >> 1;
+      for (int c = 0; c < n_pairs; c += 32) {
+        const int pp = c + lane;
+        const bool on = pp < n_pairs;
+        const uint32_t cc = on ? *reinterpret_cast<const uint32_t*>(s_idx + 2 * pp) : 0u;
+        const uint16_t* sa = s_wm + (cc & 0xffffu);
+        const uint16_t* sb = s_wm + (cc >> 16);
+        for (int r = warp; r < d; r += 4 * n_warps) {
+          uint32_t w[4];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const int rr = r + u * n_warps;
+            if (on && rr < d) w[u] = static_cast<uint32_t>(sa[rr * pc]) | (static_cast<uint32_t>(sb[rr * pc]) << 16);
+          }
+          __syncwarp();
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const int rr = r + u * n_warps;
+            if (on && rr < d) s_w32[rr * row_words + pp] = w[u];
+          }
+        }
+        __syncwarp();
       }
+      if (kc_part & 1) {                      // an odd count: the last position, after every pair (its source lies beyond them)
+        const int p = kc_part - 1;
+        const int col = s_idx[p];
+        for (int r = warp + lane * n_warps; r < d; r += 32 * n_warps) s_wm[r * pc + p] = s_wm[r * pc + col];
+      }
+    }
+    }
+
+    // ---- phase B: offsets from the published counts
+    // (a thread asks for all its words before it waits for any: the trips to memory overlap.  Asking
+    // earlier, before the local work, made the waits longer, not shorter: measured.)
+    int before = 0, in_block_before = 0, in_block = 0;
+    const int mine_part = static_cast<int>(threadIdx.x) < O.parts && O.parts > 1 ? static_cast<int>(threadIdx.x) : -1;   // parts <= 31
+    int pv = mine_part >= 0 ? probe_count(O.part_counts + b * O.parts + mine_part) : 0;
+    for (int i0 = threadIdx.x; i0 < local; i0 += 4 * blockDim.x) {
+      int v[4] = {0, 0, 0, 0};
+      const int n = (local - i0 + static_cast<int>(blockDim.x) - 1) / static_cast<int>(blockDim.x);   // words of this thread in this round (capped at four below)
+      before += wait_counts4(O.part_counts + i0, static_cast<int>(blockDim.x), n < 4 ? n : 4, v, B.status);
+    }
+    if (mine_part >= 0) {
+      if (!(pv & kReadyBit)) pv = wait_count(O.part_counts + b * O.parts + mine_part, B.status);
+      pv &= kReadyBit - 1;
+      in_block = pv;
+      if (mine_part < q) in_block_before = pv;
     }
     before = warp_sum(before);
     in_block = warp_sum(in_block);
@@ -367,73 +490,86 @@ fused_stream_kernel(const __grid_constant__ StreamBatchT<N> B) {
         *J.penalty = tot;
       }
     }
+    // no wait from here on: take the next item (the answer is only looked at after the writes below)
+    int next_item = 0;
+    if (!direct && threadIdx.x == 0) next_item = atomicAdd(B.ticket, 1);
     if (kc > 0) {
       for (int p = threadIdx.x; p < kc; p += blockDim.x) J.idx[base + p] = c0 + s_idx[p];
       // packed tile: row r of the block occupies vals[tile0 + r*kc_block, +kc_block); this part fills
-      // positions [off_in_block, off_in_block + kc) of every row.  One warp per row; whole 16-byte
-      // vectors where the destination is aligned, ragged ends by element.
-      const bool vec_ok = (reinterpret_cast<uintptr_t>(J.vals) & 15) == 0;
+      // positions [off_in_block, off_in_block + kc) of every row.
       const long long tile0 = static_cast<long long>(d) * block_base;
-      if (vec_ok && (kc_block & 7) == 0 && (tile0 & 7) == 0) {
-        // every row of the tile starts at the same offset from a 16-byte boundary: a lane keeps the
-        // eight column numbers of its vector in registers and walks the rows of its warp with them
-        const int head = (8 - (off_in_block & 7)) & 7;
-        const int n_vec = kc > head ? (kc - head) >> 3 : 0;
-        for (int v = lane; v < n_vec; v += 32) {
-          const int p = head + (v << 3);
-          int col[8];
-#pragma unroll
-          for (int i = 0; i < 8; ++i) col[i] = s_idx[p + i];
-          for (int r = warp; r < d; r += n_warps) {
-            const uint16_t* srow = s_w + r * pc;
-            uint32_t o[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-              o[i] = static_cast<uint32_t>(srow[col[2 * i]]) | (static_cast<uint32_t>(srow[col[2 * i + 1]]) << 16);
-            *reinterpret_cast<uint4*>(J.vals + tile0 + static_cast<long long>(r) * kc_block + off_in_block + p) =
-                make_uint4(o[0], o[1], o[2], o[3]);
-          }
-        }
-        const int tail0 = head + (n_vec << 3);
-        for (int r = warp; r < d; r += n_warps) {      // ragged ends of each row by element
-          const uint16_t* srow = s_w + r * pc;
-          uint16_t* out_row = J.vals + tile0 + static_cast<long long>(r) * kc_block + off_in_block;
-          if (lane < 8) {
-            if (lane < head && lane < kc) out_row[lane] = srow[s_idx[lane]];
-          } else if (lane < 16) {
-            const int p = tail0 + (lane - 8);
-            if (p >= head && p < kc) out_row[p] = srow[s_idx[p]];
-          }
-        }
-      } else {
+      const uintptr_t vals_addr = reinterpret_cast<uintptr_t>(J.vals);
+      if constexpr (kOneWave) {
+        // from the front of row r of the buffer, where the values were gathered above.  Each warp copies
+        // the rows it compacted: 16-byte pieces where the destination row is aligned (the source is),
+        // 4-byte pieces or single elements otherwise.
+        __syncwarp();
         for (int r = warp; r < d; r += n_warps) {
           const uint16_t* srow = s_w + r * pc;
           const long long e0 = tile0 + static_cast<long long>(r) * kc_block + off_in_block;
           uint16_t* out_row = J.vals + e0;
-          if (vec_ok) {
-            const int head = static_cast<int>((8 - (e0 & 7)) & 7);
-            const int n_vec = kc > head ? (kc - head) >> 3 : 0;
-            for (int v = lane; v < n_vec; v += 32) {
-              const int p = head + (v << 3);
-              uint32_t o[4];
-#pragma unroll
-              for (int i = 0; i < 4; ++i)
-                o[i] = static_cast<uint32_t>(srow[s_idx[p + 2 * i]]) | (static_cast<uint32_t>(srow[s_idx[p + 2 * i + 1]]) << 16);
-              *reinterpret_cast<uint4*>(out_row + p) = make_uint4(o[0], o[1], o[2], o[3]);
-            }
-            const int tail0 = head + (n_vec << 3);
-            if (lane < 8) {
-              if (lane < head && lane < kc) out_row[lane] = srow[s_idx[lane]];
-            } else if (lane < 16) {
-              const int p = tail0 + (lane - 8);
-              if (p >= head && p < kc) out_row[p] = srow[s_idx[p]];
-            }
-          } else {
-            for (int p = lane; p < kc; p += 32) out_row[p] = srow[s_idx[p]];
+          int done = 0;
+          if ((vals_addr & 15) == 0 && (e0 & 7) == 0) {
+            const int n_vec = kc >> 3;
+            for (int v = lane; v < n_vec; v += 32)
+              *reinterpret_cast<uint4*>(out_row + (v << 3)) = *reinterpret_cast<const uint4*>(srow + (v << 3));
+            done = n_vec << 3;
+          } else if ((vals_addr & 3) == 0 && (e0 & 1) == 0) {
+            const int n_w = kc >> 1;
+            for (int v = lane; v < n_w; v += 32)
+              *reinterpret_cast<uint32_t*>(out_row + (v << 1)) = *reinterpret_cast<const uint32_t*>(srow + (v << 1));
+            done = n_w << 1;
           }
+          for (int p = done + lane; p < kc; p += 32) out_row[p] = srow[p];
+        }
+      } else if ((vals_addr & 3) == 0 && ((kc_block | off_in_block) & 1) == 0 && (tile0 & 1) == 0) {
+        // Every row of this part starts on a 4-byte boundary.  A lane takes two neighbouring kept
+        // positions (one word of the list, two values about six columns apart: different banks from lane
+        // to lane) and the pair leaves as one 4-byte store, 128 contiguous bytes per warp; four rows of
+        // the warp at a time, eight loads in flight.
+        const int n_pairs = kc >> 1;
+        uint32_t* out32 = reinterpret_cast<uint32_t*>(J.vals + tile0 + off_in_block);
+        const size_t row_words = static_cast<size_t>(kc_block >> 1);
+        for (int pp = lane; pp < n_pairs; pp += 32) {
+          const uint32_t cc = *reinterpret_cast<const uint32_t*>(s_idx + 2 * pp);
+          const uint16_t* sa = s_w + (cc & 0xffffu);
+          const uint16_t* sb = s_w + (cc >> 16);
+          uint32_t* o = out32 + pp;
+          for (int r = warp; r < d; r += 4 * n_warps) {
+            uint32_t w[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              const int rr = r + u * n_warps;
+              if (rr < d) w[u] = static_cast<uint32_t>(sa[rr * pc]) | (static_cast<uint32_t>(sb[rr * pc]) << 16);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              const int rr = r + u * n_warps;
+              if (rr < d) o[static_cast<size_t>(rr) * row_words] = w[u];
+            }
+          }
+        }
+        if (kc & 1) {                         // an odd part of a split row-block: its last position, one thread per row
+          const int p = kc - 1;
+          for (int rr = threadIdx.x; rr < d; rr += blockDim.x)
+            J.vals[tile0 + static_cast<long long>(rr) * kc_block + off_in_block + p] = s_w[rr * pc + s_idx[p]];
+        }
+      } else {
+        for (int r = warp; r < d; r += n_warps) {
+          const uint16_t* srow = s_w + r * pc;
+          uint16_t* out_row = J.vals + tile0 + static_cast<long long>(r) * kc_block + off_in_block;
+          for (int p = lane; p < kc; p += 32) out_row[p] = srow[s_idx[p]];
         }
       }
     }
+    if (direct) break;
+    if (threadIdx.x == 0) s_item = next_item;
+    __syncthreads();                         // everybody is done with the row buffer and the lists; s_item is there
+    item = s_item;
+    if (item >= B.total_items) break;
+    I = locate(B, item);
+    parity ^= 1u;
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the buffer's readers are done before the copies write it
   }
 }
 
@@ -448,6 +584,12 @@ stream_clear_kernel(const __grid_constant__ StreamBatchT<N> B) {
   for (int i = threadIdx.x; i < n; i += blockDim.x) O.part_partial[i] = 0ull;
 }
 
+int total_parts_so_far(const StreamBatch& B, int n) {
+  int p = 0;
+  for (int i = 0; i < n; ++i) p += B.job[i].parts;
+  return p;
+}
+
 // Fills the job table; false when a matrix does not fit this kernel's limits.
 bool fill_batch(StreamBatch& B, const FusedJob* jobs, int n_jobs, int block, float eps, int squared,
                 int32_t* const* part_counts, double* const* part_partial, size_t* smem_out) {
@@ -458,22 +600,39 @@ bool fill_batch(StreamBatch& B, const FusedJob* jobs, int n_jobs, int block, flo
   int total = 0, max_part_cols = 0;
   const int max_cols = (kStreamRowBytes / (2 * block)) / 8 * 8;        // columns whose rows fit a row buffer
   if (max_cols < 8) return false;
+  // table order: ascending row-block count (insertion sort, stable; at most 96 entries)
+  int order[kStreamMaxJobs];
+  for (int i = 0; i < n_jobs; ++i) {
+    int k = i;
+    while (k > 0 && jobs[order[k - 1]].n_blocks > jobs[i].n_blocks) { order[k] = order[k - 1]; --k; }
+    order[k] = i;
+  }
   for (int i = 0; i < n_jobs; ++i) {
     StreamJob& O = B.job[i];
-    O.j = jobs[i];
-    const int cols = jobs[i].cols;
+    const int src = order[i];
+    O.j = jobs[src];
+    const int cols = O.j.cols;
     O.parts = (cols + max_cols - 1) / max_cols;
     O.part_cols = ((cols + O.parts - 1) / O.parts + 7) / 8 * 8;
     O.parts = (cols + O.part_cols - 1) / O.part_cols;
     if (O.parts > 31) return false;
-    if (static_cast<long long>(jobs[i].n_blocks) * O.parts + 2 > static_cast<long long>(jobs[i].n_blocks) * 32) return false;
-    O.first_item = total;
-    O.part_counts = part_counts[i];
-    O.part_partial = reinterpret_cast<unsigned long long*>(part_partial[i]);
-    total += jobs[i].n_blocks * O.parts;
+    if (static_cast<long long>(O.j.n_blocks) * O.parts + 2 > static_cast<long long>(O.j.n_blocks) * 32) return false;
+    O.part_counts = part_counts[src];
+    O.part_partial = reinterpret_cast<unsigned long long*>(part_partial[src]);
+    B.parts_before[i] = total_parts_so_far(B, i);
+    total += O.j.n_blocks * O.parts;
     if (O.part_cols > max_part_cols) max_part_cols = O.part_cols;
   }
   B.total_items = total;
+  B.parts_total = total_parts_so_far(B, n_jobs);
+  int seg_item = 0, prev_blocks = 0;
+  for (int i = 0; i < n_jobs; ++i) {
+    StreamJob& O = B.job[i];
+    B.seg_item[i] = seg_item;
+    O.seg_round = prev_blocks;
+    seg_item += (O.j.n_blocks - prev_blocks) * (B.parts_total - B.parts_before[i]);
+    prev_blocks = O.j.n_blocks;
+  }
   B.buf_bytes = static_cast<int>(round_up(static_cast<size_t>(block) * max_part_cols * 2, 128));
   B.ticket = B.job[0].part_counts + B.job[0].j.n_blocks * B.job[0].parts + 1;
   *smem_out = static_cast<size_t>(B.buf_bytes) + static_cast<size_t>(max_part_cols) * 3 + 16;   // rows, 2-byte list, flags
@@ -505,13 +664,17 @@ int fused_stream(const FusedJob* jobs, int n_jobs, int block, float eps, int squ
   int st = BSP_OK;
   if (ok) {
     if (!td->attr_set[7]) {
-      cudaError_t e = cudaFuncSetAttribute(fused_stream_kernel<kStreamMaxJobs>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemCap);
+      cudaError_t e = cudaFuncSetAttribute(fused_stream_kernel<kStreamMaxJobs, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemCap);
       if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(fused_stream_kernel<kStreamFewJobs>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemCap);
+        e = cudaFuncSetAttribute(fused_stream_kernel<kStreamMaxJobs, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemCap);
+      if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(fused_stream_kernel<kStreamFewJobs, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemCap);
+      if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(fused_stream_kernel<kStreamFewJobs, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemCap);
       if (e != cudaSuccess) { delete B; return cuda_fail(e); }
       td->attr_set[7] = true;
     }
-    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fused_stream_kernel<kStreamMaxJobs>, kStreamThreads, smem_max);
+    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fused_stream_kernel<kStreamMaxJobs, false>, kStreamThreads, smem_max);
     if (e != cudaSuccess) { delete B; return cuda_fail(e); }
     if (per_sm * td->sms < 32) ok = false;    // the no-deadlock argument needs 32 CTAs resident at once
   }
@@ -522,9 +685,13 @@ int fused_stream(const FusedJob* jobs, int n_jobs, int block, float eps, int squ
     if (B->total_items <= per_sm * td->sms) B->ticket = nullptr;    // one wave: item = block index
     const bool few = n <= kStreamFewJobs;
     StreamBatchT<kStreamFewJobs> small;
-    static_assert(offsetof(StreamBatchT<kStreamFewJobs>, job) == offsetof(StreamBatch, job), "tables must share their beginning");
     if (few) {
-      memcpy(&small, B, sizeof(small));
+      memcpy(&small, B, offsetof(StreamBatch, seg_item));      // the scalar fields come first in both
+      for (int i = 0; i < kStreamFewJobs; ++i) {
+        small.seg_item[i] = B->seg_item[i];
+        small.parts_before[i] = B->parts_before[i];
+        small.job[i] = B->job[i];
+      }
       stream_clear_kernel<kStreamFewJobs><<<n, 256, 0, s>>>(small);
     } else {
       stream_clear_kernel<kStreamMaxJobs><<<n, 256, 0, s>>>(*B);
@@ -532,7 +699,8 @@ int fused_stream(const FusedJob* jobs, int n_jobs, int block, float eps, int squ
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { st = cuda_fail(e); break; }
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(B->total_items);
+    const int resident = per_sm * td->sms;
+    cfg.gridDim = dim3(B->total_items < resident ? B->total_items : resident);   // CTAs loop until the tickets run out
     cfg.blockDim = dim3(kStreamThreads);
     cfg.dynamicSmemBytes = smem_max;
     cfg.stream = s;
@@ -541,8 +709,11 @@ int fused_stream(const FusedJob* jobs, int n_jobs, int block, float eps, int squ
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    e = few ? cudaLaunchKernelEx(&cfg, fused_stream_kernel<kStreamFewJobs>, small)
-            : cudaLaunchKernelEx(&cfg, fused_stream_kernel<kStreamMaxJobs>, *B);
+    const bool one_wave = B->ticket == nullptr;
+    e = few ? (one_wave ? cudaLaunchKernelEx(&cfg, fused_stream_kernel<kStreamFewJobs, true>, small)
+                        : cudaLaunchKernelEx(&cfg, fused_stream_kernel<kStreamFewJobs, false>, small))
+            : (one_wave ? cudaLaunchKernelEx(&cfg, fused_stream_kernel<kStreamMaxJobs, true>, *B)
+                        : cudaLaunchKernelEx(&cfg, fused_stream_kernel<kStreamMaxJobs, false>, *B));
     if (e != cudaSuccess) { st = cuda_fail(e); break; }
     *used = true;
   }

@@ -88,6 +88,30 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const i
     if (global_timer_ns() - start > limit) return false;
   }
 }
+// The same wait for many threads at once (a whole CTA waiting for its bulk copies): each probe lets
+// the hardware suspend the thread for up to `kSuspendNs` or until the phase completes, so the
+// waiting warps leave the issue slots to the CTAs that share the SM instead of polling.
+constexpr uint32_t kSuspendNs = 4000u;
+__device__ __forceinline__ bool mbar_try_wait_suspend(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity), "r"(kSuspendNs)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_suspended(uint32_t bar, uint32_t parity, const int* status) {
+  if (mbar_try_wait_suspend(bar, parity)) return true;
+  const unsigned long long limit = wait_limit_ns(status);
+  const unsigned long long start = global_timer_ns();
+  for (;;) {
+    if (mbar_try_wait_suspend(bar, parity)) return true;
+    if (global_timer_ns() - start > limit) return false;
+  }
+}
 // Bounded wait until *counter >= need (acquire at GPU scope): a counter in global memory that
 // other CTAs of the same launch bump.
 __device__ __forceinline__ bool wait_counter(const int* counter, int need, const int* status) {
