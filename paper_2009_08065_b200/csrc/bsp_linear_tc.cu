@@ -56,7 +56,35 @@ struct LinearParams {
   int* status;
 };
 
-constexpr int kThreadsTc = kThreads + 32;   // 11 warps: a second TMA producer warp for the weight tiles
+// Epilogue groups of four warps (one warp per quarter of the TMEM lanes), two staging buffers each.
+// Four groups with one buffer each (the same 32 KB; the exposed epilogue of a CTA's last tile then takes
+// two pieces per group instead of four) were measured 1.5 us slower per four-GEMM layer at 4096 tokens:
+// sixteen warps contend for the shared memory that the operand copies and the tensor core keep busy.
+#ifndef BSP_TC_GROUPS
+#define BSP_TC_GROUPS 2
+#endif
+constexpr int kGroups = BSP_TC_GROUPS;
+constexpr int kEpiThreads = 128 * kGroups;
+constexpr int kBufPerGroup = kEpiBuffers / kGroups;
+static_assert(kGroups == 2 || kGroups == 4, "two or four epilogue groups");
+constexpr int kWeightWarp = 2 + 4 * kGroups;            // the second TMA producer warp, for the weight tiles
+constexpr int kThreadsTc = 32 * (kWeightWarp + 1);
+
+// Named barriers of this kernel's epilogue: 5 + g among the 128 threads of group g, 3 and 4 among all of them.
+__device__ __forceinline__ void tc_group_sync(int g) { asm volatile("bar.sync %0, 128;" ::"r"(5 + g) : "memory"); }
+__device__ __forceinline__ void tc_epilogue_sync_all() { asm volatile("bar.sync 3, %0;" ::"n"(kEpiThreads) : "memory"); }
+__device__ __forceinline__ bool tc_epilogue_all_ok(bool ok) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.b32 p, %1, 0;\n\t"
+      "barrier.cta.red.and.pred q, 4, %2, p;\n\t"
+      "selp.u32 %0, 1, 0, q;\n\t}"
+      : "=r"(r)
+      : "r"(ok ? 1u : 0u), "n"(kEpiThreads)
+      : "memory");
+  return r != 0u;
+}
 
 template <int BN>
 __global__ void __launch_bounds__(kThreadsTc, 1)
@@ -87,7 +115,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_w)) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_y)) : "memory");
     for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 2); mbar_init(empty_bar(s), 1); }   // two producers arm a stage
-    for (int a = 0; a < 2; ++a) { mbar_init(acc_full_bar(a), 1); mbar_init(acc_empty_bar(a), 8); }
+    for (int a = 0; a < 2; ++a) { mbar_init(acc_full_bar(a), 1); mbar_init(acc_empty_bar(a), 4 * kGroups); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -107,7 +135,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
   // the next kernel in the stream start its own prologue as soon as SMs become free.  When the
   // caller vouches that the plan is older than the previous kernel, the weight producer does not
   // wait: its first tiles are on their way while the previous kernel finishes writing X.
-  if (!(P.plan_stable && warp == 10)) asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (!(P.plan_stable && warp == kWeightWarp)) asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   const int m_tiles = (P.tokens + kBlockM - 1) / kBlockM;
@@ -117,7 +145,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
 
   if (warp == 0 && lane == 0) {
     // ---------------------------------------------------------------- TMA producer of the X tiles
-    // (the two operands of a stage are issued by two warps, this one and warp 10, so neither waits
+    // (the two operands of a stage are issued by two warps, this one and the last one, so neither waits
     // behind the other's copy)
     int stage = 0;
     uint32_t phase = 0;
@@ -133,7 +161,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
       }
     }
     if (!ok) record_timeout(P.status, timed_out);
-  } else if (warp == 10 && lane == 0) {
+  } else if (warp == kWeightWarp && lane == 0) {
     // ---------------------------------------------------------------- TMA producer of the weight tiles
     int stage = 0;
     uint32_t phase = 0;
@@ -180,14 +208,14 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
       acc ^= 1;
     }
     if (!ok) record_timeout(P.status, timed_out);
-  } else if (warp >= 2 && warp < 10) {
+  } else if (warp >= 2 && warp < kWeightWarp) {
     // ---------------------------------------------------------------- epilogue
-    const int group = (warp - 2) >> 2;       // 0 or 1
+    const int group = (warp - 2) >> 2;
     const int quad = warp & 3;               // TMEM lanes [32*quad, 32*quad+32) belong to this warp
     const int row = quad * 32 + lane;        // token row of this thread inside the tile
-    const int epi_tid = threadIdx.x - 64;    // 0..255 among the epilogue threads
+    const int epi_tid = threadIdx.x - 64;    // index among the epilogue threads
     const bool issuer = (epi_tid & 127) == 0;  // the thread of each group that owns its TMA stores
-    const uint32_t buf0 = smem_base + S * Cfg::kStage + group * 2 * kEpiStage;   // this group's two staging buffers
+    const uint32_t buf0 = smem_base + S * Cfg::kStage + group * kBufPerGroup * kEpiStage;   // this group's staging buffers
     uint32_t my_piece = 0;                   // pieces staged by this group so far: selects the buffer
     uint16_t* s_bias = reinterpret_cast<uint16_t*>(smem + S * Cfg::kStage + kEpiBytes);  // [2][BN] bf16
     const uint32_t row_off = static_cast<uint32_t>(row) * 64u;
@@ -200,25 +228,25 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
       // Bias of this tile's columns, in the half of s_bias that belongs to this accumulator.  The
       // other group can lag by at most one tile (it has to reach the barrier below for this tile),
       // so the values it may still be reading are in the other half.
-      for (int c = epi_tid; c < BN; c += 256)
+      for (int c = epi_tid; c < BN; c += kEpiThreads)
         s_bias[acc * BN + c] = (P.bias != nullptr && n0 + c < P.n_out) ? __ldg(P.bias + n0 + c) : static_cast<uint16_t>(0);
-      epilogue_sync_all();
-      // all 256 threads take the same decision, so nobody is left alone at a named barrier below
-      if (!epilogue_all_ok(mbar_wait(acc_full_bar(acc), acc_phase[acc], P.status))) { ok = false; break; }
+      tc_epilogue_sync_all();
+      // all epilogue threads take the same decision, so nobody is left alone at a named barrier below
+      if (!tc_epilogue_all_ok(mbar_wait(acc_full_bar(acc), acc_phase[acc], P.status))) { ok = false; break; }
       tcgen05_fence_after();
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + static_cast<uint32_t>(acc * BN);
       const int pieces = (min(BN, P.n_out - n0) + kEpiCols - 1) / kEpiCols;
       bool released = false;
 #pragma unroll 1
-      for (int pc = group; pc < pieces; pc += 2) {
+      for (int pc = group; pc < pieces; pc += kGroups) {
         const int c0 = pc * kEpiCols;
-        const uint32_t buf = buf0 + (my_piece & 1u) * kEpiStage;
+        const uint32_t buf = buf0 + (my_piece % kBufPerGroup) * kEpiStage;
         ++my_piece;
-        if (issuer) tma_store_wait_read<1>();   // the store issued two pieces ago has read this buffer
-        group_sync(group);
         EpiloguePiece piece;
         piece_load(taddr + c0, smem_u32(s_bias + acc * BN + c0), piece);
-        if (pc + 2 >= pieces) {              // this warp's last read of the accumulator
+        if (issuer) tma_store_wait_read<kBufPerGroup - 1>();   // the store that last used this buffer has read it
+        tc_group_sync(group);
+        if (pc + kGroups >= pieces) {        // this warp's last read of the accumulator
           tcgen05_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(acc_empty_bar(acc));
@@ -227,7 +255,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         if (P.transposed) piece_store_transposed(piece, P.act, buf, row);
         else piece_store(piece, P.act, buf + row_off, row_xor);
         fence_async_smem();                  // make the staged piece visible to the TMA engine
-        group_sync(group);
+        tc_group_sync(group);
         if (issuer) {
           // rows beyond `tokens` / columns beyond `n_out` are clipped by the tensor map
           if (P.transposed) tma_store_2d(&map_y, m0, n0 + c0, buf);
