@@ -85,8 +85,8 @@ int bsp_group_norms(const void* W, int rows, int cols, int ldw, int block, int o
 
 /* ---------------------------------------------------------------------------------------------
  * bsp_penalty_grad — the regulariser's gradient with respect to W with the penalty weights held
- * fixed, which is what Algorithm 2's inner loop needs between two gamma updates ("Update model
- * weight W to minimize mixed_loss using Adam", mixed_loss = l1loss + f(W, b)):
+ * fixed, which is what Algorithm 2's inner loop needs between two gamma updates (its Adam step
+ * minimises the task loss plus the reweighted l1 term):
  *   BSP_PEN_L2   (Eq. 2 / Eq. 3):  G_e = scale * gamma_g * W_e / ||W_g||_2   (0 for an all-zero group)
  *   BSP_PEN_L2SQ (squared norms):  G_e = scale * 2 * alpha_g * W_e
  * gamma: float32 per-group array (shape by orientation) from an earlier bsp_group_norms call;
@@ -113,8 +113,8 @@ int bsp_pack_bound(int rows, int cols, int block, int orient,
 int bsp_pack_scratch_bytes(int rows, int cols, int block, int orient, size_t* bytes);
 
 /* ---------------------------------------------------------------------------------------------
- * bsp_prune_pack — Algorithm 1 followed by the compressed storage of Section 3.1 ("only the
- * non-zero rows/columns at the block level need to be indexed").
+ * bsp_prune_pack — Algorithm 1 followed by the compressed storage of Section 3.1 (one index per
+ * kept row or column of a block, not one per weight).
  *
  * Decision (Algorithm 1 prunes a group iff its l2 norm <= t_b): group g is KEPT iff
  *   S_g > t_b * t_b, both sides float32, S_g as defined for bsp_group_norms; a negative t_b
@@ -178,8 +178,8 @@ int bsp_prune_pack_static(const void* W, int rows, int cols, int ldw, int block,
                           int64_t* kept_weights, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
- * bsp_percentile_threshold — Section 3.1: "prune ... according to our pre-set threshold or
- * percentile".  Per-matrix threshold for a target compression rate c = total/kept:
+ * bsp_percentile_threshold — Section 3.1 lets the threshold be given or follow from a
+ * percentile.  Per-matrix threshold for a target compression rate c = total/kept:
  * with G groups, r = floor(G * (1 - 1/c)) groups are to be removed; *threshold_out (device
  * float) receives t_b = the float32 square root of the r-th smallest S_g, raised by single ulps
  * until t_b * t_b >= that S_g, so that Algorithm 1's `<=` removes that group and its ties.
@@ -199,7 +199,7 @@ int bsp_apply_mask(void* W, int rows, int cols, int ldw, int block, int orient,
 
 /* ---------------------------------------------------------------------------------------------
  * bsp_masked_adam_step — one iteration of Algorithm 2's retraining loop on one weight matrix:
- * "update W ... using Adam", then "W = W * Mask", in one pass.  Adam as published (Kingma & Ba 2015,
+ * the Adam update of W, then W = W * Mask, in one pass.  Adam as published (Kingma & Ba 2015,
  * bias-corrected; the paper names no hyper-parameters beyond the learning rate, so all are the
  * caller's):
  *   m = beta1 m + (1 - beta1) g,   v = beta2 v + (1 - beta2) g^2,

@@ -229,8 +229,8 @@ def group_any(mask: np.ndarray, block: int, orient: str) -> np.ndarray:
 
 
 # ---------------------------------------------------------------------------
-# choosing t_b from a percentile, or a keep count per block  (Section 3.1:
-# "pre-set threshold or percentile")
+# choosing t_b from a percentile, or a keep count per block  (Section 3.1 allows a given
+# threshold or a percentile)
 # ---------------------------------------------------------------------------
 def percentile_threshold(w_bits: np.ndarray, block: int, orient: str, rate: float) -> float:
     """Per-matrix threshold for a target compression rate c = total/kept.
