@@ -798,7 +798,7 @@ def run_cuda(args):
                             "tokens per GPU 4096; 16-row blocks; 3.0x compression)",
                 "step": "bsp_prepare_batched (norms+gamma+penalty, keep flags, pack of the 4 matrices, in-place mode: a clearing "
                         "kernel and one kernel that reads W once) then the 4 GEMMs in sequence (bsp_linear_planned_ex on the "
-                        "zero-expanded weights; the single chained launch bsp_linear_chain measured 8 % slower on this "
+                        "zero-expanded weights; the single chained launch bsp_linear_chain measured 6 % slower on this "
                         "workload); one CUDA graph",
                 "l2": f"flushed between steps by writing {L2_FLUSH_BYTES >> 20} MiB",
                 "parallelism": "token split, replicated weights, no collective" if world > 1 else "single GPU",

@@ -380,14 +380,15 @@ int bsp_wait_selftest(int* expired, long long* waited_ns, void* stream);
  *   Y_i = act_i( S_i (W_i * Mask_i)^T + b_i ),  S_i = columns [src_col, src_col + k_in) of X
  *   (src = -1) or of Y_src (0 <= src < i).
  * Row-tile m of an op needs only row-tile m of its source, so no grid-wide barrier separates the
- * layers; see csrc/bsp_linear_chain.cu.  Outputs are bit-identical to calling bsp_linear_planned
- * op by op.
+ * layers: the CTAs take output tiles of all ops from one list through a ticket counter, and a tile
+ * waits (bounded) until the source rows it reads have been stored; see csrc/bsp_linear_chain.cu.
+ * Outputs are bit-identical to calling bsp_linear_planned op by op.
  *
  * ops: HOST array of n_ops (1..8) descriptors; plan / bias / Y are device pointers as in
  * bsp_linear_planned (plan from bsp_linear_plan or bsp_prepare_batched).  ws: device scratch of
- * bsp_linear_chain_ws_bytes bytes, 256-byte aligned (per-row-tile completion counters; cleared by
- * the call).  Needs the alignment of the tensor-core path for every op and for src_col
- * (multiple of 8), else BSP_ERR_UNSUPPORTED; the launch is cooperative (one CTA per SM).
+ * bsp_linear_chain_ws_bytes bytes, 256-byte aligned (per-row-tile completion counters and the
+ * ticket counter; cleared by the call).  Needs the alignment of the tensor-core path for every op
+ * and for src_col (multiple of 8), else BSP_ERR_UNSUPPORTED; one persistent CTA per SM.
  * Bounded waits as bsp_linear_planned: check bsp_linear_status.
  */
 typedef struct bsp_chain_op {

@@ -399,6 +399,7 @@ plan_expand_t_kernel(const int32_t* __restrict__ blk_ptr, const int32_t* __restr
 // ------------------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------------------
+}  // namespace
 // Output-tile width: fewest (waves x per-tile cost) over the candidates.
 int choose_bn(int tokens, int n_out, int sms) {
   const int cands[4] = {256, 192, 128, 64};
@@ -414,6 +415,7 @@ int choose_bn(int tokens, int n_out, int sms) {
   }
   return best_bn;
 }
+namespace {
 
 template <int BN>
 int launch_tc(TcDevice* dev, int slot, const void* plan, const void* X, void* Y, const LinearParams& P, int ldx,

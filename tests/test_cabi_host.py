@@ -118,7 +118,7 @@ def test_argument_errors_are_caught_before_any_launch():
     n = ctypes.c_size_t()
     assert lib.bsp_linear_chain_ws_bytes(0, 128, ctypes.byref(n)) == -1
     assert lib.bsp_linear_chain_ws_bytes(9, 128, ctypes.byref(n)) == -1
-    assert lib.bsp_linear_chain_ws_bytes(4, 4096, ctypes.byref(n)) == 0 and n.value == 512
+    assert lib.bsp_linear_chain_ws_bytes(4, 4096, ctypes.byref(n)) == 0 and n.value == 768   # 4 x 32 counters and the ticket, rounded up to 256
     assert lib.bsp_linear_chain(None, 1, p, 4, 8, ws, 1 << 20, None) == -1
     # zero tokens is a valid no-op
     assert lib.bsp_linear_cuda_core(p, p, p, 8, 8, 4, p, 0, 8, None, 0, p, 8, None) == 0
