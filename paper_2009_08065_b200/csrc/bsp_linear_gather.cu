@@ -419,7 +419,7 @@ linear_gather_kernel(const __grid_constant__ CUtensorMap map_xt, const __grid_co
           }
           if (P.act == BSP_ACT_GELU) {
 #pragma unroll
-            for (int i = 0; i < 16; ++i) f[i] = gelu_erf(f[i]);
+            for (int i = 0; i < 16; i += 2) gelu_erf_pair(f[i], f[i + 1]);
           }
           if (P.transposed) {
             // output row n = rb * D + c0 + i holds this thread's token in column t: the 32 lanes of a warp

@@ -256,6 +256,39 @@ __device__ __forceinline__ float gelu_erf(float x) {
   return fmaf(-fabsf(x), q, fmaxf(x, 0.0f));
 }
 
+// Two float32 values as one 64-bit register pair, and the packed float32 FMA of this architecture
+// (fma.rn.f32x2: two independent correctly rounded FMAs in one instruction, so a result is bit for
+// bit what fmaf gives).
+__device__ __forceinline__ unsigned long long pack_f32x2(float lo, float hi) {
+  unsigned long long r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack_f32x2(unsigned long long v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ unsigned long long fma_f32x2(unsigned long long a, unsigned long long b, unsigned long long c) {
+  unsigned long long d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+// gelu_erf for two values at once: the same operations in the same order per value, with the five
+// polynomial steps issued as packed FMAs (the epilogue of a GELU layer is bound by instruction issue).
+__device__ __forceinline__ void gelu_erf_pair(float& x0, float& x1) {
+  const unsigned long long a = pack_f32x2(fminf(fabsf(x0), 6.0f), fminf(fabsf(x1), 6.0f));
+  unsigned long long p = fma_f32x2(pack_f32x2(-0.000518865308f, -0.000518865308f), a, pack_f32x2(0.00738722592f, 0.00738722592f));
+  p = fma_f32x2(p, a, pack_f32x2(-0.0525380379f, -0.0525380379f));
+  p = fma_f32x2(p, a, pack_f32x2(-0.459276694f, -0.459276694f));
+  p = fma_f32x2(p, a, pack_f32x2(-1.15108313f, -1.15108313f));
+  p = fma_f32x2(p, a, pack_f32x2(-1.00000084f, -1.00000084f));
+  float p0, p1, q0, q1;
+  unpack_f32x2(p, p0, p1);
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(q0) : "f"(p0));
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(q1) : "f"(p1));
+  x0 = fmaf(-fabsf(x0), q0, fmaxf(x0, 0.0f));
+  x1 = fmaf(-fabsf(x1), q1, fmaxf(x1, 0.0f));
+}
+
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   uint32_t r;
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));   // upper half <- first source
@@ -292,7 +325,7 @@ __device__ __forceinline__ void piece_store(const EpiloguePiece& p, int act, uin
     }
     if (act == BSP_ACT_GELU) {
 #pragma unroll
-      for (int i = 0; i < 8; ++i) f[i] = gelu_erf(f[i]);
+      for (int i = 0; i < 8; i += 2) gelu_erf_pair(f[i], f[i + 1]);
     }
     st_shared_v4(dst_row + ((static_cast<uint32_t>(j) ^ row_xor) << 4), pack_bf16x2(f[0], f[1]), pack_bf16x2(f[2], f[3]),
                  pack_bf16x2(f[4], f[5]), pack_bf16x2(f[6], f[7]));
@@ -314,7 +347,7 @@ __device__ __forceinline__ void piece_store_transposed(const EpiloguePiece& p, i
     }
     if (act == BSP_ACT_GELU) {
 #pragma unroll
-      for (int i = 0; i < 8; ++i) f[i] = gelu_erf(f[i]);
+      for (int i = 0; i < 8; i += 2) gelu_erf_pair(f[i], f[i + 1]);
     }
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
