@@ -57,6 +57,7 @@ struct StreamBatchT {
   float eps;
   int total_items, buf_bytes;
   int parts_total;           // column ranges of one round over every matrix of the batch
+  int sms, stagger_ns;       // start of the CTAs that share an SM, one after the other (ticket variant)
   int* ticket;
   int* status;               // receives BSP_ERR_TIMEOUT when a bounded wait expires
   // Item order (see locate): the table is sorted by row-block count; a matrix's "segment" is the run of
@@ -237,7 +238,17 @@ fused_stream_kernel(const __grid_constant__ StreamBatchT<N> B) {
     // kernel; the ticket and the slots it zeroes are touched only from here on
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel may set up on SMs that become free
-    if (!direct) s_item = atomicAdd(B.ticket, 1);
+    if (!direct) {
+      // CTAs that start together and work on items of one size stay in step: all of an SM's CTAs load,
+      // then all compute.  The k-th CTA of an SM (block numbers go round the SMs) therefore takes its
+      // first ticket k * stagger later, so that loads and arithmetic of different CTAs overlap.
+      const unsigned long long delay = static_cast<unsigned long long>(blockIdx.x / B.sms) * B.stagger_ns;
+      if (delay) {
+        const unsigned long long t0 = tc::global_timer_ns();
+        while (tc::global_timer_ns() - t0 < delay) __nanosleep(100);
+      }
+      s_item = atomicAdd(B.ticket, 1);
+    }
   }
   __syncthreads();
   if (!direct) {
@@ -682,6 +693,10 @@ int fused_stream(const FusedJob* jobs, int n_jobs, int block, float eps, int squ
     const int n = n_jobs - j0 < kStreamMaxJobs ? n_jobs - j0 : kStreamMaxJobs;
     fill_batch(*B, jobs + j0, n, block, eps, squared, part_counts + j0, part_partial + j0, &smem);
     B->status = td->status;
+    B->sms = td->sms;
+    // (measured on the 72-matrix stack: 80.8 us without, 76.8 / 74.8 / 76.8 / 78.8 us at 400 / 800 / 1200 / 1600 ns;
+    // a batch of only a few waves would lose more at the start than it gains)
+    B->stagger_ns = B->total_items >= 4 * per_sm * td->sms ? 750 : 0;
     if (B->total_items <= per_sm * td->sms) B->ticket = nullptr;    // one wave: item = block index
     const bool few = n <= kStreamFewJobs;
     StreamBatchT<kStreamFewJobs> small;
