@@ -2,8 +2,9 @@
 // read from HBM exactly once.
 //
 // A work item is one row-block of one matrix (or a column range of it, so that its rows fit 24 KB
-// of shared memory).  Every CTA takes one item from a ticket counter, so every item with a smaller
-// number has been taken, and is being worked on, before.  The CTA
+// of shared memory).  Items are numbered round by round across the matrices of the batch (see
+// locate).  A CTA takes items from a ticket counter, so every item with a smaller number has been
+// taken, and is being worked on, before; for each item it
 //   load     has the item's rows brought into shared memory by bulk asynchronous copies (one per
 //            row, all in flight at once, completion on an mbarrier);
 //   phase A  computes the float32 sums of squares from shared memory (rows in increasing order, the
@@ -14,13 +15,17 @@
 //   phase B  reads the published counts of the items before it in the same matrix (bounded
 //            relaxed loads), which give blk_ptr and the position of its part of the packed tile,
 //            and writes indices and tile from shared memory.
-// Shared memory per CTA is small (26 KB at 16-row blocks), so eight CTAs share an SM and their
+// Shared memory per CTA is small (27 KB at 16-row blocks), so eight CTAs share an SM and their
 // phases overlap: the latency of one item's chain is hidden by the other seven.
 // Why this cannot deadlock: a published count depends on nobody, and a taken item is published
 // without waiting.  An item waits for items with a smaller number (all taken) and, when its
-// row-block is split into column ranges, for the later ranges of its own block; at most one block
-// straddles the ticket counter, so fewer than 32 CTAs can wait for items nobody has taken, and the
-// GPU holds more CTAs than that at once.
+// row-block is split into column ranges, for the later ranges of its own block, which are the next
+// tickets; at most one block straddles the ticket counter, so fewer than 32 CTAs can wait for items
+// nobody has taken, and the GPU holds more CTAs than that at once.  A CTA takes its next ticket only
+// after the last wait of its current item, so a ticket is never held by a CTA that is waiting.
+// A batch of at most one wave of CTAs runs without the counter (item = block index): it relies on
+// the hardware starting the blocks of a grid in index order, as it does; were that ever not so, the
+// bounded waits would end the launch with BSP_ERR_TIMEOUT rather than hang it.
 // Counts and penalty partials are published as single words that carry their own "ready" bit (the
 // lowest mantissa bit of the float64 partial), read with relaxed loads: a reader needs nothing but
 // the word itself, so no fence is involved.  The last item of a matrix adds the partials in a fixed
