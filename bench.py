@@ -616,6 +616,31 @@ def other_workloads(device, peaks, args):
     return out
 
 
+TRAFFIC_PROFILE = os.path.join("profiles", "linear_tc_kernel_bert_base_T4096.md")
+TRAFFIC_SOURCES = ("paper_2009_08065_b200/csrc/bsp_linear_tc.cu", "paper_2009_08065_b200/csrc/bsp_tc.cuh")
+
+
+def profiled_traffic():
+    """DRAM bytes (read + write) of the four GEMM launches as ncu counted them, from the `traffic-record` line of
+    the kernel's profile summary, or None when the kernel's sources have changed since that capture (the line
+    carries their SHA-256) or the record is missing."""
+    import hashlib
+    root = os.path.dirname(os.path.abspath(__file__))
+    try:
+        h = hashlib.sha256()
+        for f in TRAFFIC_SOURCES:
+            with open(os.path.join(root, f), "rb") as fh:
+                h.update(fh.read())
+        with open(os.path.join(root, TRAFFIC_PROFILE)) as fh:
+            line = next(l for l in fh if l.startswith("traffic-record:"))
+        rec = dict(kv.split("=", 1) for kv in line.split(":", 1)[1].split())
+        if rec.get("sha256") != h.hexdigest():
+            return None
+        return {k: int(v) for k, v in rec.items() if k != "sha256"}
+    except (OSError, StopIteration, ValueError):
+        return None
+
+
 def section_8d_bytes(tokens, spec, kept_weights):
     """Algorithmic bytes of one pruned linear: X once, the kept values and one index per kept group, Y once, the bias."""
     return (2 * tokens * spec.k_in + 2 * kept_weights + 4 * (kept_weights // spec.block)
@@ -789,6 +814,9 @@ def run_cuda(args):
         hbm_binds = t_hbm >= t_tensor
         ach_tf, ach_gbs = step_flops / gemm_total / 1e9, sum(alg_bytes) / gemm_total / 1e6
         names = [e["spec"].name.split(".")[1] for e in layer.lin]
+        traffic = profiled_traffic()
+        if traffic is not None and sorted(traffic) != sorted(names):
+            traffic = None
         line = {
             "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": round(total_ms / args.steps, 5), "higher_is_better": True,
@@ -837,9 +865,11 @@ def run_cuda(args):
                        "step, every prefix its own CUDA graph replayed after an L2 flush in the timed loop",
                 "algorithmic_bytes": sum(alg_bytes),
                 "algorithmic_bytes_formula": "per linear 2TK + 2 kept + 4 kept/d + 2TN + 2N (X once, kept values, one index per kept group, Y once, bias)",
-                "traffic": None,
-                "traffic_note": "dram bytes of the four launches are in profiles/linear_tc_kernel_bert_base_T4096.md (one ncu capture per launch); "
-                                "not re-measured by this run",
+                "traffic": sum(traffic.values()) if traffic else None,
+                "traffic_per_launch": traffic,
+                "traffic_note": "dram__bytes_read.sum + dram__bytes_write.sum of the four launches, one ncu capture per launch of "
+                                "`bench.py --case <linear>` (" + TRAFFIC_PROFILE + "); not re-measured by this run, and null when the "
+                                "kernel's sources no longer match the hash recorded with that capture",
                 "peak_source": f"{'hbm_gbs' if hbm_binds else 'bf16_tflops burst'}, {peak_src}",
                 "weight_side_ms": round(weight_ms, 5),
                 "per_launch": {names[i]: {"ms": round(share[i], 5), "nonzero_tflops": round(flops[i] / share[i] / 1e9, 1),
