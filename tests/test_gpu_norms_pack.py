@@ -303,6 +303,42 @@ def test_prepare_batched_streaming_batch_larger_than_the_gpu():
             job.penalty.fill_(-5.0)
 
 
+@pytest.mark.parametrize("block,n_jobs,seed", [(16, 40, 900), (8, 9, 901), (32, 7, 902)])
+def test_prepare_batched_matrices_of_unequal_sizes(block, n_jobs, seed):
+    """Matrices with different row-block counts and widths (some split into column ranges, some of one
+    block) in one call: items are numbered round by round across the matrices, and the rounds thin
+    out as the short matrices run out.  40 matrices make several waves (tickets); 9 and 7 fit one wave.
+    Odd kept counts per block exercise the unaligned tile paths.  Pack against the oracle, bit for bit."""
+    rng = np.random.default_rng(seed)
+    eps = 1e-3
+    jobs, refs = [], []
+    for n in range(n_jobs):
+        rows = block * int(rng.choice([1, 2, 3, 5, 24, 48, 96]))
+        cols = 8 * int(rng.choice([1, 3, 12, 96, 97, 200, 384]))
+        w = si.student_t_bf16(seed + n, f"mixed{n}", (rows, cols), 3.0, 0.02)
+        t_b = float(np.quantile(O.group_norms(w, block, "C"), float(rng.uniform(0.1, 0.9))))
+        pk = bsp.PackedMatrix.allocate(rows, cols, block, bsp.ORIENT_C, DEV)
+        pk.idx.fill_(-7)
+        jobs.append(bsp.LayerJob(W=to_dev(w), out=pk, threshold=t_b,
+                                 penalty=torch.full((1,), -5.0, dtype=torch.float64, device=DEV)))
+        refs.append((w, t_b))
+    for _ in range(2):                                   # the second call starts from the first one's scratch
+        bsp.bsp_prepare_batched(jobs, block, eps, bsp.PEN_L2)
+        bsp.bsp_linear_status()
+        torch.cuda.synchronize()
+        for job, (w, t_b) in zip(jobs, refs):
+            keep_ref = O.keep_flags(w, block, "C", t_b)
+            ref_ptr, ref_idx, ref_vals = O.pack(w, keep_ref, block, "C")
+            blk_ptr, idx, vals, keep, kept = packed_to_host(job.out)
+            assert np.array_equal(keep, keep_ref) and np.array_equal(blk_ptr, ref_ptr)
+            assert np.array_equal(idx, ref_idx) and np.array_equal(vals, ref_vals)
+            assert kept == block * int(keep_ref.sum())
+            n_ref = O.group_norms(w, block, "C")
+            assert float(job.penalty.item()) == pytest.approx(O.penalty_l2(n_ref, O.gamma_update(n_ref, eps)), rel=REL)
+            job.out.idx.fill_(-7)
+            job.penalty.fill_(-5.0)
+
+
 def test_prepare_batched_in_place_masks_w_and_writes_nothing_else():
     """A job whose plan is its W: the pruned groups are zeroed inside W (Algorithm 2's W = W * Mask), every other
     output is what the separate-plan call gives, a second call on the now-masked W with threshold 0 leaves W
