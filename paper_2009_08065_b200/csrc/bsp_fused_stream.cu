@@ -235,10 +235,19 @@ fused_stream_kernel(const __grid_constant__ StreamBatchT<N> B) {
     const FusedJob& J0 = B.job[I.jn].j;
     asm volatile("" ::"l"(J0.W), "r"(J0.ldw), "l"(J0.flags), "l"(J0.vals), "l"(B.job[I.jn].part_counts));
   }
+  if (warp == 0) {
+    if (lane == 0) {
+      mbar_init(bar, 1);
+      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncwarp();
+    // One wave: the rows are asked for before the wait for the clearing kernel.  That kernel is an
+    // ordinary launch, so whatever wrote W earlier in the stream had finished before it began, and
+    // this grid was started after that; only the published counts depend on the clearing itself.
+    if (direct) issue_rows(B, I, smem_u32(s_raw), bar, lane);
+  }
   if (threadIdx.x == 0) {
-    mbar_init(bar, 1);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     // launched with programmatic stream serialization: everything above overlapped the clearing
     // kernel; the ticket and the slots it zeroes are touched only from here on
     asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -267,7 +276,7 @@ fused_stream_kernel(const __grid_constant__ StreamBatchT<N> B) {
   // counter overlaps those writes.
   uint32_t parity = 0u;
   for (;;) {
-    if (warp == 0) issue_rows(B, I, smem_u32(s_raw), bar, lane);
+    if (warp == 0 && !direct) issue_rows(B, I, smem_u32(s_raw), bar, lane);
     const StreamJob& O = B.job[I.jn];
     const FusedJob& J = O.j;
     const int b = I.b, q = I.q, c0 = I.c0, pc = I.pc, local = I.local;
