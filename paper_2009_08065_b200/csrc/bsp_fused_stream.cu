@@ -699,8 +699,12 @@ int fused_stream(const FusedJob* jobs, int n_jobs, int block, float eps, int squ
       if (e != cudaSuccess) { delete B; return cuda_fail(e); }
       td->attr_set[7] = true;
     }
+    int per_sm_one_wave = 0;
     cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fused_stream_kernel<kStreamMaxJobs, false>, kStreamThreads, smem_max);
+    if (e == cudaSuccess)
+      e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm_one_wave, fused_stream_kernel<kStreamMaxJobs, true>, kStreamThreads, smem_max);
     if (e != cudaSuccess) { delete B; return cuda_fail(e); }
+    if (per_sm_one_wave < per_sm) per_sm = per_sm_one_wave;      // "one wave" must hold for the variant that assumes it
     if (per_sm * td->sms < 32) ok = false;    // the no-deadlock argument needs 32 CTAs resident at once
   }
   for (int j0 = 0; j0 < n_jobs && ok && st == BSP_OK; j0 += kStreamMaxJobs) {
