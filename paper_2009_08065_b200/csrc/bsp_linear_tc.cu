@@ -561,13 +561,15 @@ extern "C" int bsp_linear_planned_ex(const void* plan, int n_out, int k_in, int 
   TcDevice* dev = tc_device();
   if (dev == nullptr) return BSP_ERR_CUDA;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  // Measured on B200: CTA pairs win (about 5 %) once the problem runs for many waves, where the L2 -> SM
-  // operand traffic binds; for a few waves the one-CTA kernel's shorter start-up wins (about 2 us).
+  // Measured on B200, single launches after an L2 flush: without GELU the CTA-pair kernel is level or ahead
+  // from about 1.25 x #SM pair-tiles on (8192 tokens x 2304 outputs: 3 %; 16384 x 768: 3-9 %; 32768 tokens: 4-11 %;
+  // a 1024 x 4096 weight at 16384 tokens: 30 %, the one-CTA kernel's last wave being half empty there) and behind
+  // below that (one encoder layer at 4096 tokens: +0 to +4 us per launch; 8192 x 768 x 768: +13 %), where its
+  // longer start-up shows.  With GELU the epilogue is the longer side of a tile and the two are level on average
+  // (0.92-1.05 over six shapes), so those launches stay with the one-CTA kernel.
   const long long pair_tiles = static_cast<long long>((tokens + 255) / 256) * ((n_out + 255) / 256);
-  // With GELU the epilogue is the longer side of a tile and the one-CTA kernel's slower main loop hides
-  // more of it: 202 us against 209 us at 32768 x 4096 x 1024.
   const bool pair = algo == BSP_LINEAR_CTA_PAIR ||
-                    (algo == BSP_LINEAR_AUTO && pair_tiles >= 4LL * dev->sms && act == BSP_ACT_NONE && !transposed);
+                    (algo == BSP_LINEAR_AUTO && 4 * pair_tiles >= 5LL * dev->sms && act == BSP_ACT_NONE && !transposed);
   if (pair) return launch_tc_pair(dev, plan, X, Y, tokens, n_out, k_in, act, bias, ldx, ldy, s);
   LinearParams P{tokens, n_out, k_in, act, (algo_flags & BSP_LINEAR_PLAN_STABLE) ? 1 : 0, transposed ? 1 : 0,
                  static_cast<const uint16_t*>(bias), dev->status};
